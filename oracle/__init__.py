@@ -1,0 +1,180 @@
+"""TEST INFRASTRUCTURE -- ctypes front end of the CPU oracle (`comet_oracle.cpp`).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It shares nothing with the CUDA library.  Arrays are numpy
+uint64, C-contiguous, in the paper's mathematical shapes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "comet_oracle.cpp")
+_LIB = os.path.join(_HERE, "libcomet_oracle.so")
+_lib = None
+
+U64 = np.uint64
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (plain -O2, no threading, no arch flags)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", _LIB, _SRC])
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a: np.ndarray):
+    assert a.flags["C_CONTIGUOUS"], "oracle arrays must be C-contiguous"
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _u64(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == U64
+    return a
+
+
+def reconstruct(s0, s1):
+    s0, s1 = _u64(s0), _u64(s1)
+    out = np.empty_like(s0)
+    lib().orc_reconstruct(_p(s0), _p(s1), _p(out), ctypes.c_size_t(s0.size))
+    return out
+
+
+def index_set(block_mask, block: int, groups: int = 1) -> np.ndarray:
+    m = np.ascontiguousarray(block_mask, dtype=np.uint8)
+    I = np.empty(max(1, m.size * block * groups), dtype=np.int32)
+    n = lib().orc_index_set(_p(m), ctypes.c_int(m.size), ctypes.c_int(block), ctypes.c_int(groups), _p(I))
+    return I[:n].copy()
+
+
+def index_cols(Y, I):
+    Y = _u64(Y)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    K, D = Y.shape
+    out = np.empty((K, I.size), dtype=U64)
+    lib().orc_index_cols(_p(Y), ctypes.c_int(K), ctypes.c_int(D), _p(I), ctypes.c_int(I.size), _p(out))
+    return out
+
+
+def index_rows(Y, I):
+    Y = _u64(Y)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    D, N = Y.shape
+    out = np.empty((I.size, N), dtype=U64)
+    lib().orc_index_rows(_p(Y), ctypes.c_int(N), _p(I), ctypes.c_int(I.size), _p(out))
+    return out
+
+
+def merge_cols(R, I, D: int):
+    R = _u64(R)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    T, n = R.shape
+    Z = np.empty((T, D), dtype=U64)
+    lib().orc_merge_cols(_p(R), ctypes.c_int(T), ctypes.c_int(n), _p(I), ctypes.c_int(D), _p(Z))
+    return Z
+
+
+def mask_operand(share, mask_share):
+    share, mask_share = _u64(share), _u64(mask_share)
+    assert share.shape == mask_share.shape
+    out = np.empty_like(share)
+    lib().orc_mask_operand(_p(share), _p(mask_share), _p(out), ctypes.c_size_t(share.size))
+    return out
+
+
+def beaver_combine(party: int, E, F, Ai, Bi, Ci):
+    E, F, Ai, Bi, Ci = map(_u64, (E, F, Ai, Bi, Ci))
+    T, K = E.shape
+    K2, N = F.shape
+    assert K2 == K and Ai.shape == (T, K) and Bi.shape == (K, N) and Ci.shape == (T, N)
+    Z = np.empty((T, N), dtype=U64)
+    lib().orc_beaver_combine(ctypes.c_int(party), ctypes.c_int(T), ctypes.c_int(K), ctypes.c_int(N),
+                             _p(E), _p(F), _p(Ai), _p(Bi), _p(Ci), _p(Z))
+    return Z
+
+
+def beaver_combine_at(party: int, E, F, Ai, Bi, Ci, rows, cols):
+    E, F, Ai, Bi, Ci = map(_u64, (E, F, Ai, Bi, Ci))
+    T, K = E.shape
+    _, N = F.shape
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    cols = np.ascontiguousarray(cols, dtype=np.int32)
+    out = np.empty(rows.size, dtype=U64)
+    lib().orc_beaver_combine_at(ctypes.c_int(party), ctypes.c_int(K), ctypes.c_int(N),
+                                _p(E), _p(F), _p(Ai), _p(Bi), _p(Ci),
+                                ctypes.c_int(rows.size), _p(rows), _p(cols), _p(out))
+    return out
+
+
+def _pairs(*pairs):
+    flat = []
+    for s0, s1 in pairs:
+        flat += [_u64(s0), _u64(s1)]
+    return flat
+
+
+def pi_matmul(X, Y, A, B, C):
+    """Both parties of Pi_MatMul.  Each argument is a pair (share0, share1).
+    Returns dict with E, F, Z pairs."""
+    X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1 = _pairs(X, Y, A, B, C)
+    T, K = X0.shape
+    _, N = Y0.shape
+    E0, E1 = np.empty((T, K), U64), np.empty((T, K), U64)
+    F0, F1 = np.empty((K, N), U64), np.empty((K, N), U64)
+    Z0, Z1 = np.empty((T, N), U64), np.empty((T, N), U64)
+    lib().orc_pi_matmul(ctypes.c_int(T), ctypes.c_int(K), ctypes.c_int(N),
+                        *[_p(a) for a in (X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, Z0, Z1)])
+    return {"E": (E0, E1), "F": (F0, F1), "Z": (Z0, Z1)}
+
+
+def somm(X, Y, I, A, B, C):
+    """Protocol 2 with a token-shared mask.  Y pair is [K, Dy]; I indexes its
+    columns.  Returns compact messages and result: E [T,K], F [K,n], R [T,n]."""
+    X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1 = _pairs(X, Y, A, B, C)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    T, K = X0.shape
+    _, Dy = Y0.shape
+    n = I.size
+    assert A0.shape == (T, K) and B0.shape == (K, n) and C0.shape == (T, n)
+    E0, E1 = np.empty((T, K), U64), np.empty((T, K), U64)
+    F0, F1 = np.empty((K, n), U64), np.empty((K, n), U64)
+    R0, R1 = np.empty((T, n), U64), np.empty((T, n), U64)
+    lib().orc_somm(ctypes.c_int(T), ctypes.c_int(K), ctypes.c_int(Dy), _p(I), ctypes.c_int(n),
+                   *[_p(a) for a in (X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, R0, R1)])
+    return {"E": (E0, E1), "F": (F0, F1), "Z": (R0, R1)}
+
+
+def simm(X, Y, I, A, B, C):
+    """Protocol 3 with a token-shared mask.  X pair is compact [T,n]; Y pair is
+    [D, N]; I lists the neuron of each compact column.  Returns E [T,n],
+    F [n,N], Z [T,N]."""
+    X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1 = _pairs(X, Y, A, B, C)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    T, n = X0.shape
+    _, N = Y0.shape
+    assert I.size == n and A0.shape == (T, n) and B0.shape == (n, N) and C0.shape == (T, N)
+    E0, E1 = np.empty((T, n), U64), np.empty((T, n), U64)
+    F0, F1 = np.empty((n, N), U64), np.empty((n, N), U64)
+    Z0, Z1 = np.empty((T, N), U64), np.empty((T, N), U64)
+    lib().orc_simm(ctypes.c_int(T), ctypes.c_int(n), ctypes.c_int(N), _p(I),
+                   *[_p(a) for a in (X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, Z0, Z1)])
+    return {"E": (E0, E1), "F": (F0, F1), "Z": (Z0, Z1)}
+
+
+def truncate(party: int, Z, frac_bits: int):
+    Z = _u64(Z)
+    out = np.empty_like(Z)
+    lib().orc_truncate(ctypes.c_int(party), _p(Z), _p(out), ctypes.c_size_t(Z.size), ctypes.c_int(frac_bits))
+    return out

@@ -1,0 +1,223 @@
+// TEST INFRASTRUCTURE -- not part of the product.
+//
+// Plain, slow, single-threaded CPU statement of what the sparse secret-shared
+// FFN path computes, written from the paper (arXiv 2505.07239, "Comet") in the
+// paper's order and notation.  It shares no code with the CUDA library, is
+// never tuned, and is only ever called by the tests, by the smoke check and by
+// the benchmark's CPU-baseline leg.
+//
+// Ring: Z_{2^64}; every value is a uint64_t and C++ unsigned arithmetic is the
+// ring arithmetic.  Matrices are row-major in the paper's mathematical shapes
+// (X is [rows, inner], Y is [inner, cols]).  Parties: the paper's P_1, P_2 are
+// i = 0, 1 here, so the paper's factor (i-1) in Eq. 1 is the factor i.
+//
+// Pins (see tests/test_oracle_*.py): Eq. 1 reconstructs the plaintext product
+// for any triple with c = ab (checked against Python big integers and numpy);
+// all-ones mask == dense; masked neurons contribute exactly zero; truncation
+// closed forms and the {0,1}-ulp invariant; hand-computed fixtures.
+// Parity unpinned: the individual share values Z_i (as opposed to their sum)
+// are fixed only by Eq. 1 itself plus this repository's seeded inputs.
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+typedef uint64_t u64;
+
+extern "C" {
+
+// ---------------------------------------------------------------------------
+// Section 2.1, "Additive secret sharing": reconstruction x = [x]_1 + [x]_2.
+// ---------------------------------------------------------------------------
+void orc_reconstruct(const u64* s0, const u64* s1, u64* out, size_t count) {
+    for (size_t t = 0; t < count; ++t) out[t] = s0[t] + s1[t];
+}
+
+// ---------------------------------------------------------------------------
+// Index sets.  Protocol 2 line 3 (I_y of the single connected component) and
+// Protocol 3 lines 1-5 (the nonzero columns j) for a sparsity distribution
+// that is one block mask shared by all tokens: neuron j is active iff
+// block_mask[j / bs] != 0.  With `groups` = 2 (gated FFN, Y = [W_gate || W_up]
+// of width 2*D) the set is I followed by D + I.  Ascending order.
+// Returns the number of indices written.
+// ---------------------------------------------------------------------------
+int orc_index_set(const uint8_t* block_mask, int nb, int bs, int groups, int32_t* I) {
+    int D = nb * bs;
+    int count = 0;
+    for (int g = 0; g < groups; ++g)
+        for (int j = 0; j < D; ++j)
+            if (block_mask[j / bs] != 0) I[count++] = g * D + j;
+    return count;
+}
+
+// Protocol 2 line 5: IndexCols(Y, I_y).  Y is [K, D]; out is [K, n].
+void orc_index_cols(const u64* Y, int K, int D, const int32_t* I, int n, u64* out) {
+    for (int k = 0; k < K; ++k)
+        for (int c = 0; c < n; ++c) out[(size_t)k * n + c] = Y[(size_t)k * D + I[c]];
+}
+
+// Protocol 3 line 9: IndexRow(Y, j) for every j in I.  Y is [D, N]; out is [n, N].
+void orc_index_rows(const u64* Y, int N, const int32_t* I, int n, u64* out) {
+    for (int r = 0; r < n; ++r)
+        for (int c = 0; c < N; ++c) out[(size_t)r * N + c] = Y[(size_t)I[r] * N + c];
+}
+
+// Protocol 2 line 8, Merge: compact columns back to a dense [T, D] layout,
+// zero (in this share) at every inactive position.
+void orc_merge_cols(const u64* R, int T, int n, const int32_t* I, int D, u64* Z) {
+    for (size_t t = 0; t < (size_t)T * D; ++t) Z[t] = 0;
+    for (int r = 0; r < T; ++r)
+        for (int c = 0; c < n; ++c) Z[(size_t)r * D + I[c]] = R[(size_t)r * n + c];
+}
+
+// ---------------------------------------------------------------------------
+// Pi_MatMul, the matrix form of Eq. 1, one party's side.
+//
+// Step 1 (before the exchange), Section 2.1 "Multiplication" / Section 5.1:
+//   [E]_i = [X]_i - [A]_i,   [F]_i = [Y]_i - [B]_i.
+// ---------------------------------------------------------------------------
+void orc_mask_operand(const u64* share, const u64* mask_share, u64* out, size_t count) {
+    for (size_t t = 0; t < count; ++t) out[t] = share[t] - mask_share[t];
+}
+
+// Plain ring product P = L * R, L [T,K], R [K,N] (accumulating row by row).
+static void ring_product(const u64* L, const u64* R, int T, int K, int N, u64* P) {
+    for (size_t t = 0; t < (size_t)T * N; ++t) P[t] = 0;
+    for (int r = 0; r < T; ++r)
+        for (int k = 0; k < K; ++k) {
+            u64 l = L[(size_t)r * K + k];
+            const u64* Rrow = R + (size_t)k * N;
+            u64* Prow = P + (size_t)r * N;
+            for (int c = 0; c < N; ++c) Prow[c] += l * Rrow[c];
+        }
+}
+
+// Step 2 (after the exchange): E = [E]_0 + [E]_1 and F = [F]_0 + [F]_1 are
+// public, and Eq. 1 with d -> E (left), e -> F (right) reads
+//   [Z]_i = [C]_i + E * [B]_i + [A]_i * F + i * (E * F),
+// three separate products, exactly as the equation is printed.
+void orc_beaver_combine(int party, int T, int K, int N, const u64* E, const u64* F,
+                        const u64* Ai, const u64* Bi, const u64* Ci, u64* Zi) {
+    std::vector<u64> EB((size_t)T * N), AF((size_t)T * N), EF((size_t)T * N);
+    ring_product(E, Bi, T, K, N, EB.data());
+    ring_product(Ai, F, T, K, N, AF.data());
+    ring_product(E, F, T, K, N, EF.data());
+    for (size_t t = 0; t < (size_t)T * N; ++t)
+        Zi[t] = Ci[t] + EB[t] + AF[t] + (u64)party * EF[t];
+}
+
+// The same Eq. 1 evaluated at a list of output positions only (one dot product
+// triple per sample), for sizes where the full product is too slow on a CPU.
+void orc_beaver_combine_at(int party, int K, int N, const u64* E, const u64* F,
+                           const u64* Ai, const u64* Bi, const u64* Ci,
+                           int n_samples, const int32_t* rows, const int32_t* cols, u64* out) {
+    for (int s = 0; s < n_samples; ++s) {
+        int r = rows[s], c = cols[s];
+        u64 eb = 0, af = 0, ef = 0;
+        for (int k = 0; k < K; ++k) {
+            u64 e = E[(size_t)r * K + k], a = Ai[(size_t)r * K + k];
+            u64 f = F[(size_t)k * N + c], b = Bi[(size_t)k * N + c];
+            eb += e * b;
+            af += a * f;
+            ef += e * f;
+        }
+        out[s] = Ci[(size_t)r * N + c] + eb + af + (u64)party * ef;
+    }
+}
+
+// Both parties of one Pi_MatMul call.  Inputs are pairs of shares (index 0/1).
+// Outputs: the four messages and the two result shares.
+void orc_pi_matmul(int T, int K, int N,
+                   const u64* X0, const u64* X1, const u64* Y0, const u64* Y1,
+                   const u64* A0, const u64* A1, const u64* B0, const u64* B1,
+                   const u64* C0, const u64* C1,
+                   u64* E0, u64* E1, u64* F0, u64* F1, u64* Z0, u64* Z1) {
+    size_t nx = (size_t)T * K, ny = (size_t)K * N;
+    orc_mask_operand(X0, A0, E0, nx);
+    orc_mask_operand(X1, A1, E1, nx);
+    orc_mask_operand(Y0, B0, F0, ny);
+    orc_mask_operand(Y1, B1, F1, ny);
+    std::vector<u64> E(nx), F(ny);
+    orc_reconstruct(E0, E1, E.data(), nx);   // the exchange
+    orc_reconstruct(F0, F1, F.data(), ny);
+    orc_beaver_combine(0, T, K, N, E.data(), F.data(), A0, B0, C0, Z0);
+    orc_beaver_combine(1, T, K, N, E.data(), F.data(), A1, B1, C1, Z1);
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 2 (SOMM) for a token-shared mask: the bipartite graph is complete
+// between all T rows of X and the active columns, i.e. one connected
+// component with I_x = all rows, I_y = I.  Y is [K, Dy] (Dy = groups * d_ff).
+// Outputs are compact: messages E_i [T,K], F_i [K,n]; result R_i [T,n].
+// ---------------------------------------------------------------------------
+void orc_somm(int T, int K, int Dy, const int32_t* I, int n,
+              const u64* X0, const u64* X1, const u64* Y0, const u64* Y1,
+              const u64* A0, const u64* A1, const u64* B0, const u64* B1,
+              const u64* C0, const u64* C1,
+              u64* E0, u64* E1, u64* F0, u64* F1, u64* R0, u64* R1) {
+    std::vector<u64> Yt0((size_t)K * n), Yt1((size_t)K * n);
+    orc_index_cols(Y0, K, Dy, I, n, Yt0.data());          // line 5
+    orc_index_cols(Y1, K, Dy, I, n, Yt1.data());
+    orc_pi_matmul(T, K, n, X0, X1, Yt0.data(), Yt1.data(), // line 6
+                  A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, R0, R1);
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 3 (SIMM), column by row.  X here is already compact, [T, n], its
+// column c standing for neuron I[c]; R_j is all T rows for every nonzero
+// column (token-shared mask).  Each column's Pi_MatMul is the outer product of
+// a T-vector with row I[c] of Y [D, N]; it uses column c of A' [T,n] and row c
+// of B' [n,N] as its (a_j, b_j), and the dealer's C' [T,N] is the sum over j
+// of the per-column c_j = a_j b_j^T, added once in Merge&Sum (line 12).
+// Outputs: messages E_i [T,n], F_i [n,N]; result Z_i [T,N].
+// ---------------------------------------------------------------------------
+void orc_simm(int T, int n, int N, const int32_t* I,
+              const u64* X0, const u64* X1, const u64* Y0, const u64* Y1,
+              const u64* A0, const u64* A1, const u64* B0, const u64* B1,
+              const u64* C0, const u64* C1,
+              u64* E0, u64* E1, u64* F0, u64* F1, u64* Z0, u64* Z1) {
+    const u64* Xs[2] = {X0, X1};
+    const u64* Ys[2] = {Y0, Y1};
+    const u64* As[2] = {A0, A1};
+    const u64* Bs[2] = {B0, B1};
+    const u64* Cs[2] = {C0, C1};
+    u64* Es[2] = {E0, E1};
+    u64* Fs[2] = {F0, F1};
+    u64* Zs[2] = {Z0, Z1};
+    for (int i = 0; i < 2; ++i)
+        for (size_t t = 0; t < (size_t)T * N; ++t) Zs[i][t] = Cs[i][t];
+    std::vector<u64> e(T), f(N);
+    for (int c = 0; c < n; ++c) {                    // lines 6-11, one column j = I[c]
+        int j = I[c];
+        for (int i = 0; i < 2; ++i) {
+            for (int r = 0; r < T; ++r)              // lines 7-8 + masking of x''
+                Es[i][(size_t)r * n + c] = Xs[i][(size_t)r * n + c] - As[i][(size_t)r * n + c];
+            for (int q = 0; q < N; ++q)              // line 9 + masking of y
+                Fs[i][(size_t)c * N + q] = Ys[i][(size_t)j * N + q] - Bs[i][(size_t)c * N + q];
+        }
+        for (int r = 0; r < T; ++r) e[r] = E0[(size_t)r * n + c] + E1[(size_t)r * n + c];
+        for (int q = 0; q < N; ++q) f[q] = F0[(size_t)c * N + q] + F1[(size_t)c * N + q];
+        for (int i = 0; i < 2; ++i)                  // line 10 (Eq. 1 without c_j) + line 12 sum
+            for (int r = 0; r < T; ++r) {
+                u64 a = As[i][(size_t)r * n + c];
+                for (int q = 0; q < N; ++q) {
+                    u64 b = Bs[i][(size_t)c * N + q];
+                    Zs[i][(size_t)r * N + q] += e[r] * b + a * f[q] + (u64)i * (e[r] * f[q]);
+                }
+            }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Local fixed-point truncation by f bits (the paper is silent; two-party local
+// truncation on the unsigned words): party 0 shifts its share logically,
+// party 1 negates, shifts logically and negates again.
+// ---------------------------------------------------------------------------
+void orc_truncate(int party, const u64* in, u64* out, size_t count, int f) {
+    for (size_t t = 0; t < count; ++t) {
+        if (party == 0) out[t] = in[t] >> f;
+        else out[t] = (u64)0 - (((u64)0 - in[t]) >> f);
+    }
+}
+
+}  // extern "C"

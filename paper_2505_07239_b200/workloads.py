@@ -1,0 +1,293 @@
+"""Seeded synthetic workloads for the sparse secret-shared FFN path.
+
+This module only *draws inputs*: plaintext activations and weights, their
+fixed-point encodings, uniformly random additive shares, block masks with the
+structure of each benchmark configuration, and the dealer's Beaver triples.
+It holds none of the protocol's arithmetic (no masking, no Eq. 1, no
+truncation); both the CPU oracle used by the tests and the CUDA library are
+fed from here and otherwise share nothing.
+
+All matrices are produced in the paper's mathematical shapes (X [T, d],
+W1 [d, D], W2 [D, d], B [K, N]); `lib_layout` transposes the right-hand
+operands into the output-feature-major layout the CUDA library stores.
+
+Random numbers come from a counter-based generator defined here: word number
+`c` of stream `s` under master seed `m` is finalise(m, s, c), so any tensor can
+be regenerated independently of every other.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Dict, Optional
+
+import numpy as np
+
+U64 = np.uint64
+_MASK64 = (1 << 64) - 1
+
+
+# ---------------------------------------------------------------------------
+# counter-based generator
+# ---------------------------------------------------------------------------
+def _stream_id(name: str) -> int:
+    """Deterministic 64-bit id of a stream name (multiply-xor over the bytes)."""
+    h = 0x243F6A8885A308D3
+    for ch in name.encode():
+        h = ((h ^ ch) * 0x100000001B3 + 0x9E3779B97F4A7C15) & _MASK64
+        h ^= h >> 29
+    return h
+
+
+def _finalise(z: np.ndarray) -> np.ndarray:
+    """Bijective 64-bit finaliser: two xor-shift-multiply rounds and a last xor-shift."""
+    with np.errstate(over="ignore"):
+        z = (z ^ (z >> U64(30))) * U64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> U64(27))) * U64(0x94D049BB133111EB)
+        z = z ^ (z >> U64(31))
+    return z
+
+
+def random_u64(seed: int, stream: str, count: int, offset: int = 0) -> np.ndarray:
+    """`count` uniform 64-bit words of stream `stream` under master seed `seed`."""
+    sid = _stream_id(stream)
+    base = (sid * 0xD1342543DE82EF95 + (seed & _MASK64) * 0x2545F4914F6CDD1D + 0x632BE59BD9B4E019) & _MASK64
+    with np.errstate(over="ignore"):
+        ctr = np.arange(offset, offset + count, dtype=U64) * U64(0x9E3779B97F4A7C15) + U64(base)
+    return _finalise(_finalise(ctr) ^ U64(sid))
+
+
+def random_unit(seed: int, stream: str, count: int) -> np.ndarray:
+    """Uniform doubles in [0, 1) from the top 53 bits of each word."""
+    return (random_u64(seed, stream, count) >> U64(11)).astype(np.float64) * (1.0 / (1 << 53))
+
+
+def random_normal(seed: int, stream: str, count: int, sigma: float) -> np.ndarray:
+    """N(0, sigma) by the polar-free Box-Muller transform on two uniform streams."""
+    u1 = random_unit(seed, stream + "/bm1", count)
+    u2 = random_unit(seed, stream + "/bm2", count)
+    r = np.sqrt(-2.0 * np.log(1.0 - u1))
+    return sigma * r * np.cos(2.0 * math.pi * u2)
+
+
+# ---------------------------------------------------------------------------
+# fixed point and sharing (data preparation by the data owner / model owner)
+# ---------------------------------------------------------------------------
+def encode(v: np.ndarray, frac_bits: int) -> np.ndarray:
+    """Real -> ring: round(v * 2^f) as a two's-complement 64-bit word."""
+    return np.floor(v * float(1 << frac_bits) + 0.5).astype(np.int64).view(U64)
+
+
+def decode(u: np.ndarray, frac_bits: int) -> np.ndarray:
+    """Ring -> real: signed interpretation divided by 2^f."""
+    return np.ascontiguousarray(u).view(np.int64).astype(np.float64) / float(1 << frac_bits)
+
+
+def split_shares(value: np.ndarray, seed: int, stream: str):
+    """Additive sharing: share 0 uniform, share 1 = value - share 0 (mod 2^64)."""
+    s0 = random_u64(seed, stream + "/share0", value.size).reshape(value.shape)
+    with np.errstate(over="ignore"):
+        s1 = value - s0
+    return s0, s1
+
+
+# ---------------------------------------------------------------------------
+# configurations
+# ---------------------------------------------------------------------------
+@dataclasses.dataclass(frozen=True)
+class FFNConfig:
+    name: str
+    tokens: int
+    d_model: int
+    d_ff: int
+    block: int
+    frac_bits: int
+    gated: bool
+    active_fraction: float
+    mask_kind: str            # "uniform" | "runs" | "pool_union"
+    x_dist: str               # "uniform" | "normal"
+    w_dist: str               # "uniform" | "normal0.02"
+    steps: int = 1            # decode: number of single-token steps, fresh mask each
+
+    @property
+    def n_blocks(self) -> int:
+        return self.d_ff // self.block
+
+    @property
+    def groups(self) -> int:
+        return 2 if self.gated else 1
+
+    def n_active_blocks(self, sparsity: Optional[float] = None) -> int:
+        p = self.active_fraction if sparsity is None else 1.0 - sparsity
+        return max(1, int(math.floor(p * self.n_blocks + 0.5)))
+
+
+CONFIGS: Dict[str, FFNConfig] = {
+    "tiny": FFNConfig("tiny", 16, 256, 1024, 32, 12, False, 0.10, "uniform", "uniform", "uniform"),
+    "opt125m": FFNConfig("opt125m", 128, 768, 3072, 32, 13, False, 0.10, "runs", "normal", "normal0.02"),
+    "opt1.3b": FFNConfig("opt1.3b", 512, 2048, 8192, 32, 16, False, 0.10, "uniform", "normal", "normal0.02"),
+    "llama7b": FFNConfig("llama7b", 256, 4096, 11008, 64, 16, True, 0.15, "pool_union", "normal", "normal0.02"),
+    "opt6.7b-decode": FFNConfig("opt6.7b-decode", 32, 4096, 16384, 32, 16, False, 0.08, "uniform", "normal",
+                                "normal0.02", steps=64),
+}
+SWEEP_SPARSITIES = (0.0, 0.5, 0.8, 0.9, 0.95)
+
+
+# ---------------------------------------------------------------------------
+# block masks
+# ---------------------------------------------------------------------------
+def _choose_k(seed: int, stream: str, population: int, k: int) -> np.ndarray:
+    keys = random_u64(seed, stream, population)
+    return np.sort(np.argsort(keys, kind="stable")[:k])
+
+
+def block_mask(cfg: FFNConfig, seed: int, sparsity: Optional[float] = None, step: int = 0) -> np.ndarray:
+    """0/1 byte per block, with the structure the configuration names."""
+    nb = cfg.n_blocks
+    k = cfg.n_active_blocks(sparsity)
+    tag = f"{cfg.name}/mask/s{sparsity}/step{step}"
+    m = np.zeros(nb, dtype=np.uint8)
+    if cfg.mask_kind == "uniform":
+        m[_choose_k(seed, tag, nb, k)] = 1
+    elif cfg.mask_kind == "runs":
+        # runs of active blocks: uniform start among free blocks, length
+        # Geometric(1/4) on {1,2,...} (mean 4), clipped by occupied blocks,
+        # the end of the layer and the remaining budget
+        u = random_unit(seed, tag + "/runs", 4 * nb + 16)
+        pos = 0
+        placed = 0
+        while placed < k:
+            free = np.flatnonzero(m == 0)
+            start = int(free[int(u[pos] * len(free))])
+            length = 1 + int(math.floor(math.log(1.0 - u[pos + 1]) / math.log(0.75)))
+            pos += 2
+            b = start
+            while b < nb and m[b] == 0 and length > 0 and placed < k:
+                m[b] = 1
+                b += 1
+                length -= 1
+                placed += 1
+    elif cfg.mask_kind == "pool_union":
+        # candidate pool of exactly k blocks; each token activates a pool block
+        # with probability 0.05; the layer mask is the union over tokens
+        pool = _choose_k(seed, tag + "/pool", nb, k)
+        u = random_unit(seed, tag + "/tok", cfg.tokens * k).reshape(cfg.tokens, k)
+        hit = (u < 0.05).any(axis=0)
+        m[pool[hit]] = 1
+        if not m.any():
+            m[pool[0]] = 1
+    else:
+        raise ValueError(cfg.mask_kind)
+    return m
+
+
+def active_neurons(mask: np.ndarray, block: int) -> np.ndarray:
+    """Ascending neuron indices of the active blocks (for building inputs only)."""
+    blocks = np.flatnonzero(mask)
+    return (blocks[:, None] * block + np.arange(block)[None, :]).reshape(-1).astype(np.int32)
+
+
+# ---------------------------------------------------------------------------
+# plaintext tensors and their shares
+# ---------------------------------------------------------------------------
+def _draw(dist: str, seed: int, stream: str, shape) -> np.ndarray:
+    count = int(np.prod(shape))
+    if dist == "uniform":
+        return (2.0 * random_unit(seed, stream, count) - 1.0).reshape(shape)
+    if dist == "normal":
+        return random_normal(seed, stream, count, 1.0).reshape(shape)
+    if dist == "normal0.02":
+        return random_normal(seed, stream, count, 0.02).reshape(shape)
+    raise ValueError(dist)
+
+
+def model_shares(cfg: FFNConfig, seed: int, plain: bool = True) -> dict:
+    """Weights of one FFN: encoded ring values and the two shares of each.
+
+    Returns {"W1": (ring, s0, s1), "WG": ... (gated only), "W2": ...} in
+    mathematical shapes W1/WG [d, D], W2 [D, d].  With plain=False the weights
+    are not drawn from their distribution at all: the shares themselves are
+    uniform words (their sum is then an arbitrary ring element), which is all
+    a timing run or a share-parity test needs, and is much cheaper.
+    """
+    out = {}
+    names = [("W1", (cfg.d_model, cfg.d_ff)), ("W2", (cfg.d_ff, cfg.d_model))]
+    if cfg.gated:
+        names.insert(1, ("WG", (cfg.d_model, cfg.d_ff)))
+    for name, shape in names:
+        if plain:
+            ring = encode(_draw(cfg.w_dist, seed, f"{cfg.name}/{name}", shape), cfg.frac_bits)
+            s0, s1 = split_shares(ring, seed, f"{cfg.name}/{name}")
+        else:
+            count = int(np.prod(shape))
+            s0 = random_u64(seed, f"{cfg.name}/{name}/share0", count).reshape(shape)
+            s1 = random_u64(seed, f"{cfg.name}/{name}/share1", count).reshape(shape)
+            with np.errstate(over="ignore"):
+                ring = s0 + s1
+        out[name] = (ring, s0, s1)
+    return out
+
+
+def activation_shares(cfg: FFNConfig, seed: int, step: int = 0, tokens: Optional[int] = None):
+    """Input activations X [T, d]: (ring, share0, share1)."""
+    T = cfg.tokens if tokens is None else tokens
+    ring = encode(_draw(cfg.x_dist, seed, f"{cfg.name}/X/step{step}", (T, cfg.d_model)), cfg.frac_bits)
+    s0, s1 = split_shares(ring, seed, f"{cfg.name}/X/step{step}")
+    return ring, s0, s1
+
+
+def hidden_shares(cfg: FFNConfig, seed: int, n_active: int, step: int = 0, tokens: Optional[int] = None):
+    """A synthetic post-activation hidden state [T, n] for exercising the
+    down-projection alone: |N(0,1)| with about half the entries zero, encoded
+    and shared.  (The end-to-end tests derive the hidden state from the
+    up-projection instead.)"""
+    T = cfg.tokens if tokens is None else tokens
+    v = _draw("normal", seed, f"{cfg.name}/H/step{step}", (T, n_active))
+    ring = encode(np.maximum(v, 0.0), cfg.frac_bits)
+    s0, s1 = split_shares(ring, seed, f"{cfg.name}/H/step{step}")
+    return ring, s0, s1
+
+
+def ring_matmul(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """Exact product mod 2^64 of two uint64 matrices (library integer matmul)."""
+    try:
+        import torch
+
+        ta = torch.from_numpy(np.ascontiguousarray(a).view(np.int64))
+        tb = torch.from_numpy(np.ascontiguousarray(b).view(np.int64))
+        return (ta @ tb).numpy().view(U64)
+    except ImportError:  # pragma: no cover
+        with np.errstate(over="ignore"):
+            return a @ b
+
+
+def dealer_triple(seed: int, stream: str, rows: int, inner: int, cols: int, valid: bool = True) -> dict:
+    """Matrix Beaver triple for one [rows, inner] x [inner, cols] product.
+
+    A, B uniform; C = A B mod 2^64; each split into two uniform shares.  With
+    valid=False the C shares are just uniform words (no product is formed):
+    share-by-share parity and timing do not need c = ab, only the
+    reconstruction checks do.
+    """
+    A = random_u64(seed, stream + "/A", rows * inner).reshape(rows, inner)
+    B = random_u64(seed, stream + "/B", inner * cols).reshape(inner, cols)
+    A0, A1 = split_shares(A, seed, stream + "/A")
+    B0, B1 = split_shares(B, seed, stream + "/B")
+    if valid:
+        C = ring_matmul(A, B)
+        C0, C1 = split_shares(C, seed, stream + "/C")
+    else:
+        C = None
+        C0 = random_u64(seed, stream + "/C/share0", rows * cols).reshape(rows, cols)
+        C1 = random_u64(seed, stream + "/C/share1", rows * cols).reshape(rows, cols)
+    return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1)}
+
+
+def reshare(value: np.ndarray, seed: int, stream: str):
+    """Fresh uniform sharing of a ring tensor (used after the activation functionality)."""
+    return split_shares(value, seed, stream)
+
+
+def lib_layout(right_operand: np.ndarray) -> np.ndarray:
+    """[inner, cols] (paper shape) -> [cols, inner] contiguous (library storage)."""
+    return np.ascontiguousarray(right_operand.T)
