@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse secret-shared FFN path on B200.
+
+One "step" is one pass of the whole path for both parties over one batch of
+synthetic input: mask compaction, up-projection (open, exchange, combine),
+truncation, down-projection, truncation.  Default workload: the OPT-1.3B-shaped
+FFN (tokens 512, d_model 2048, d_ff 8192, 16 fractional bits) at 90 % block
+sparsity.  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload opt1.3b] [--sparsity 0.9] [--path auto|simt|limb]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2505_07239_b200 import workloads as wl  # noqa: E402
+
+METRIC = "sparse shared-FFN Z_2^64 MACs/s"
+UNIT = "MAC64/s"
+L2_FLUSH_BYTES = 512 << 20
+
+
+def ffn_macs(cfg, T, n):
+    """Algorithmic ring MACs of one step, both parties: 2*T*K*N per party per product."""
+    g = cfg.groups
+    return 2 * (2 * T * cfg.d_model * g * n) + 2 * (2 * T * n * cfg.d_model)
+
+
+def ffn_bytes(cfg, T, n):
+    """Algorithmic bytes of one step, both parties: 8*(6KN + 6TK + 2TN) per party per product."""
+    d, g = cfg.d_model, cfg.groups
+    up = 8 * (6 * d * g * n + 6 * T * d + 2 * T * g * n)
+    dn = 8 * (6 * n * d + 6 * T * n + 2 * T * d)
+    return 2 * (up + dn)
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- inputs
+def make_inputs(cfg, seed, sparsity, step, T):
+    """One batch in the paper's shapes: mask, X shares, triples, synthetic hidden state."""
+    mask = wl.block_mask(cfg, seed, sparsity, step)
+    n = int(mask.sum()) * cfg.block
+    g, d = cfg.groups, cfg.d_model
+    _, X0, X1 = wl.activation_shares(cfg, seed, step=step, tokens=T)
+    up = wl.dealer_triple(seed, f"bench/up/{step}", T, d, g * n, valid=False)
+    dn = wl.dealer_triple(seed, f"bench/dn/{step}", T, n, d, valid=False)
+    _, H0, H1 = wl.hidden_shares(cfg, seed, n, step=step, tokens=T)
+    return {"mask": mask, "n": n, "X": (X0, X1), "up": up, "dn": dn, "H": (H0, H1)}
+
+
+def lib_tensors(inp):
+    """Per party, (tensor id -> numpy array in the library's storage layout)."""
+    from paper_2505_07239_b200 import binding as cb
+
+    out = []
+    for p in (0, 1):
+        out.append({
+            cb.X: inp["X"][p], cb.A_UP: inp["up"]["A"][1 + p], cb.B_UP: wl.lib_layout(inp["up"]["B"][1 + p]),
+            cb.C_UP: inp["up"]["C"][1 + p], cb.H: inp["H"][p], cb.A_DN: inp["dn"]["A"][1 + p],
+            cb.B_DN: wl.lib_layout(inp["dn"]["B"][1 + p]), cb.C_DN: inp["dn"]["C"][1 + p]})
+    return out
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def time_oracle(cfg, seed, sparsity, budget_s=15.0):
+    """The oracle as it stands, single thread, on a bounded sample (a prefix of
+    the token rows) of the same workload: SOMM, truncate, SIMM, truncate."""
+    import oracle
+
+    W = wl.model_shares(cfg, seed, plain=False)
+    g = cfg.groups
+
+    def run(T):
+        inp = make_inputs(cfg, seed, sparsity, 0, T)
+        I1 = oracle.index_set(inp["mask"], cfg.block, 1)
+        Ig = oracle.index_set(inp["mask"], cfg.block, g)
+        Wup = tuple(np.concatenate([W["WG"][s], W["W1"][s]], axis=1) if cfg.gated else W["W1"][s] for s in (1, 2))
+        t0 = time.perf_counter()
+        oracle.index_set(inp["mask"], cfg.block, g)
+        r = oracle.somm(inp["X"], Wup, Ig, inp["up"]["A"][1:], inp["up"]["B"][1:], inp["up"]["C"][1:])
+        for p in (0, 1):
+            oracle.truncate(p, r["Z"][p], cfg.frac_bits)
+        y = oracle.simm(inp["H"], W["W2"][1:], I1, inp["dn"]["A"][1:], inp["dn"]["B"][1:], inp["dn"]["C"][1:])
+        for p in (0, 1):
+            oracle.truncate(p, y["Z"][p], cfg.frac_bits)
+        dt = time.perf_counter() - t0
+        return dt, ffn_macs(cfg, T, inp["n"])
+
+    probe_T = min(cfg.tokens, 8)
+    dt, macs = run(probe_T)
+    T = int(max(probe_T, min(cfg.tokens, probe_T * budget_s / max(dt, 1e-6))))
+    if T > probe_T:
+        dt, macs = run(T)
+    return {"value": macs / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 3),
+            "sample": f"first {T} of {cfg.tokens} token rows of the same workload, whole path, both parties"}
+
+
+def run_reference(args, cfg, sparsity):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, args.steps)
+    per = max(2.0, min(30.0, 120.0 / (steps + args.warmup)))
+    vals = []
+    for s in range(args.warmup + steps):
+        r = time_oracle(cfg, 1234 + s, sparsity, budget_s=per)
+        if s >= args.warmup:
+            vals.append(r)
+    value = float(np.mean([v["value"] for v in vals]))
+    n = cfg.n_active_blocks(sparsity) * cfg.block
+    ms = ffn_macs(cfg, cfg.tokens, n) / value * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, sparsity), "note": "CPU oracle, one thread, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": vals[-1]["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_name(cfg, sparsity):
+    n = cfg.n_active_blocks(sparsity) * cfg.block
+    return (f"{cfg.name} FFN tokens={cfg.tokens} d_model={cfg.d_model} d_ff={cfg.d_ff} f={cfg.frac_bits} "
+            f"block={cfg.block} sparsity={sparsity:.2f} n_active={n}")
+
+
+# --------------------------------------------------------------------------- GPU leg
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="opt1.3b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--sparsity", type=float, default=None)
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "limb"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.workload]
+    sparsity = args.sparsity
+    if sparsity is None:
+        sparsity = 0.9 if args.workload == "opt1.3b" else 1.0 - cfg.active_fraction
+    if args.impl == "reference":
+        return run_reference(args, cfg, sparsity)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_07239_b200 import binding as cb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    T, d, g = cfg.tokens, cfg.d_model, cfg.groups
+    seed = 1000 + rank          # every rank runs its own independent FFN problem (weak scaling, no collective)
+    path = {"auto": cb.PATH_AUTO, "simt": cb.PATH_SIMT, "limb": cb.PATH_LIMB}[args.path]
+    stream = torch.cuda.Stream(device=dev)
+    n_cap = cfg.n_active_blocks(sparsity) * cfg.block
+    ctx = cb.Comet(T, d, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.gated, local, n_cap, path, stream)
+    W = wl.model_shares(cfg, seed, plain=False)
+    with torch.cuda.stream(stream):
+        for p in (0, 1):
+            ctx.load_shares(p, cb.W1, cb.to_device(wl.lib_layout(W["W1"][1 + p]), dev))
+            ctx.load_shares(p, cb.W2, cb.to_device(wl.lib_layout(W["W2"][1 + p]), dev))
+            if cfg.gated:
+                ctx.load_shares(p, cb.WG, cb.to_device(wl.lib_layout(W["WG"][1 + p]), dev))
+    ctx.synchronize()
+    del W
+
+    # rotating input sets: a fresh mask (so different weight rows), X, triples and H each
+    R = 4
+    sets = []
+    for s in range(R):
+        inp = make_inputs(cfg, seed, sparsity, s, T)
+        host = lib_tensors(inp)
+        pinned = [{k: torch.from_numpy(v.view(np.int64)).pin_memory() for k, v in hp.items()} for hp in host]
+        devt = [{k: v.to(dev) for k, v in hp.items()} for hp in pinned]
+        sets.append({"n": inp["n"], "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
+                     "mask_dev": torch.from_numpy(inp["mask"]).to(dev), "pinned": pinned, "dev": devt})
+    torch.cuda.synchronize(dev)
+    n = sets[0]["n"]
+    macs = ffn_macs(cfg, T, n)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    y_host = [torch.empty((T, d), dtype=torch.int64).pin_memory() for _ in (0, 1)]
+    UP_IDS = (cb.X, cb.A_UP, cb.B_UP, cb.C_UP)
+    DN_IDS = (cb.H, cb.A_DN, cb.B_DN, cb.C_DN)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def device_step(s, timed):
+        """Inputs resident in HBM: only the path's own calls sit between the event pairs."""
+        st = sets[s % R]
+        with torch.cuda.stream(stream):
+            flush.zero_()                                  # evict L2 between steps
+            e = [ev() for _ in range(6)]
+            e[0].record(stream)
+            ctx.set_mask(st["mask_dev"])
+            e[1].record(stream)
+            for p in (0, 1):
+                for tid in UP_IDS:
+                    ctx.load_shares(p, tid, st["dev"][p][tid])
+            e[2].record(stream)
+            ctx.ffn_up(T)
+            ctx.truncate(cb.Z_UP)
+            e[3].record(stream)
+            for p in (0, 1):
+                for tid in DN_IDS:
+                    ctx.load_shares(p, tid, st["dev"][p][tid])
+            e[4].record(stream)
+            ctx.ffn_down(T)
+            ctx.truncate(cb.Y)
+            e[5].record(stream)
+        return e if timed else None
+
+    def e2e_step(s):
+        """Through the C ABI with HOST buffers: H2D of every per-step input and D2H of the result inside."""
+        st = sets[s % R]
+        with torch.cuda.stream(stream):
+            flush.zero_()
+            e0, e1 = ev(), ev()
+            e0.record(stream)
+            ctx.set_mask(st["mask_host"].numpy())
+            for p in (0, 1):
+                for tid in UP_IDS:
+                    ctx.load_shares(p, tid, st["pinned"][p][tid])
+            ctx.ffn_up(T)
+            ctx.truncate(cb.Z_UP)
+            for p in (0, 1):
+                for tid in DN_IDS:
+                    ctx.load_shares(p, tid, st["pinned"][p][tid])
+            ctx.ffn_down(T)
+            ctx.truncate(cb.Y)
+            for p in (0, 1):
+                ctx.get_into(p, cb.Y, y_host[p])
+            e1.record(stream)
+        return e0, e1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing
+    for s in range(args.warmup):
+        device_step(s, False)
+    barrier()
+    ctx.set_profiling(True)
+    launches0 = ctx.stats().kernel_launches
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    wall0 = time.perf_counter()
+    events = [device_step(args.warmup + s, True) for s in range(args.steps)]
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop() if rank == 0 else None
+    stats = ctx.stats()
+    ctx.set_profiling(False)
+    launches = stats.kernel_launches - launches0
+    step_ms = [e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) + e[4].elapsed_time(e[5]) for e in events]
+    total_ms = float(sum(step_ms))
+
+    # ---- end-to-end timing (host buffers)
+    for s in range(3):
+        e2e_step(s)
+    barrier()
+    pairs = [e2e_step(3 + s) for s in range(args.steps)]
+    barrier()
+    e2e_ms = float(sum(a.elapsed_time(b) for a, b in pairs))
+    h2d = sum(t.numel() * 8 for p in (0, 1) for t in sets[0]["pinned"][p].values()) + sets[0]["mask_host"].numel()
+    d2h = 2 * T * d * 8 + 4
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = t.tolist()
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * macs / (ms_per_step * 1e-3)
+        phase = {name: {"ms_per_step": stats.phase_ms[k] / args.steps, "launches_per_step":
+                        stats.phase_launches[k] / args.steps} for k, name in enumerate(cb.PHASE_NAMES)}
+        comb_launch_ms = stats.phase_ms[3] / max(1, stats.phase_launches[3])
+        comb_macs_per_launch = macs / 2          # up and down combine launches carry half the MACs each here
+        used_path = {cb.PATH_SIMT: "simt", cb.PATH_LIMB: "limb"}.get(stats.matmul_path, "?")
+        peaks = {}
+        try:
+            peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        except OSError:
+            pass
+        hbm = peaks.get("hbm_gbs", 6650.0)
+        bf16 = peaks.get("bf16_tflops", 1590.0)
+        src = "measured" if peaks else "fallback"
+        achieved = comb_macs_per_launch / (comb_launch_ms * 1e-3) / 1e12
+        if used_path == "limb":
+            # int8 tensor peak = measured bf16 peak x nominal ratio 2, in MAC/s, over 36 limb products per ring MAC
+            peak = bf16 * 1e12 / 2 * 2 / 36 / 1e12
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
+                    "peak_source": f"{src} bf16 GEMM peak x2 (int8 nominal ratio), as MAC/s, / 36 limb products"}
+        else:
+            # 148 SMs x 64 32-bit integer multiply-add lanes per clock x max SM clock / 4 issue slots per ring MAC
+            peak = 148 * 64 * 1.965e9 / 4 / 1e12
+            roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
+                    "peak_source": "148 SM x 64 int32 mul-add lanes/clk x 1.965 GHz / 4 issue slots per 64-bit MAC"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["kernel"] = "combine_" + used_path
+        roof["traffic"] = None
+        t_roof = max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (roof["peak"] * 1e12))
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": workload_name(cfg, sparsity), "matmul_path": used_path,
+                       "l2": "512 MiB buffer written between steps, and 4 rotating input sets with different masks",
+                       "timed": "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream",
+                       "parallelism": f"independent FFN per GPU x{world}"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "e2e": {"value": world * macs / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+                    "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "roofline": roof,
+            "path_roofline": {"algorithmic_bytes": ffn_bytes(cfg, T, n), "algorithmic_macs": macs,
+                              "hbm_gbs": hbm, "hbm_source": src, "roofline_ms": t_roof * 1e3,
+                              "frac": t_roof * 1e3 / ms_per_step},
+            "phases": phase,
+            "wall_ms_per_step_incl_untimed": wall / args.steps * 1e3,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = time_oracle(cfg, 1234, sparsity)
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

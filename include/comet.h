@@ -1,0 +1,206 @@
+/*
+ * comet.h -- C ABI of the B200 library for the per-party local arithmetic of the
+ * sparsity-aware secret-shared feed-forward layer (Comet, arXiv 2505.07239).
+ *
+ * Both parties of a 2-party additive sharing over Z_{2^64} are simulated on one
+ * GPU; the "messages" the two servers would exchange are device buffers owned by
+ * the context.  A party's kernels read only that party's shares and the two
+ * message buffers.
+ *
+ * Conventions
+ *   - Every word is a uint64_t ring element; arithmetic is mod 2^64.
+ *   - Left operands are row-major [tokens, inner].  Right operands (weights,
+ *     their masks B and the messages F) are stored OUTPUT-FEATURE-MAJOR, i.e.
+ *     as the transpose of the paper's matrix: W1 and WG are [d_ff, d_model],
+ *     W2 is [d_model, d_ff], B_UP is [g*n, d_model], B_DN is [d_model, n].
+ *     (n = active neurons, g = 2 for a gated FFN, else 1.)
+ *   - Compact column c of the up-projection stands for neuron I[c mod n], I the
+ *     ascending list of neurons in active blocks; for g = 2 columns [0,n) are
+ *     the gate projection and [n,2n) the up projection.
+ *   - Parties are 0 and 1 (the paper's P_1, P_2); party 1 carries the public
+ *     product term of Eq. 1.
+ *   - Every call returns COMET_OK or a negative error code; nothing traps or
+ *     aborts, and no exception crosses the ABI.  Arguments are validated on the
+ *     host before anything is launched.
+ *   - Pointers passed in belong to the caller.  `location` says where they
+ *     point: COMET_DEVICE (memory of the context's GPU) or COMET_HOST (pinned or
+ *     pageable host memory).  The library copies what it is given into memory
+ *     it allocated at comet_init; nothing of the caller's is kept.
+ *   - All work is enqueued on the CUDA stream given to comet_init.  Calls are
+ *     asynchronous with respect to the host except comet_set_mask (it returns
+ *     the public count n), comet_get/comet_load_shares with host pointers to
+ *     pageable memory, comet_stats and comet_destroy.
+ */
+#ifndef COMET_H_
+#define COMET_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct comet_ctx comet_ctx;
+
+enum {
+    COMET_OK = 0,
+    COMET_ERR_INVALID_ARG = -1, /* null pointer, unknown id, bad party / location       */
+    COMET_ERR_SHAPE = -2,       /* sizes disagree with the configuration or the mask    */
+    COMET_ERR_STATE = -3,       /* call out of order (e.g. ffn_up before its inputs)    */
+    COMET_ERR_OOM = -4,         /* device allocation failed in comet_init               */
+    COMET_ERR_CUDA = -5,        /* a CUDA runtime call failed; see comet_last_cuda_error */
+    COMET_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out                   */
+};
+
+enum { COMET_DEVICE = 0, COMET_HOST = 1 };
+
+/* matmul_path */
+enum {
+    COMET_PATH_AUTO = 0,   /* the path the measurements favour                              */
+    COMET_PATH_SIMT = 1,   /* 64-bit multiply-add on the integer ALUs                         */
+    COMET_PATH_LIMB = 2    /* 8-bit limb planes on the int8 tensor cores, recombined mod 2^64 */
+};
+
+/* Tensor ids.  "in" tensors are set with comet_load_shares, "out" tensors are
+ * produced by the library; every id can be read back with comet_get.  Shapes
+ * are [rows, cols] as stored (see Conventions). */
+enum {
+    COMET_X = 0,      /* in : activations                [T, d_model]           */
+    COMET_W1 = 1,     /* in : up (or fc1) weights        [d_ff, d_model]        */
+    COMET_WG = 2,     /* in : gate weights (gated only)  [d_ff, d_model]        */
+    COMET_W2 = 3,     /* in : down (or fc2) weights      [d_model, d_ff]        */
+    COMET_A_UP = 4,   /* in : triple, masks X            [T, d_model]           */
+    COMET_B_UP = 5,   /* in : triple, masks W[:, I]      [g*n, d_model]         */
+    COMET_C_UP = 6,   /* in : triple, C = A B            [T, g*n]               */
+    COMET_H = 7,      /* in : post-activation hidden     [T, n]                 */
+    COMET_A_DN = 8,   /* in : triple, masks H            [T, n]                 */
+    COMET_B_DN = 9,   /* in : triple, masks W2[I, :]     [d_model, n]           */
+    COMET_C_DN = 10,  /* in : triple                     [T, d_model]           */
+    COMET_E_UP = 11,  /* out: message X_i - A_i          [T, d_model]           */
+    COMET_F_UP = 12,  /* out: message W_i[:, I] - B_i    [g*n, d_model]         */
+    COMET_Z_UP = 13,  /* out: up-projection share        [T, g*n]               */
+    COMET_E_DN = 14,  /* out: message H_i - A'_i         [T, n]                 */
+    COMET_F_DN = 15,  /* out: message W2_i[I, :] - B'_i  [d_model, n]           */
+    COMET_Y = 16,     /* out: down-projection share      [T, d_model]           */
+    COMET_NUM_TENSORS = 17
+};
+
+typedef struct {
+    int32_t max_tokens;   /* capacity in token rows (T of any later call <= this)       */
+    int32_t d_model;      /* multiple of 16                                             */
+    int32_t d_ff;         /* multiple of `block`                                        */
+    int32_t block;        /* neurons per mask block, multiple of 16                     */
+    int32_t frac_bits;    /* fixed-point fractional bits f, 1..31                       */
+    int32_t gated;        /* 0: Y = act(X W1) W2;  1: Y = (act(X WG) * (X W1)) W2       */
+    int32_t device;       /* CUDA device ordinal                                        */
+    int32_t max_active;   /* capacity in active neurons, 0 = d_ff                       */
+    int32_t matmul_path;  /* COMET_PATH_*                                               */
+} comet_config;
+
+/* phases of the path, for the per-phase timers of comet_stats */
+enum {
+    COMET_PHASE_COMPACT = 0,  /* mask compaction                                   */
+    COMET_PHASE_OPEN = 1,     /* E_i = X_i - A_i and F_i = gather(W_i) - B_i        */
+    COMET_PHASE_PREP = 2,     /* operand preparation after the exchange (limb path) */
+    COMET_PHASE_COMBINE = 3,  /* the gathered ring matmul + Beaver combine          */
+    COMET_PHASE_TRUNCATE = 4, /* local truncation                                   */
+    COMET_NUM_PHASES = 5
+};
+
+typedef struct {
+    int64_t message_bytes;   /* bytes of E_i and F_i written by the last ffn_up/ffn_down, both parties:
+                                2 * 8 * (T*K + K*N), the communication cost C_1 of the optimality proof */
+    int64_t ring_macs;       /* 64-bit multiply-adds of the last ffn_up/ffn_down, both parties: 2 * 2*T*K*N */
+    int32_t n_active;        /* active neurons under the current mask                            */
+    int32_t n_active_blocks;
+    int32_t tokens;          /* T of the last ffn call                                           */
+    int32_t matmul_path;     /* path actually used by the last ffn call                          */
+    int64_t kernel_launches; /* kernels launched by this context since comet_init                */
+    /* filled only while profiling is on (comet_set_profiling): device time and launch
+       count per phase since profiling was switched on, from CUDA events on the stream */
+    double phase_ms[COMET_NUM_PHASES];
+    int64_t phase_launches[COMET_NUM_PHASES];
+} comet_stats_t;
+
+/* Create a context: validates the configuration, selects the device, and
+ * allocates every buffer the later calls use (shares, triples, messages,
+ * results) for the stated capacities.  `cuda_stream` is a cudaStream_t (NULL =
+ * the default stream); the library never creates or destroys streams.
+ * Errors: INVALID_ARG, SHAPE (divisibility rules above), OOM, CUDA. */
+int comet_init(const comet_config* config, void* cuda_stream, comet_ctx** out);
+
+/* Release everything comet_init allocated (synchronises the stream first). */
+void comet_destroy(comet_ctx* ctx);
+
+/* Section 2.1 / Section 3.3: each server holds its additive share of the input,
+ * of the weights, and of the dealer's correlated randomness.  Copies `rows*cols`
+ * words of party `party`'s share of tensor `tensor_id` (an "in" id) into the
+ * context.  Triples and H are sized by the current mask, so they are loaded
+ * after comet_set_mask; a shape that disagrees with the configuration or with
+ * the mask is COMET_ERR_SHAPE.  Loading X, A_UP or H fixes T for the next ffn
+ * call. */
+int comet_load_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* ptr, int location,
+                      int64_t rows, int64_t cols);
+
+/* Protocol 2 line 3 and Protocol 3 lines 1-5 under a block mask shared by all
+ * tokens: turn the plaintext sparsity distribution (one byte per block, non-zero
+ * = active) into the ascending list of active blocks, i.e. the index set I.
+ * `n_blocks` must equal d_ff / block.  Returns the number of active NEURONS in
+ * *n_active_out (the sparsity level is public in the threat model of Section
+ * 3.2), which costs one 4-byte device-to-host copy and a stream synchronise.
+ * Zero active blocks is legal.  Invalidates previously loaded triples and H. */
+int comet_set_mask(comet_ctx* ctx, const uint8_t* block_mask, int location, int32_t n_blocks,
+                   int32_t* n_active_out);
+
+/* Protocol 2 (SOMM) specialised to one connected component, with Pi_MatMul as
+ * the matrix form of Eq. 1: for both parties E_i = X_i - A_i,
+ * F_i = W_i[:, I] - B_i (column gather of the paper = row gather of the stored
+ * transpose), then after the exchange Z_i = C_i + E B_i + A_i F + i E F over the
+ * active columns only, at scale 2f.  Needs X, W1 (and WG), A_UP, B_UP, C_UP.
+ * Result in COMET_Z_UP; messages in COMET_E_UP / COMET_F_UP.  With n = 0 it does
+ * nothing. */
+int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
+
+/* Protocol 3 (SIMM) with R_j = all tokens for every active column j, so that
+ * Merge&Sum of the per-column products is one matmul with inner size n:
+ * E'_i = H_i - A'_i, F'_i = W2_i[I, :] - B'_i, Y_i = C'_i + E' B'_i + A'_i F' +
+ * i E' F'.  Needs H, W2, A_DN, B_DN, C_DN.  Result in COMET_Y.  With n = 0 both
+ * parties' Y is all zero. */
+int comet_ffn_down(comet_ctx* ctx, int32_t tokens);
+
+/* Local fixed-point truncation by f bits, in place, of COMET_Z_UP or COMET_Y for
+ * both parties (the paper does not describe truncation; this is the two-party
+ * local rule): party 0: s -> s >> f (logical); party 1: s -> -((-s) >> f). */
+int comet_truncate(comet_ctx* ctx, int tensor_id);
+
+/* Copy party `party`'s copy of any tensor to caller memory.  `capacity` is in
+ * words and must cover the tensor's current size; the number of words written
+ * is returned in *written (may be NULL). */
+int comet_get(comet_ctx* ctx, int party, int tensor_id, uint64_t* out, int location, int64_t capacity,
+              int64_t* written);
+
+/* The compacted index list: ascending ids of the active blocks (int32).
+ * `capacity` in entries; the count goes to *n_active_blocks_out. */
+int comet_get_index(comet_ctx* ctx, int32_t* out, int location, int32_t capacity, int32_t* n_active_blocks_out);
+
+/* Counters of the last calls.  Synchronises nothing unless profiling is on, in
+ * which case it waits for the stream and folds the pending event pairs into
+ * phase_ms / phase_launches. */
+int comet_stats(comet_ctx* ctx, comet_stats_t* out);
+
+/* Switch the per-phase CUDA-event timers on (non-zero) or off; switching on
+ * clears phase_ms / phase_launches.  While on, every phase of every call is
+ * bracketed by two events recorded on the context's stream. */
+int comet_set_profiling(comet_ctx* ctx, int on);
+
+/* Text for an error code; never NULL. */
+const char* comet_strerror(int code);
+
+/* cudaError_t of the last failing runtime call of this context (0 if none). */
+int comet_last_cuda_error(comet_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMET_H_ */

@@ -1,0 +1,197 @@
+"""Thin ctypes binding of libcomet_b200.so (the C ABI of include/comet.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  Tensors are torch uint64/int64 CUDA tensors or numpy/torch host
+arrays; torch is used for device memory and streams and for nothing else.
+There is no CPU fallback: if the shared library is missing or fails to load,
+importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from .build import LIB_PATH
+
+OK = 0
+DEVICE, HOST = 0, 1
+PATH_AUTO, PATH_SIMT, PATH_LIMB = 0, 1, 2
+
+(X, W1, WG, W2, A_UP, B_UP, C_UP, H, A_DN, B_DN, C_DN,
+ E_UP, F_UP, Z_UP, E_DN, F_DN, Y) = range(17)
+NUM_TENSORS = 17
+
+EXPORTS = (
+    "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
+    "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
+    "comet_set_profiling",
+)
+NUM_PHASES = 5
+PHASE_NAMES = ("compact", "open", "prep", "combine", "truncate")
+
+
+class CometConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "max_tokens", "d_model", "d_ff", "block", "frac_bits", "gated", "device", "max_active", "matmul_path")]
+
+
+class CometStats(ctypes.Structure):
+    _fields_ = [("message_bytes", ctypes.c_int64), ("ring_macs", ctypes.c_int64), ("n_active", ctypes.c_int32),
+                ("n_active_blocks", ctypes.c_int32), ("tokens", ctypes.c_int32), ("matmul_path", ctypes.c_int32),
+                ("kernel_launches", ctypes.c_int64), ("phase_ms", ctypes.c_double * 5),
+                ("phase_launches", ctypes.c_int64 * 5)]
+
+
+class CometError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {_lib.comet_strerror(code).decode()} ({code})")
+        self.code = code
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2505_07239_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.comet_init.argtypes = [ctypes.POINTER(CometConfig), vp, ctypes.POINTER(vp)]
+    lib.comet_destroy.argtypes = [vp]
+    lib.comet_destroy.restype = None
+    lib.comet_load_shares.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64, i64]
+    lib.comet_set_mask.argtypes = [vp, vp, ctypes.c_int, i32, ctypes.POINTER(i32)]
+    lib.comet_ffn_up.argtypes = [vp, i32]
+    lib.comet_ffn_down.argtypes = [vp, i32]
+    lib.comet_truncate.argtypes = [vp, ctypes.c_int]
+    lib.comet_get.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64, ctypes.POINTER(i64)]
+    lib.comet_get_index.argtypes = [vp, vp, ctypes.c_int, i32, ctypes.POINTER(i32)]
+    lib.comet_stats.argtypes = [vp, ctypes.POINTER(CometStats)]
+    lib.comet_strerror.argtypes = [ctypes.c_int]
+    lib.comet_strerror.restype = ctypes.c_char_p
+    lib.comet_last_cuda_error.argtypes = [vp]
+    lib.comet_set_profiling.argtypes = [vp, ctypes.c_int]
+    return lib
+
+
+_lib = _load()
+
+
+def library():
+    """The loaded ctypes library (for tests that poke the raw ABI)."""
+    return _lib
+
+
+def _ptr_loc(t):
+    """(address, location, element count) of a torch tensor or numpy array of 8-byte words."""
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"] and t.dtype.itemsize == 8
+        return t.ctypes.data, HOST, t.size
+    assert t.is_contiguous() and t.element_size() == 8
+    return t.data_ptr(), (DEVICE if t.is_cuda else HOST), t.numel()
+
+
+class Comet:
+    """One secret-shared FFN layer on one GPU (both parties), over the C ABI."""
+
+    def __init__(self, max_tokens: int, d_model: int, d_ff: int, block: int, frac_bits: int, gated: bool = False,
+                 device: int = 0, max_active: int = 0, matmul_path: int = PATH_AUTO,
+                 stream: Optional[torch.cuda.Stream] = None):
+        self.cfg = CometConfig(max_tokens, d_model, d_ff, block, frac_bits, int(gated), device, max_active,
+                               matmul_path)
+        self.device = torch.device("cuda", device)
+        self.stream = stream
+        self._h = ctypes.c_void_p()
+        sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+        self._check(_lib.comet_init(ctypes.byref(self.cfg), sp, ctypes.byref(self._h)), "comet_init")
+        self.groups = 2 if gated else 1
+        self.n_active = 0
+
+    # ------------------------------------------------------------------ plumbing
+    def _check(self, code: int, what: str):
+        if code != OK:
+            raise CometError(code, what)
+
+    def close(self):
+        if self._h:
+            _lib.comet_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def synchronize(self):
+        if self.stream is not None:
+            self.stream.synchronize()
+        else:
+            torch.cuda.default_stream(self.device).synchronize()
+
+    # ------------------------------------------------------------------ the six calls
+    def load_shares(self, party: int, tensor_id: int, t):
+        ptr, loc, _ = _ptr_loc(t)
+        rows, cols = t.shape
+        self._check(_lib.comet_load_shares(self._h, party, tensor_id, ptr, loc, rows, cols), "comet_load_shares")
+
+    def set_mask(self, mask) -> int:
+        if isinstance(mask, np.ndarray):
+            assert mask.dtype == np.uint8 and mask.flags["C_CONTIGUOUS"]
+            ptr, loc, nb = mask.ctypes.data, HOST, mask.size
+        else:
+            assert mask.dtype == torch.uint8 and mask.is_contiguous()
+            ptr, loc, nb = mask.data_ptr(), (DEVICE if mask.is_cuda else HOST), mask.numel()
+        n = ctypes.c_int32(0)
+        self._check(_lib.comet_set_mask(self._h, ptr, loc, nb, ctypes.byref(n)), "comet_set_mask")
+        self.n_active = n.value
+        return n.value
+
+    def ffn_up(self, tokens: int):
+        self._check(_lib.comet_ffn_up(self._h, tokens), "comet_ffn_up")
+
+    def ffn_down(self, tokens: int):
+        self._check(_lib.comet_ffn_down(self._h, tokens), "comet_ffn_down")
+
+    def truncate(self, tensor_id: int):
+        self._check(_lib.comet_truncate(self._h, tensor_id), "comet_truncate")
+
+    # ------------------------------------------------------------------ read-back
+    def get_into(self, party: int, tensor_id: int, out) -> int:
+        """Copy a tensor into caller memory (device tensor, or pinned/pageable host array)."""
+        ptr, loc, cap = _ptr_loc(out)
+        written = ctypes.c_int64(0)
+        self._check(_lib.comet_get(self._h, party, tensor_id, ptr, loc, cap, ctypes.byref(written)), "comet_get")
+        return written.value
+
+    def get(self, party: int, tensor_id: int, shape) -> np.ndarray:
+        """Read a tensor back to a numpy uint64 array of the given stored shape."""
+        out = torch.empty(int(np.prod(shape)), dtype=torch.int64, device=self.device)
+        n = self.get_into(party, tensor_id, out)
+        self.synchronize()
+        assert n == out.numel(), (n, shape)
+        return out.cpu().numpy().view(np.uint64).reshape(shape)
+
+    def get_index(self) -> np.ndarray:
+        nb = self.cfg.d_ff // self.cfg.block
+        out = torch.empty(nb, dtype=torch.int32, device=self.device)
+        cnt = ctypes.c_int32(0)
+        self._check(_lib.comet_get_index(self._h, out.data_ptr(), DEVICE, nb, ctypes.byref(cnt)), "comet_get_index")
+        self.synchronize()
+        return out[:cnt.value].cpu().numpy()
+
+    def set_profiling(self, on: bool):
+        self._check(_lib.comet_set_profiling(self._h, int(on)), "comet_set_profiling")
+
+    def stats(self) -> CometStats:
+        s = CometStats()
+        self._check(_lib.comet_stats(self._h, ctypes.byref(s)), "comet_stats")
+        return s
+
+
+def to_device(a: np.ndarray, device="cuda:0") -> torch.Tensor:
+    """numpy uint64 -> torch int64 CUDA tensor holding the same words."""
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int64)).to(device)

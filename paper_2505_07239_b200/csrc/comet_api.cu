@@ -1,0 +1,483 @@
+// C ABI of the library: context, host-side validation and kernel launches.
+// Every argument is checked on the host before anything is enqueued; device
+// code never traps.  See include/comet.h for the contract of each call.
+#include "../../include/comet.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "kernels_open.cuh"
+#include "kernels_simt.cuh"
+
+using comet::u64;
+
+struct comet_ctx {
+    comet_config cfg;
+    cudaStream_t stream;
+    int groups;                   // 1 or 2
+    int64_t cap_T, cap_n;         // capacities
+    int sm_count;
+    u64* buf[2][COMET_NUM_TENSORS];
+    int64_t cap_words[COMET_NUM_TENSORS];
+    bool loaded[2][COMET_NUM_TENSORS];
+    uint8_t* d_mask;
+    int32_t* d_ids;
+    int32_t* d_count;
+    int32_t* h_count;             // pinned
+    bool mask_set;
+    int32_t n_active, n_active_blocks;
+    int32_t tokens;               // T fixed by the last load of X / A_UP / H
+    bool up_done, down_done;
+    int32_t up_tokens, down_tokens;
+    comet_stats_t stats;
+    int last_cuda_error;
+    // per-phase timers: pairs of events recorded around each phase while profiling is on
+    bool profiling;
+    struct Pending { cudaEvent_t start, stop; int phase, launches; };
+    std::vector<Pending>* pending;
+    std::vector<cudaEvent_t>* free_events;
+};
+
+namespace {
+
+#define COMET_CUDA(ctx, call)                                  \
+    do {                                                       \
+        cudaError_t err__ = (call);                            \
+        if (err__ != cudaSuccess) {                            \
+            (ctx)->last_cuda_error = (int)err__;               \
+            return COMET_ERR_CUDA;                             \
+        }                                                      \
+    } while (0)
+
+// Brackets the launches of one phase with two events when profiling is on.
+struct PhaseTimer {
+    comet_ctx* c;
+    comet_ctx::Pending p;
+    bool on;
+    static cudaEvent_t take(comet_ctx* c) {
+        if (!c->free_events->empty()) {
+            cudaEvent_t e = c->free_events->back();
+            c->free_events->pop_back();
+            return e;
+        }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    PhaseTimer(comet_ctx* ctx, int phase, int launches) : c(ctx), on(ctx->profiling) {
+        if (!on) return;
+        p.phase = phase;
+        p.launches = launches;
+        p.start = take(c);
+        p.stop = take(c);
+        cudaEventRecord(p.start, c->stream);
+    }
+    ~PhaseTimer() {
+        if (!on) return;
+        cudaEventRecord(p.stop, c->stream);
+        c->pending->push_back(p);
+    }
+};
+
+inline int is_input(int id) { return id >= COMET_X && id <= COMET_C_DN; }
+
+// current shape of a tensor as stored; rows = cols = 0 when not defined yet
+void tensor_shape(const comet_ctx* c, int id, int64_t T, int64_t* rows, int64_t* cols) {
+    const int64_t d = c->cfg.d_model, D = c->cfg.d_ff, n = c->n_active, gn = (int64_t)c->groups * n;
+    switch (id) {
+        case COMET_X: case COMET_A_UP: case COMET_E_UP: case COMET_C_DN: case COMET_Y: *rows = T; *cols = d; break;
+        case COMET_W1: case COMET_WG: *rows = D; *cols = d; break;
+        case COMET_W2: *rows = d; *cols = D; break;
+        case COMET_B_UP: case COMET_F_UP: *rows = gn; *cols = d; break;
+        case COMET_C_UP: case COMET_Z_UP: *rows = T; *cols = gn; break;
+        case COMET_H: case COMET_A_DN: case COMET_E_DN: *rows = T; *cols = n; break;
+        case COMET_B_DN: case COMET_F_DN: *rows = d; *cols = n; break;
+        default: *rows = 0; *cols = 0;
+    }
+}
+
+int64_t tensor_capacity(const comet_ctx* c, int id) {
+    const int64_t d = c->cfg.d_model, D = c->cfg.d_ff, T = c->cap_T, n = c->cap_n, gn = c->groups * n;
+    switch (id) {
+        case COMET_X: case COMET_A_UP: case COMET_E_UP: case COMET_C_DN: case COMET_Y: return T * d;
+        case COMET_W1: return D * d;
+        case COMET_WG: return c->groups == 2 ? D * d : 0;
+        case COMET_W2: return d * D;
+        case COMET_B_UP: case COMET_F_UP: return gn * d;
+        case COMET_C_UP: case COMET_Z_UP: return T * gn;
+        case COMET_H: case COMET_A_DN: case COMET_E_DN: return T * n;
+        case COMET_B_DN: case COMET_F_DN: return d * n;
+        default: return 0;
+    }
+}
+
+inline int ew_grid(const comet_ctx* c, int64_t items, int threads) {
+    int64_t want = (items + threads - 1) / threads;
+    int64_t cap = (int64_t)c->sm_count * 8;
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+cudaMemcpyKind copy_kind(int location, bool to_library) {
+    if (location == COMET_DEVICE) return cudaMemcpyDeviceToDevice;
+    return to_library ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+}
+
+int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA, int idB, int idC, int idZ) {
+    comet::CombineArgs a;
+    for (int p = 0; p < 2; ++p) {
+        a.E[p] = c->buf[p][idE];
+        a.F[p] = c->buf[p][idF];
+        a.A[p] = c->buf[p][idA];
+        a.B[p] = c->buf[p][idB];
+        a.C[p] = c->buf[p][idC];
+        a.Z[p] = c->buf[p][idZ];
+    }
+    a.M = M; a.N = N; a.K = K;
+    dim3 grid((N + comet::simt::BN - 1) / comet::simt::BN, (M + comet::simt::BM - 1) / comet::simt::BM, 2);
+    PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
+    comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, c->stream>>>(a);
+    c->stats.kernel_launches += 1;
+    c->stats.matmul_path = COMET_PATH_SIMT;
+    COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* comet_strerror(int code) {
+    switch (code) {
+        case COMET_OK: return "ok";
+        case COMET_ERR_INVALID_ARG: return "invalid argument";
+        case COMET_ERR_SHAPE: return "shape disagrees with the configuration or the current mask";
+        case COMET_ERR_STATE: return "call out of order: a required input has not been loaded";
+        case COMET_ERR_OOM: return "device memory allocation failed";
+        case COMET_ERR_CUDA: return "a CUDA runtime call failed";
+        case COMET_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown error code";
+    }
+}
+
+int comet_last_cuda_error(comet_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
+    if (!cfg || !out) return COMET_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->gated != 0 && cfg->gated != 1) return COMET_ERR_INVALID_ARG;
+    if (cfg->matmul_path < COMET_PATH_AUTO || cfg->matmul_path > COMET_PATH_LIMB) return COMET_ERR_INVALID_ARG;
+    if (cfg->device < 0) return COMET_ERR_INVALID_ARG;
+    if (cfg->max_tokens < 1 || cfg->d_model < 16 || cfg->d_ff < 16 || cfg->block < 16) return COMET_ERR_SHAPE;
+    if (cfg->d_model % 16 || cfg->block % 16 || cfg->d_ff % cfg->block) return COMET_ERR_SHAPE;
+    if (cfg->frac_bits < 1 || cfg->frac_bits > 31) return COMET_ERR_SHAPE;
+    if (cfg->max_active < 0 || cfg->max_active > cfg->d_ff || cfg->max_active % cfg->block) return COMET_ERR_SHAPE;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device >= ndev) {
+        cudaGetLastError();
+        return COMET_ERR_CUDA;
+    }
+    comet_ctx* c = new (std::nothrow) comet_ctx;
+    if (!c) return COMET_ERR_OOM;
+    std::memset(c, 0, sizeof(*c));
+    c->pending = new (std::nothrow) std::vector<comet_ctx::Pending>();
+    c->free_events = new (std::nothrow) std::vector<cudaEvent_t>();
+    if (!c->pending || !c->free_events) {
+        delete c->pending;
+        delete c->free_events;
+        delete c;
+        return COMET_ERR_OOM;
+    }
+    c->cfg = *cfg;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->groups = cfg->gated ? 2 : 1;
+    c->cap_T = cfg->max_tokens;
+    c->cap_n = cfg->max_active ? cfg->max_active : cfg->d_ff;
+    if (cudaSetDevice(cfg->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete c->pending;
+        delete c->free_events;
+        delete c;
+        return COMET_ERR_CUDA;
+    }
+    bool ok = true;
+    for (int id = 0; id < COMET_NUM_TENSORS && ok; ++id) {
+        c->cap_words[id] = tensor_capacity(c, id);
+        for (int p = 0; p < 2 && ok; ++p)
+            if (c->cap_words[id] > 0)
+                ok = cudaMalloc((void**)&c->buf[p][id], (size_t)c->cap_words[id] * sizeof(u64)) == cudaSuccess;
+    }
+    const int nb = cfg->d_ff / cfg->block;
+    ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_ids, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_count, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMallocHost((void**)&c->h_count, sizeof(int32_t)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        comet_destroy(c);
+        return COMET_ERR_OOM;
+    }
+    *out = c;
+    return COMET_OK;
+}
+
+void comet_destroy(comet_ctx* c) {
+    if (!c) return;
+    cudaSetDevice(c->cfg.device);
+    cudaStreamSynchronize(c->stream);
+    for (int id = 0; id < COMET_NUM_TENSORS; ++id)
+        for (int p = 0; p < 2; ++p)
+            if (c->buf[p][id]) cudaFree(c->buf[p][id]);
+    if (c->d_mask) cudaFree(c->d_mask);
+    if (c->d_ids) cudaFree(c->d_ids);
+    if (c->d_count) cudaFree(c->d_count);
+    if (c->h_count) cudaFreeHost(c->h_count);
+    for (auto& p : *c->pending) {
+        cudaEventDestroy(p.start);
+        cudaEventDestroy(p.stop);
+    }
+    for (auto e : *c->free_events) cudaEventDestroy(e);
+    delete c->pending;
+    delete c->free_events;
+    cudaGetLastError();
+    delete c;
+}
+
+int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* ptr, int location, int64_t rows,
+                      int64_t cols) {
+    if (!c || (party != 0 && party != 1) || !is_input(tensor_id)) return COMET_ERR_INVALID_ARG;
+    if (!ptr && rows * cols != 0) return COMET_ERR_INVALID_ARG;      // an empty tensor may come with a null pointer
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_WG && c->groups != 2) return COMET_ERR_INVALID_ARG;
+    const bool needs_mask = tensor_id == COMET_B_UP || tensor_id == COMET_C_UP || tensor_id == COMET_H ||
+                            tensor_id == COMET_A_DN || tensor_id == COMET_B_DN;
+    if (needs_mask && !c->mask_set) return COMET_ERR_STATE;
+    const bool token_rows = tensor_id == COMET_X || tensor_id == COMET_A_UP || tensor_id == COMET_C_UP ||
+                            tensor_id == COMET_H || tensor_id == COMET_A_DN || tensor_id == COMET_C_DN;
+    if (token_rows && (rows < 1 || rows > c->cap_T)) return COMET_ERR_SHAPE;
+    int64_t er, ec;
+    tensor_shape(c, tensor_id, rows, &er, &ec);
+    if (rows != er || cols != ec) return COMET_ERR_SHAPE;
+    if (rows * cols > c->cap_words[tensor_id]) return COMET_ERR_SHAPE;
+    if (rows * cols > 0)
+        COMET_CUDA(c, cudaMemcpyAsync(c->buf[party][tensor_id], ptr, (size_t)(rows * cols) * sizeof(u64),
+                                      copy_kind(location, true), c->stream));
+    c->loaded[party][tensor_id] = true;
+    if (token_rows) c->tokens = (int32_t)rows;
+    return COMET_OK;
+}
+
+int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_t n_blocks, int32_t* n_active_out) {
+    if (!c || !block_mask || !n_active_out) return COMET_ERR_INVALID_ARG;
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (n_blocks != c->cfg.d_ff / c->cfg.block) return COMET_ERR_SHAPE;
+    COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, block_mask, (size_t)n_blocks, copy_kind(location, true), c->stream));
+    {
+        PhaseTimer timer(c, COMET_PHASE_COMPACT, 1);
+        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_mask, n_blocks, c->d_ids, c->d_count);
+    }
+    c->stats.kernel_launches += 1;
+    COMET_CUDA(c, cudaGetLastError());
+    COMET_CUDA(c, cudaMemcpyAsync(c->h_count, c->d_count, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+    const int32_t blocks = *c->h_count;
+    const int64_t n = (int64_t)blocks * c->cfg.block;
+    if (n > c->cap_n) {            // more active neurons than the context was sized for
+        c->mask_set = false;
+        return COMET_ERR_SHAPE;
+    }
+    c->n_active_blocks = blocks;
+    c->n_active = (int32_t)n;
+    c->mask_set = true;
+    c->up_done = c->down_done = false;
+    for (int p = 0; p < 2; ++p)
+        for (int id = COMET_A_UP; id <= COMET_C_DN; ++id) c->loaded[p][id] = false;
+    c->stats.n_active = c->n_active;
+    c->stats.n_active_blocks = blocks;
+    *n_active_out = c->n_active;
+    return COMET_OK;
+}
+
+int comet_ffn_up(comet_ctx* c, int32_t tokens) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    if (tokens < 1 || tokens > c->cap_T) return COMET_ERR_SHAPE;
+    if (!c->mask_set) return COMET_ERR_STATE;
+    const int need[] = {COMET_X, COMET_W1, COMET_A_UP, COMET_B_UP, COMET_C_UP};
+    for (int p = 0; p < 2; ++p) {
+        for (int id : need)
+            if (!c->loaded[p][id]) return COMET_ERR_STATE;
+        if (c->groups == 2 && !c->loaded[p][COMET_WG]) return COMET_ERR_STATE;
+    }
+    const int d = c->cfg.d_model, n = c->n_active, g = c->groups, bs = c->cfg.block;
+    c->stats.tokens = tokens;
+    c->stats.message_bytes = 2ll * 8 * ((int64_t)tokens * d + (int64_t)d * g * n);
+    c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)d * g * n;
+    c->up_tokens = tokens;
+    c->up_done = true;
+    if (n == 0) return COMET_OK;
+
+    comet::PartyPtrs X, A, W0, W1, B;
+    comet::PartyOut E, F;
+    for (int p = 0; p < 2; ++p) {
+        X.p[p] = c->buf[p][COMET_X];
+        A.p[p] = c->buf[p][COMET_A_UP];
+        E.p[p] = c->buf[p][COMET_E_UP];
+        W0.p[p] = (g == 2) ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1];
+        W1.p[p] = c->buf[p][COMET_W1];
+        B.p[p] = c->buf[p][COMET_B_UP];
+        F.p[p] = c->buf[p][COMET_F_UP];
+    }
+    const int64_t pairs = (int64_t)tokens * d / 2;
+    {
+        PhaseTimer timer(c, COMET_PHASE_OPEN, 2);
+        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(X, A, E, pairs);
+        int rows_grid = g * n < c->sm_count * 8 ? g * n : c->sm_count * 8;
+        comet::open_weight_rows_kernel<<<dim3(rows_grid, 2), 256, 0, c->stream>>>(W0, W1, B, F, c->d_ids, n, g, bs,
+                                                                                   d);
+    }
+    c->stats.kernel_launches += 2;
+    COMET_CUDA(c, cudaGetLastError());
+    return launch_combine(c, tokens, g * n, d, COMET_E_UP, COMET_F_UP, COMET_A_UP, COMET_B_UP, COMET_C_UP,
+                          COMET_Z_UP);
+}
+
+int comet_ffn_down(comet_ctx* c, int32_t tokens) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    if (tokens < 1 || tokens > c->cap_T) return COMET_ERR_SHAPE;
+    if (!c->mask_set) return COMET_ERR_STATE;
+    const int d = c->cfg.d_model, n = c->n_active, bs = c->cfg.block, D = c->cfg.d_ff;
+    for (int p = 0; p < 2; ++p) {
+        if (!c->loaded[p][COMET_W2] || !c->loaded[p][COMET_C_DN]) return COMET_ERR_STATE;
+        if (n > 0 && (!c->loaded[p][COMET_H] || !c->loaded[p][COMET_A_DN] || !c->loaded[p][COMET_B_DN]))
+            return COMET_ERR_STATE;
+    }
+    c->stats.tokens = tokens;
+    c->stats.message_bytes = 2ll * 8 * ((int64_t)tokens * n + (int64_t)n * d);
+    c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)n * d;
+    c->down_tokens = tokens;
+    c->down_done = true;
+    if (n == 0) {
+        // no active neuron: the product is empty and both result shares are zero
+        for (int p = 0; p < 2; ++p)
+            COMET_CUDA(c, cudaMemsetAsync(c->buf[p][COMET_Y], 0, (size_t)tokens * d * sizeof(u64), c->stream));
+        return COMET_OK;
+    }
+    comet::PartyPtrs H, A, W, B;
+    comet::PartyOut E, F;
+    for (int p = 0; p < 2; ++p) {
+        H.p[p] = c->buf[p][COMET_H];
+        A.p[p] = c->buf[p][COMET_A_DN];
+        E.p[p] = c->buf[p][COMET_E_DN];
+        W.p[p] = c->buf[p][COMET_W2];
+        B.p[p] = c->buf[p][COMET_B_DN];
+        F.p[p] = c->buf[p][COMET_F_DN];
+    }
+    const int64_t pairs = (int64_t)tokens * n / 2;
+    {
+        PhaseTimer timer(c, COMET_PHASE_OPEN, 2);
+        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(H, A, E, pairs);
+        const int64_t wpairs = (int64_t)d * n / 2;
+        comet::open_weight_strips_kernel<<<dim3(ew_grid(c, wpairs, 256), 2), 256, 0, c->stream>>>(
+            W, B, F, c->d_ids, n, bs, d, D);
+    }
+    c->stats.kernel_launches += 2;
+    COMET_CUDA(c, cudaGetLastError());
+    return launch_combine(c, tokens, d, n, COMET_E_DN, COMET_F_DN, COMET_A_DN, COMET_B_DN, COMET_C_DN, COMET_Y);
+}
+
+int comet_truncate(comet_ctx* c, int tensor_id) {
+    if (!c || (tensor_id != COMET_Z_UP && tensor_id != COMET_Y)) return COMET_ERR_INVALID_ARG;
+    const bool up = tensor_id == COMET_Z_UP;
+    if (up ? !c->up_done : !c->down_done) return COMET_ERR_STATE;
+    int64_t rows, cols;
+    tensor_shape(c, tensor_id, up ? c->up_tokens : c->down_tokens, &rows, &cols);
+    const int64_t pairs = rows * cols / 2;
+    if (pairs == 0) return COMET_OK;
+    comet::PartyOut Z;
+    for (int p = 0; p < 2; ++p) Z.p[p] = c->buf[p][tensor_id];
+    {
+        PhaseTimer timer(c, COMET_PHASE_TRUNCATE, 1);
+        comet::truncate_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(Z, pairs, c->cfg.frac_bits);
+    }
+    c->stats.kernel_launches += 1;
+    COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
+int comet_get(comet_ctx* c, int party, int tensor_id, uint64_t* out, int location, int64_t capacity,
+              int64_t* written) {
+    if (!c || !out || (party != 0 && party != 1) || tensor_id < 0 || tensor_id >= COMET_NUM_TENSORS)
+        return COMET_ERR_INVALID_ARG;
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_WG && c->groups != 2) return COMET_ERR_INVALID_ARG;
+    int64_t T = c->tokens;
+    if (tensor_id == COMET_E_UP || tensor_id == COMET_Z_UP) T = c->up_tokens;
+    if (tensor_id == COMET_E_DN || tensor_id == COMET_Y) T = c->down_tokens;
+    int64_t rows, cols;
+    tensor_shape(c, tensor_id, T, &rows, &cols);
+    const int64_t words = rows * cols;
+    if (is_input(tensor_id) ? !c->loaded[party][tensor_id]
+                            : !((tensor_id == COMET_E_UP || tensor_id == COMET_F_UP || tensor_id == COMET_Z_UP)
+                                    ? c->up_done : c->down_done))
+        return COMET_ERR_STATE;
+    if (capacity < words) return COMET_ERR_SHAPE;
+    if (words > 0)
+        COMET_CUDA(c, cudaMemcpyAsync(out, c->buf[party][tensor_id], (size_t)words * sizeof(u64),
+                                      copy_kind(location, false), c->stream));
+    if (written) *written = words;
+    return COMET_OK;
+}
+
+int comet_get_index(comet_ctx* c, int32_t* out, int location, int32_t capacity, int32_t* n_active_blocks_out) {
+    if (!c || !out || !n_active_blocks_out) return COMET_ERR_INVALID_ARG;
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (!c->mask_set) return COMET_ERR_STATE;
+    if (capacity < c->n_active_blocks) return COMET_ERR_SHAPE;
+    if (c->n_active_blocks > 0)
+        COMET_CUDA(c, cudaMemcpyAsync(out, c->d_ids, (size_t)c->n_active_blocks * sizeof(int32_t),
+                                      copy_kind(location, false), c->stream));
+    *n_active_blocks_out = c->n_active_blocks;
+    return COMET_OK;
+}
+
+int comet_stats(comet_ctx* c, comet_stats_t* out) {
+    if (!c || !out) return COMET_ERR_INVALID_ARG;
+    if (!c->pending->empty()) {
+        COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+        for (auto& p : *c->pending) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, p.start, p.stop) == cudaSuccess) {
+                c->stats.phase_ms[p.phase] += ms;
+                c->stats.phase_launches[p.phase] += p.launches;
+            }
+            c->free_events->push_back(p.start);
+            c->free_events->push_back(p.stop);
+        }
+        c->pending->clear();
+        cudaGetLastError();
+    }
+    *out = c->stats;
+    return COMET_OK;
+}
+
+int comet_set_profiling(comet_ctx* c, int on) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    comet_stats_t tmp;
+    const int rc = comet_stats(c, &tmp);      // drain what is pending
+    if (rc != COMET_OK) return rc;
+    c->profiling = on != 0;
+    if (c->profiling)
+        for (int k = 0; k < COMET_NUM_PHASES; ++k) {
+            c->stats.phase_ms[k] = 0.0;
+            c->stats.phase_launches[k] = 0;
+        }
+    return COMET_OK;
+}
+
+}  // extern "C"

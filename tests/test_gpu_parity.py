@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle,
+bit for bit, on the same seeded inputs."""
+import ctypes
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from paper_2505_07239_b200 import workloads as wl  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def hz():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from tests import harness
+
+    return harness
+
+
+def _ok(report):
+    assert report["mismatches"] == 0, [c for c in report["compared"] if c[2]]
+    return report
+
+
+PATHS = [1]   # COMET_PATH_SIMT
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_tiny_full(hz, path):
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["tiny"], seed=1, matmul_path=path))
+    assert r["n_active"] == 96 and r["up_reconstructs"]
+    # 12 fractional bits, |w| <= 1, 96 active neurons: bounded by n * 2^-f, not by 2^-10
+    assert r["float64_max_abs_err"] < 96 * 2.0 ** -12
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_opt125m_full(hz, path):
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=2, matmul_path=path))
+    assert r["n_active"] == 320 and r["up_reconstructs"]
+    assert r["float64_max_abs_err"] < 2.0 ** -10
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_opt13b_95_full(hz, path):
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt1.3b"], seed=3, sparsity=0.95, matmul_path=path))
+    assert r["n_active"] == 416 and r["up_reconstructs"]
+    assert r["float64_max_abs_err"] < 2.0 ** -10
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("tokens", [1, 17, 130])
+def test_ragged_token_counts(hz, path, tokens):
+    _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=4, tokens=tokens, matmul_path=path, float_report=False))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_gated_small(hz, path):
+    cfg = wl.FFNConfig("gated-small", 40, 128, 512, 64, 16, True, 0.25, "uniform", "normal", "normal0.02")
+    r = _ok(hz.run_and_compare_full(cfg, seed=5, matmul_path=path))
+    assert r["n_active"] == 128 and r["up_reconstructs"]
+    assert r["float64_max_abs_err"] < 2.0 ** -10
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_all_ones_mask_is_the_dense_product(hz, path):
+    cfg = wl.CONFIGS["tiny"]
+    r = _ok(hz.run_and_compare_full(cfg, seed=6, sparsity=0.0, matmul_path=path))
+    assert r["n_active"] == cfg.d_ff and r["up_reconstructs"]
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_single_block_first_and_last(hz, path):
+    cfg = wl.CONFIGS["tiny"]
+    for b in (0, cfg.n_blocks - 1):
+        m = np.zeros(cfg.n_blocks, np.uint8)
+        m[b] = 1
+        r = _ok(hz.run_and_compare_full(cfg, seed=7, mask=m, matmul_path=path, float_report=False))
+        assert r["n_active"] == cfg.block
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("sparsity", [0.0, 0.5, 0.8, 0.9])
+def test_opt13b_sweep_sampled(hz, path, sparsity):
+    _ok(hz.run_and_compare_sampled(wl.CONFIGS["opt1.3b"], seed=8, sparsity=sparsity, matmul_path=path))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_llama7b_sampled(hz, path):
+    r = _ok(hz.run_and_compare_sampled(wl.CONFIGS["llama7b"], seed=9, matmul_path=path))
+    assert 23 * 64 <= r["n_active"] <= 26 * 64
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_opt67b_decode_steps_sampled(hz, path):
+    cfg = wl.CONFIGS["opt6.7b-decode"]
+    W = wl.model_shares(cfg, 10, plain=False)
+    ctx = hz.make_context(cfg, cfg.tokens, path, max_active=2048)
+    hz.load_weights(ctx, cfg, W)
+    for step in (0, 1, 63):       # fresh mask, X and triples per step, weights loaded once
+        r = _ok(hz.run_and_compare_sampled(cfg, seed=10, step=step, matmul_path=path, ctx=ctx, weights=W,
+                                           samples=256))
+        assert r["n_active"] == 1312
+    ctx.close()
+
+
+def test_masked_neurons_contribute_exactly_zero(hz):
+    """Garbage in the weight shares of inactive neurons leaves every output bit unchanged."""
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["tiny"]
+    T, d, f = cfg.tokens, cfg.d_model, cfg.frac_bits
+    seed = 11
+    W = wl.model_shares(cfg, seed, plain=False)
+    mask = wl.block_mask(cfg, seed)
+    I = wl.active_neurons(mask, cfg.block)
+    dead = np.setdiff1d(np.arange(cfg.d_ff), I)
+    _, X0, X1 = wl.activation_shares(cfg, seed)
+    outs = []
+    for garble in (False, True):
+        Wv = {k: tuple(a.copy() for a in v) for k, v in W.items()}
+        if garble:
+            rng = np.random.default_rng(0)
+            for slot in (1, 2):
+                Wv["W1"][slot][:, dead] = rng.integers(0, 1 << 64, (d, dead.size), dtype=np.uint64)
+                Wv["W2"][slot][dead, :] = rng.integers(0, 1 << 64, (dead.size, d), dtype=np.uint64)
+        ctx = hz.make_context(cfg, T)
+        hz.load_weights(ctx, cfg, Wv)
+        for p, Xs in ((0, X0), (1, X1)):
+            ctx.load_shares(p, cb.X, cb.to_device(Xs))
+        n = ctx.set_mask(mask)
+        hz.load_triple_up(ctx, wl.dealer_triple(seed, "u", T, d, n, valid=False))
+        ctx.ffn_up(T)
+        ctx.truncate(cb.Z_UP)
+        _, H0, H1 = wl.hidden_shares(cfg, seed, n)
+        for p, Hs in ((0, H0), (1, H1)):
+            ctx.load_shares(p, cb.H, cb.to_device(Hs))
+        hz.load_triple_down(ctx, wl.dealer_triple(seed, "d", T, n, d, valid=False))
+        ctx.ffn_down(T)
+        ctx.truncate(cb.Y)
+        outs.append([ctx.get(p, t, s) for p in (0, 1) for t, s in ((cb.Z_UP, (T, n)), (cb.Y, (T, d)),
+                                                                    (cb.F_UP, (n, d)), (cb.F_DN, (d, n)))])
+        ctx.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+def test_no_active_neuron(hz):
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["tiny"]
+    T, d = cfg.tokens, cfg.d_model
+    W = wl.model_shares(cfg, 12, plain=False)
+    ctx = hz.make_context(cfg, T)
+    hz.load_weights(ctx, cfg, W)
+    _, X0, X1 = wl.activation_shares(cfg, 12)
+    for p, Xs in ((0, X0), (1, X1)):
+        ctx.load_shares(p, cb.X, cb.to_device(Xs))
+    assert ctx.set_mask(np.zeros(cfg.n_blocks, np.uint8)) == 0
+    assert ctx.get_index().size == 0
+    tri = wl.dealer_triple(12, "u", T, d, 0, valid=False)
+    hz.load_triple_up(ctx, tri)
+    ctx.ffn_up(T)                       # nothing to do
+    ctx.truncate(cb.Z_UP)
+    for p in (0, 1):
+        ctx.load_shares(p, cb.C_DN, cb.to_device(np.ones((T, d), np.uint64)))
+    ctx.ffn_down(T)
+    ctx.truncate(cb.Y)
+    for p in (0, 1):
+        assert not ctx.get(p, cb.Y, (T, d)).any()
+    ctx.close()
+
+
+def test_run_to_run_determinism(hz):
+    a = hz.run_and_compare_sampled(wl.CONFIGS["opt125m"], seed=13, samples=64)
+    b = hz.run_and_compare_sampled(wl.CONFIGS["opt125m"], seed=13, samples=64)
+    assert a["mismatches"] == 0 and b["mismatches"] == 0
+
+
+def test_errors_are_status_codes(hz):
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["tiny"]
+    T, d, D = cfg.tokens, cfg.d_model, cfg.d_ff
+    ctx = hz.make_context(cfg, T)
+    lib = cb.library()
+    h = ctx._h
+    buf = torch.zeros(D * d, dtype=torch.int64, device="cuda")
+    n = ctypes.c_int32(-5)
+    # wrong order
+    assert lib.comet_ffn_up(h, T) == -3
+    assert lib.comet_truncate(h, cb.Z_UP) == -3
+    assert lib.comet_load_shares(h, 0, cb.B_UP, buf.data_ptr(), 0, 96, d) == -3      # needs the mask first
+    # bad arguments
+    assert lib.comet_load_shares(h, 2, cb.X, buf.data_ptr(), 0, T, d) == -1
+    assert lib.comet_load_shares(h, 0, cb.Z_UP, buf.data_ptr(), 0, T, d) == -1       # not an input
+    assert lib.comet_load_shares(h, 0, cb.WG, buf.data_ptr(), 0, D, d) == -1         # not gated
+    assert lib.comet_load_shares(h, 0, cb.X, None, 0, T, d) == -1
+    assert lib.comet_load_shares(h, 0, cb.X, buf.data_ptr(), 5, T, d) == -1
+    # bad shapes
+    assert lib.comet_load_shares(h, 0, cb.X, buf.data_ptr(), 0, T + 1, d) == -2
+    assert lib.comet_load_shares(h, 0, cb.X, buf.data_ptr(), 0, T, d + 16) == -2
+    assert lib.comet_load_shares(h, 0, cb.W1, buf.data_ptr(), 0, d, D) == -2         # transposed
+    m = torch.ones(cfg.n_blocks, dtype=torch.uint8, device="cuda")
+    assert lib.comet_set_mask(h, m.data_ptr(), 0, cfg.n_blocks - 1, ctypes.byref(n)) == -2
+    assert lib.comet_set_mask(h, m.data_ptr(), 0, cfg.n_blocks, ctypes.byref(n)) == 0 and n.value == D
+    assert lib.comet_load_shares(h, 0, cb.B_UP, buf.data_ptr(), 0, 96, d) == -2      # n is d_ff now
+    assert lib.comet_ffn_up(h, T + 1) == -2
+    assert lib.comet_ffn_up(h, T) == -3                                              # inputs still missing
+    assert lib.comet_truncate(h, cb.X) == -1
+    assert lib.comet_get(h, 0, cb.Y, buf.data_ptr(), 0, T * d, None) == -3
+    # a context sized for fewer active neurons refuses a denser mask
+    small = cb.Comet(T, d, D, cfg.block, cfg.frac_bits, False, 0, 64)
+    assert lib.comet_set_mask(small._h, m.data_ptr(), 0, cfg.n_blocks, ctypes.byref(n)) == -2
+    small.close()
+    # the context is still usable afterwards
+    ctx.close()
+    hz.run_and_compare_full(cfg, seed=14, float_report=False)
