@@ -50,7 +50,8 @@ enum {
     COMET_ERR_STATE = -3,       /* call out of order (e.g. ffn_up before its inputs)    */
     COMET_ERR_OOM = -4,         /* device allocation failed in comet_init               */
     COMET_ERR_CUDA = -5,        /* a CUDA runtime call failed; see comet_last_cuda_error */
-    COMET_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out                   */
+    COMET_ERR_TIMEOUT = -6,     /* a bounded device-side wait ran out                   */
+    COMET_ERR_SCRATCH_LIMIT = -7 /* problem too large for the built-in static scratch array */
 };
 
 enum { COMET_DEVICE = 0, COMET_HOST = 1 };
@@ -199,6 +200,50 @@ const char* comet_strerror(int code);
 
 /* cudaError_t of the last failing runtime call of this context (0 if none). */
 int comet_last_cuda_error(comet_ctx* ctx);
+
+/* ---------------------------------------------------------------------------
+ * Allocation-free Pi_MatMul.  (The paper has no counterpart; this exists for
+ * deployment reasons only.)
+ *
+ * Some hosts of this library must not, or cannot, allocate device memory at
+ * the moment they need a product: a serving process whose framework has
+ * already handed all of the GPU's memory to its own pool (a raw cudaMalloc
+ * then fails or fights the pool), or a latency-critical loop in which
+ * cudaMalloc/cudaFree would stall the whole device.  comet_init allocates, so
+ * it is closed to them.  This one call needs no context and allocates nothing,
+ * on the host or on the device: it runs one dense Beaver matrix product for
+ * both parties,
+ *     E_i = X_i - A_i,  F_i = Y_i - B_i,  Z_i = C_i + E B_i + A_i F + i E F,
+ * and keeps the four message buffers E_0, E_1, F_0, F_1 -- the only memory the
+ * product needs beyond its inputs and outputs -- in an array that is part of
+ * the library image itself.  That array is COMET_STATIC_SCRATCH_WORDS 64-bit
+ * words (8 MiB); every GPU on which the library is used holds it from the
+ * moment the library is loaded there until the process exits.
+ *
+ * All pointers are DEVICE pointers on the CURRENT device, owned by the caller:
+ * X[i], A[i] are [T, K]; Y[i], B[i] are [N, K] (output-feature-major, like the
+ * weights above); C[i], Z[i] are [T, N]; i = 0, 1 is the party.  K must be a
+ * multiple of 8 and N a multiple of 4.  The work is enqueued on `cuda_stream`
+ * (NULL = default stream) and the call returns without waiting for it.
+ *
+ * Limit: 2 * (T*K + N*K) <= COMET_STATIC_SCRATCH_WORDS, otherwise nothing is
+ * launched and COMET_ERR_SCRATCH_LIMIT is returned.  Other errors: INVALID_ARG
+ * (null pointer), SHAPE (non-positive size or the divisibility rule), CUDA.
+ *
+ * The first call on each device looks up the device address of the array
+ * (once per device; no allocation).  Make that first call outside any stream
+ * capture.
+ *
+ * The array is shared by every call in the process and is never cleared:
+ * a call overwrites all of the part it uses before reading it, so stale
+ * contents are harmless, but two calls whose work overlaps in time on the same
+ * GPU (different streams, or different host threads) race on it.  Serialise
+ * them, e.g. by using one stream.
+ */
+#define COMET_STATIC_SCRATCH_WORDS (1u << 20)
+int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* const X[2], const uint64_t* const A[2],
+                               const uint64_t* const Y[2], const uint64_t* const B[2], const uint64_t* const C[2],
+                               uint64_t* const Z[2], int32_t T, int32_t K, int32_t N);
 
 #ifdef __cplusplus
 }

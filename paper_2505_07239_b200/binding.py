@@ -28,8 +28,10 @@ NUM_TENSORS = 17
 EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
-    "comet_set_profiling",
+    "comet_set_profiling", "comet_beaver_matmul_static",
 )
+STATIC_SCRATCH_WORDS = 1 << 20
+ERR_SCRATCH_LIMIT = -7
 NUM_PHASES = 5
 PHASE_NAMES = ("compact", "open", "prep", "combine", "truncate")
 
@@ -74,6 +76,8 @@ def _load():
     lib.comet_strerror.restype = ctypes.c_char_p
     lib.comet_last_cuda_error.argtypes = [vp]
     lib.comet_set_profiling.argtypes = [vp, ctypes.c_int]
+    pair = ctypes.c_void_p * 2
+    lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
     return lib
 
 
@@ -195,3 +199,29 @@ class Comet:
 def to_device(a: np.ndarray, device="cuda:0") -> torch.Tensor:
     """numpy uint64 -> torch int64 CUDA tensor holding the same words."""
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int64)).to(device)
+
+
+def beaver_matmul_static(X, A, Y, B, C, Z, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Allocation-free dense Beaver product for both parties (comet_beaver_matmul_static).
+
+    For callers that cannot allocate device memory when they need the product
+    (all memory already owned by a framework's pool, or a serving loop that must
+    not stall on cudaMalloc): the message buffers live in an 8 MiB array inside
+    the library.  Each argument is a pair (party 0, party 1) of CUDA tensors of
+    8-byte words on the current device: X, A [T, K]; Y, B [N, K]; C, Z [T, N].
+    Returns the library's status code (0 = ok) instead of raising, so that the
+    size-limit refusal can be observed.  Calls that overlap on the GPU race on
+    the shared array: keep them on one stream.
+    """
+    T, K = X[0].shape
+    N = Y[0].shape[0]
+    pair = ctypes.c_void_p * 2
+
+    def ptrs(ts, shape):
+        for t in ts:
+            assert t.is_cuda and t.is_contiguous() and t.element_size() == 8 and tuple(t.shape) == shape
+        return pair(ts[0].data_ptr(), ts[1].data_ptr())
+
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    return _lib.comet_beaver_matmul_static(sp, ptrs(X, (T, K)), ptrs(A, (T, K)), ptrs(Y, (N, K)), ptrs(B, (N, K)),
+                                           ptrs(C, (T, N)), ptrs(Z, (T, N)), T, K, N)

@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -160,6 +161,8 @@ const char* comet_strerror(int code) {
         case COMET_ERR_OOM: return "device memory allocation failed";
         case COMET_ERR_CUDA: return "a CUDA runtime call failed";
         case COMET_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case COMET_ERR_SCRATCH_LIMIT:
+            return "problem exceeds the library's static scratch array (COMET_STATIC_SCRATCH_WORDS)";
         default: return "unknown error code";
     }
 }
@@ -481,3 +484,84 @@ int comet_set_profiling(comet_ctx* c, int on) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Allocation-free Pi_MatMul: the message buffers live in the library image.
+// ---------------------------------------------------------------------------
+namespace {
+
+// Scratch for E_0, E_1, F_0, F_1 of comet_beaver_matmul_static.  In host code
+// this name is only a handle for cudaGetSymbolAddress, never an address to hand
+// to a kernel; each GPU that loads the library carries its own 8 MiB copy.
+static __device__ __align__(256) unsigned long long g_static_scratch[COMET_STATIC_SCRATCH_WORDS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+u64* g_static_scratch_addr[kMaxDevices] = {};    // device address of the array, per device ordinal
+
+// Device address of the scratch array on the current device (looked up once per device).
+cudaError_t static_scratch_on_current_device(u64** out) {
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        err = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (err != cudaSuccess) return err;
+        g_static_scratch_addr[dev] = static_cast<u64*>(p);
+    }
+    *out = g_static_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* const X[2], const uint64_t* const A[2],
+                                          const uint64_t* const Y[2], const uint64_t* const B[2],
+                                          const uint64_t* const C[2], uint64_t* const Z[2], int32_t T, int32_t K,
+                                          int32_t N) {
+    if (!X || !A || !Y || !B || !C || !Z) return COMET_ERR_INVALID_ARG;
+    for (int p = 0; p < 2; ++p)
+        if (!X[p] || !A[p] || !Y[p] || !B[p] || !C[p] || !Z[p]) return COMET_ERR_INVALID_ARG;
+    if (T < 1 || K < 8 || N < 4 || K % 8 || N % 4) return COMET_ERR_SHAPE;
+    const int64_t left = (int64_t)T * K, right = (int64_t)N * K;
+    if (2 * (left + right) > (int64_t)COMET_STATIC_SCRATCH_WORDS) return COMET_ERR_SCRATCH_LIMIT;
+
+    u64* scratch = nullptr;
+    if (static_scratch_on_current_device(&scratch) != cudaSuccess) {
+        cudaGetLastError();
+        return COMET_ERR_CUDA;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // carve the array: E_0 | E_1 | F_0 | F_1 (every word used below is written before it is read)
+    u64* E[2] = {scratch, scratch + left};
+    u64* F[2] = {scratch + 2 * left, scratch + 2 * left + right};
+
+    comet::PartyPtrs x, a, y, b;
+    comet::PartyOut e, f;
+    comet::CombineArgs args;
+    for (int p = 0; p < 2; ++p) {
+        x.p[p] = reinterpret_cast<const u64*>(X[p]);
+        a.p[p] = reinterpret_cast<const u64*>(A[p]);
+        y.p[p] = reinterpret_cast<const u64*>(Y[p]);
+        b.p[p] = reinterpret_cast<const u64*>(B[p]);
+        e.p[p] = E[p];
+        f.p[p] = F[p];
+        args.E[p] = E[p];
+        args.F[p] = F[p];
+        args.A[p] = a.p[p];
+        args.B[p] = b.p[p];
+        args.C[p] = reinterpret_cast<const u64*>(C[p]);
+        args.Z[p] = reinterpret_cast<u64*>(Z[p]);
+    }
+    args.M = T; args.N = N; args.K = K;
+    auto blocks = [](int64_t pairs) { return (unsigned)((pairs + 255) / 256 < 1184 ? (pairs + 255) / 256 : 1184); };
+    comet::open_activation_kernel<<<dim3(blocks(left / 2), 2), 256, 0, stream>>>(x, a, e, left / 2);
+    comet::open_activation_kernel<<<dim3(blocks(right / 2), 2), 256, 0, stream>>>(y, b, f, right / 2);
+    dim3 grid((N + comet::simt::BN - 1) / comet::simt::BN, (T + comet::simt::BM - 1) / comet::simt::BM, 2);
+    comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, stream>>>(args);
+    if (cudaGetLastError() != cudaSuccess) return COMET_ERR_CUDA;
+    return COMET_OK;
+}
