@@ -11,6 +11,7 @@
 
 #include <cuda_runtime.h>
 
+#include "kernels_limb.cuh"
 #include "kernels_open.cuh"
 #include "kernels_simt.cuh"
 
@@ -25,6 +26,12 @@ struct comet_ctx {
     u64* buf[2][COMET_NUM_TENSORS];
     int64_t cap_words[COMET_NUM_TENSORS];
     bool loaded[2][COMET_NUM_TENSORS];
+    // limb path: blocked limb planes per party (left: E and V_i; right: B_i and F), and the device error flag
+    int path;                     // COMET_PATH_SIMT or COMET_PATH_LIMB
+    uint8_t* planes_left[2][2];
+    uint8_t* planes_right[2][2];
+    size_t planes_left_bytes, planes_right_bytes;
+    int* d_error;
     uint8_t* d_mask;
     int32_t* d_ids;
     int32_t* d_count;
@@ -128,7 +135,61 @@ cudaMemcpyKind copy_kind(int location, bool to_library) {
     return to_library ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
 }
 
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Tensor-core path: Z <- C, blocked limb planes of (E, V_i) and (F, B_i), then the persistent stream-K kernel.
+int launch_combine_limb(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA, int idB, int idC, int idZ) {
+    namespace lb = comet::limb;
+    const int kb = ceil_div(K, lb::KC), mt = ceil_div(M, lb::BM), nt = ceil_div(N, lb::BN);
+    if ((size_t)mt * kb * lb::A_BLOCK_BYTES > c->planes_left_bytes ||
+        (size_t)nt * kb * lb::B_BLOCK_BYTES > c->planes_right_bytes)
+        return COMET_ERR_SHAPE;
+    {
+        PhaseTimer timer(c, COMET_PHASE_PREP, 3);
+        const int64_t pairs = (int64_t)M * N / 2;
+        comet::copy_pairs_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
+            c->buf[0][idC], c->buf[1][idC], c->buf[0][idZ], c->buf[1][idZ], pairs);
+        comet::PlanesArgs l;
+        l.in0 = c->buf[0][idE]; l.in1 = c->buf[1][idE];
+        l.rows = M; l.K = K; l.kblocks = kb; l.tile_rows = lb::BM;
+        comet::PlanesArgs r;
+        r.in0 = c->buf[0][idF]; r.in1 = c->buf[1][idF];
+        r.rows = N; r.K = K; r.kblocks = kb; r.tile_rows = lb::BN;
+        for (int p = 0; p < 2; ++p) {
+            l.in2[p] = c->buf[p][idA]; l.out_sum[p] = c->planes_left[p][0]; l.out_own[p] = c->planes_left[p][1];
+            l.add_sum[p] = p;                      // V_i = A_i + i*E
+            r.in2[p] = c->buf[p][idB]; r.out_sum[p] = c->planes_right[p][1]; r.out_own[p] = c->planes_right[p][0];
+            r.add_sum[p] = 0;                      // B_i as it is
+        }
+        comet::limb_planes_kernel<<<dim3(kb, ceil_div(M, lb::PREP_ROWS), 2), 256, 0, c->stream>>>(l);
+        comet::limb_planes_kernel<<<dim3(kb, ceil_div(N, lb::PREP_ROWS), 2), 256, 0, c->stream>>>(r);
+    }
+    c->stats.kernel_launches += 3;
+    COMET_CUDA(c, cudaGetLastError());
+    comet::LimbArgs a;
+    for (int p = 0; p < 2; ++p) {
+        a.Epl[p] = c->planes_left[p][0];
+        a.Vpl[p] = c->planes_left[p][1];
+        a.Bpl[p] = c->planes_right[p][0];
+        a.Fpl[p] = c->planes_right[p][1];
+        a.Z[p] = c->buf[p][idZ];
+    }
+    a.M = M; a.N = N; a.mt = mt; a.nt = nt; a.kb = kb;
+    a.error_flag = c->d_error;
+    const long long total_units = 2ll * mt * nt * 2 * kb;
+    const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
+    {
+        PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
+        comet::combine_limb_kernel<<<grid, lb::THREADS, lb::SMEM_BYTES, c->stream>>>(a);
+    }
+    c->stats.kernel_launches += 1;
+    c->stats.matmul_path = COMET_PATH_LIMB;
+    COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
 int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA, int idB, int idC, int idZ) {
+    if (c->path == COMET_PATH_LIMB) return launch_combine_limb(c, M, N, K, idE, idF, idA, idB, idC, idZ);
     comet::CombineArgs a;
     for (int p = 0; p < 2; ++p) {
         a.E[p] = c->buf[p][idE];
@@ -216,11 +277,32 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
             if (c->cap_words[id] > 0)
                 ok = cudaMalloc((void**)&c->buf[p][id], (size_t)c->cap_words[id] * sizeof(u64)) == cudaSuccess;
     }
+    c->path = cfg->matmul_path == COMET_PATH_AUTO ? COMET_PATH_SIMT : cfg->matmul_path;
+    if (c->path == COMET_PATH_LIMB) {
+        namespace lb = comet::limb;
+        const int d = cfg->d_model;
+        const int64_t n = c->cap_n, gn = c->groups * n;
+        const int64_t kb_up = (d + lb::KC - 1) / lb::KC, kb_dn = (n + lb::KC - 1) / lb::KC;
+        const int64_t kb_max = kb_up > kb_dn ? kb_up : kb_dn;
+        const int64_t mt = (c->cap_T + lb::BM - 1) / lb::BM;
+        const int64_t right_up = ((gn + lb::BN - 1) / lb::BN) * kb_up, right_dn = ((d + lb::BN - 1) / lb::BN) * kb_dn;
+        c->planes_left_bytes = (size_t)(mt * kb_max) * lb::A_BLOCK_BYTES;
+        c->planes_right_bytes = (size_t)(right_up > right_dn ? right_up : right_dn) * lb::B_BLOCK_BYTES;
+        for (int p = 0; p < 2 && ok; ++p)
+            for (int w = 0; w < 2 && ok; ++w) {
+                ok = cudaMalloc((void**)&c->planes_left[p][w], c->planes_left_bytes) == cudaSuccess;
+                ok = ok && cudaMalloc((void**)&c->planes_right[p][w], c->planes_right_bytes) == cudaSuccess;
+            }
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)lb::SMEM_BYTES) == cudaSuccess;
+    }
+    ok = ok && cudaMalloc((void**)&c->d_error, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_error, 0, sizeof(int)) == cudaSuccess;
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_ids, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_count, sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMallocHost((void**)&c->h_count, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMallocHost((void**)&c->h_count, 2 * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         comet_destroy(c);
@@ -237,6 +319,12 @@ void comet_destroy(comet_ctx* c) {
     for (int id = 0; id < COMET_NUM_TENSORS; ++id)
         for (int p = 0; p < 2; ++p)
             if (c->buf[p][id]) cudaFree(c->buf[p][id]);
+    for (int p = 0; p < 2; ++p)
+        for (int w = 0; w < 2; ++w) {
+            if (c->planes_left[p][w]) cudaFree(c->planes_left[p][w]);
+            if (c->planes_right[p][w]) cudaFree(c->planes_right[p][w]);
+        }
+    if (c->d_error) cudaFree(c->d_error);
     if (c->d_mask) cudaFree(c->d_mask);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
@@ -288,7 +376,9 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     COMET_CUDA(c, cudaMemcpyAsync(c->h_count, c->d_count, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    COMET_CUDA(c, cudaMemcpyAsync(c->h_count + 1, c->d_error, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (c->h_count[1] != 0) return COMET_ERR_TIMEOUT;     // an earlier kernel gave up on a bounded wait
     const int32_t blocks = *c->h_count;
     const int64_t n = (int64_t)blocks * c->cfg.block;
     if (n > c->cap_n) {            // more active neurons than the context was sized for

@@ -1,0 +1,429 @@
+// K4, tensor-core variant: the gathered ring matmul + Beaver combine
+//   Z_i = C_i + E*B_i + A_i*F + i*E*F = C_i + E*B_i + V_i*F,   V_i = A_i + i*E   (Eq. 1, party i)
+// on the int8 tensor cores of sm_100a (tcgen05.mma kind::i8, accumulators in TMEM).
+//
+// A 64-bit ring word is eight unsigned 8-bit limbs, x = sum_p x_p 2^(8p).  Mod 2^64 only limb pairs with
+// p + q <= 7 matter: x*y = sum_{s=0..7} 2^(8s) D_s, D_s = sum_{p+q=s} x_p y_q (36 of the 64 limb products).
+// Each D_s summed over the contraction index is one 32-bit accumulator per output element: 8 accumulators
+// of 128 x 64 fill the 512 TMEM columns of an SM exactly.  Only D_s mod 2^(64-8s) is needed, so 32-bit
+// wrap-around is harmless for s >= 4, and for s <= 3 the exact sum (s+1)*K*255^2 stays below 2^32 while a
+// segment accumulates at most 16384 contraction elements.
+//
+// Operands are kept as "blocked limb planes": for a tile of R rows (128 left, 64 right) and a block of 32
+// contraction elements, 8 planes of R x 32 bytes, each stored as the tensor core's K-major no-swizzle
+// canonical layout (8-row x 16-byte core matrices; the two 16-byte K halves of a row group adjacent).  One
+// block is one contiguous bulk copy into shared memory.  With the planes of the right operand stacked
+// along N, limb plane p of the left operand meets planes 0..7-p of the right operand in ONE instruction
+// whose N spans accumulators D_p..D_7 (split in two when N > 256): 12 instructions per 32-deep step.
+//
+// Work is split stream-K style over a persistent grid: the (party, tile, k-block) space is cut into equal
+// contiguous ranges, every segment's partial sums are added to Z with red.global.add.u64 -- exact and
+// order-independent in the ring -- and Z is pre-loaded with C_i.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace comet {
+
+typedef unsigned long long u64;
+
+namespace limb {
+constexpr int BM = 128, BN = 64, KC = 32, PLANES = 8;
+constexpr int A_BLOCK_BYTES = PLANES * BM * KC;   // 32 KiB
+constexpr int B_BLOCK_BYTES = PLANES * BN * KC;   // 16 KiB
+constexpr int STAGES = 4;
+constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <= 3 below 2^32
+constexpr int THREADS = 192;                      // warps 0-3 epilogue, warp 4 copy producer, warp 5 MMA issuer
+constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
+constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + 1024;
+constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s at 1.9 GHz: every wait gives up after this
+constexpr unsigned LBO_BYTES = 128, SBO_BYTES = 256;
+
+// byte offset of (plane p, row r, contraction index k in [0,32)) inside a block of `rows` rows
+__host__ __device__ __forceinline__ int block_offset(int rows, int p, int r, int k) {
+    return p * rows * KC + (r >> 3) * 256 + (k >> 4) * 128 + (r & 7) * 16 + (k & 15);
+}
+}  // namespace limb
+
+// ---------------------------------------------------------------------------
+// Operand preparation after the exchange: blocked limb planes of
+//   S = in0 + in1              (the opened value E or F; identical for both parties, one copy each)
+//   W = in2 + (add_sum ? S : 0) (the party's own operand: V_i = A_i + i*E on the left, B_i on the right)
+// grid = (k-blocks, ceil(rows / 64), party); 256 threads; rows/k beyond the logical size are zero.
+// ---------------------------------------------------------------------------
+struct PlanesArgs {
+    const u64* in0;          // message of party 0, [rows, K]
+    const u64* in1;          // message of party 1
+    const u64* in2[2];       // party's own share
+    uint8_t* out_sum[2];     // blocked planes of S, per party
+    uint8_t* out_own[2];     // blocked planes of W, per party
+    int add_sum[2];
+    int rows, K;             // logical sizes (K multiple of 16)
+    int kblocks;             // ceil(K / 32)
+    int tile_rows;           // 128 (left operand) or 64 (right operand)
+};
+
+__device__ __forceinline__ void limb_transpose4(unsigned x0, unsigned x1, unsigned x2, unsigned x3,
+                                                unsigned& p0, unsigned& p1, unsigned& p2, unsigned& p3) {
+    const unsigned t0 = __byte_perm(x0, x1, 0x5140), t1 = __byte_perm(x2, x3, 0x5140);
+    const unsigned t2 = __byte_perm(x0, x1, 0x7362), t3 = __byte_perm(x2, x3, 0x7362);
+    p0 = __byte_perm(t0, t1, 0x5410);
+    p1 = __byte_perm(t0, t1, 0x7632);
+    p2 = __byte_perm(t2, t3, 0x5410);
+    p3 = __byte_perm(t2, t3, 0x7632);
+}
+
+__global__ void __launch_bounds__(256)
+limb_planes_kernel(PlanesArgs a) {
+    using namespace limb;
+    __shared__ u64 sS[PREP_ROWS][KC + 1];
+    __shared__ u64 sW[PREP_ROWS][KC + 1];
+    const int party = blockIdx.z;
+    const int kb = blockIdx.x;
+    const int row0 = blockIdx.y * PREP_ROWS;
+    const int tid = threadIdx.x;
+    const u64* __restrict__ in2 = party ? a.in2[1] : a.in2[0];
+    const bool add = (party ? a.add_sum[1] : a.add_sum[0]) != 0;
+
+    // phase 1: coalesced 16-byte loads, 16 threads per row
+    {
+        const int kk = (tid & 15) * 2;
+        const int k = kb * KC + kk;
+#pragma unroll
+        for (int it = 0; it < PREP_ROWS / 16; ++it) {
+            const int r = it * 16 + (tid >> 4);
+            const int row = row0 + r;
+            u64 s0 = 0, s1 = 0, w0 = 0, w1 = 0;
+            if (row < a.rows && k < a.K) {
+                const size_t o = (size_t)row * a.K + k;
+                const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(a.in0 + o));
+                const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(a.in1 + o));
+                const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(in2 + o));
+                s0 = x.x + y.x;
+                s1 = x.y + y.y;
+                w0 = z.x + (add ? s0 : 0ull);
+                w1 = z.y + (add ? s1 : 0ull);
+            }
+            sS[r][kk] = s0;
+            sS[r][kk + 1] = s1;
+            sW[r][kk] = w0;
+            sW[r][kk + 1] = w1;
+        }
+    }
+    __syncthreads();
+
+    // phase 2: one thread per (output, 16-k half, row): split 16 words into 8 limb planes of 16 bytes
+    {
+        const int which = tid >> 7;              // 0: S, 1: W
+        const int half = (tid >> 6) & 1;
+        const int r = tid & 63;
+        const u64(*src)[KC + 1] = which ? sW : sS;
+        unsigned lo[16], hi[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const u64 v = src[r][half * 16 + j];
+            lo[j] = (unsigned)v;
+            hi[j] = (unsigned)(v >> 32);
+        }
+        uint4 plane[8];
+        limb_transpose4(lo[0], lo[1], lo[2], lo[3], plane[0].x, plane[1].x, plane[2].x, plane[3].x);
+        limb_transpose4(lo[4], lo[5], lo[6], lo[7], plane[0].y, plane[1].y, plane[2].y, plane[3].y);
+        limb_transpose4(lo[8], lo[9], lo[10], lo[11], plane[0].z, plane[1].z, plane[2].z, plane[3].z);
+        limb_transpose4(lo[12], lo[13], lo[14], lo[15], plane[0].w, plane[1].w, plane[2].w, plane[3].w);
+        limb_transpose4(hi[0], hi[1], hi[2], hi[3], plane[4].x, plane[5].x, plane[6].x, plane[7].x);
+        limb_transpose4(hi[4], hi[5], hi[6], hi[7], plane[4].y, plane[5].y, plane[6].y, plane[7].y);
+        limb_transpose4(hi[8], hi[9], hi[10], hi[11], plane[4].z, plane[5].z, plane[6].z, plane[7].z);
+        limb_transpose4(hi[12], hi[13], hi[14], hi[15], plane[4].w, plane[5].w, plane[6].w, plane[7].w);
+
+        const int row = row0 + r;
+        const int tile = row / a.tile_rows, rin = row - tile * a.tile_rows;
+        uint8_t* base = which ? (party ? a.out_own[1] : a.out_own[0]) : (party ? a.out_sum[1] : a.out_sum[0]);
+        uint8_t* blk = base + ((size_t)tile * a.kblocks + kb) * (size_t)(PLANES * a.tile_rows * KC);
+#pragma unroll
+        for (int p = 0; p < 8; ++p)
+            *reinterpret_cast<uint4*>(blk + block_offset(a.tile_rows, p, rin, half * 16)) = plane[p];
+    }
+}
+
+// Z_i <- C_i (the accumulation target of the tensor-core kernel starts from the triple's C share)
+__global__ void __launch_bounds__(256)
+copy_pairs_kernel(const u64* s0, const u64* s1, u64* d0, u64* d1, int64_t pairs) {
+    const ulonglong2* __restrict__ s = reinterpret_cast<const ulonglong2*>(blockIdx.y ? s1 : s0);
+    ulonglong2* __restrict__ d = reinterpret_cast<ulonglong2*>(blockIdx.y ? d1 : d0);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < pairs; t += stride) d[t] = __ldg(s + t);
+}
+
+// ---------------------------------------------------------------------------
+// PTX wrappers (sm_100a)
+// ---------------------------------------------------------------------------
+namespace ptx {
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* d) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+}  // namespace ptx
+
+struct LimbArgs {
+    const uint8_t* Epl[2];   // left planes of E = E_0 + E_1, per party: [m-tile][k-block][32 KiB]
+    const uint8_t* Vpl[2];   // left planes of V_i = A_i + i*E
+    const uint8_t* Bpl[2];   // right planes of B_i: [n-tile][k-block][16 KiB]
+    const uint8_t* Fpl[2];   // right planes of F = F_0 + F_1
+    u64* Z[2];               // [M, N], pre-loaded with C_i; partial sums are added atomically
+    int M, N;
+    int mt, nt, kb;          // tiles and k-blocks per operand pair; one tile runs over 2*kb blocks
+    int* error_flag;         // set to 1 if a bounded wait ran out
+};
+
+// Bounded wait: false (and the CTA-wide abort flag raised) if the barrier did not flip in time or another
+// role already gave up.
+__device__ __forceinline__ bool limb_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limb::WAIT_CYCLES) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ uint64_t limb_smem_desc(uint32_t addr) {
+    // K-major, no swizzle: bits 0-13 address>>4, 16-29 leading byte offset>>4 (between the two 16-byte K
+    // halves), 32-45 stride byte offset>>4 (between 8-row groups), 46-47 descriptor version 1
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(limb::LBO_BYTES >> 4) << 16) |
+           ((uint64_t)(limb::SBO_BYTES >> 4) << 32) | (1ull << 46);
+}
+
+__global__ void __launch_bounds__(limb::THREADS, 1)
+combine_limb_kernel(LimbArgs a) {
+    using namespace limb;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[STAGES];
+    __shared__ __align__(8) uint64_t empty_bar[STAGES];
+    __shared__ __align__(8) uint64_t accum_full_bar, accum_empty_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + (size_t)STAGES * A_BLOCK_BYTES;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long tile_units = 2ll * a.kb;
+    const long long total_units = 2ll * a.mt * a.nt * tile_units;
+    const long long u_begin = total_units * blockIdx.x / gridDim.x;
+    const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_u32(&accum_full_bar), 1);
+        ptx::mbar_init(ptx::smem_u32(&accum_empty_bar), 128);
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    if (warp == 0) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::fence_before_sync();
+    __syncthreads();
+    ptx::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 4) {
+        // ---------------- producer: one bulk copy per operand block ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (long long u = u_begin; u < u_end && ok; ++u) {
+                ok = limb_wait(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag);
+                if (!ok) break;
+                const long long tile = u / tile_units;
+                int kpos = (int)(u - tile * tile_units);
+                const int per_party = a.mt * a.nt;
+                const int party = (int)(tile / per_party);
+                const int t2 = (int)(tile - (long long)party * per_party);
+                const int tm = t2 / a.nt, tn = t2 - tm * a.nt;
+                const bool second = kpos >= a.kb;
+                if (second) kpos -= a.kb;
+                const uint8_t* left = second ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]);
+                const uint8_t* right = second ? (party ? a.Fpl[1] : a.Fpl[0]) : (party ? a.Bpl[1] : a.Bpl[0]);
+                const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
+                ptx::mbar_expect_tx(bar, A_BLOCK_BYTES + B_BLOCK_BYTES);
+                ptx::bulk_g2s(ptx::smem_u32(sA + (size_t)stage * A_BLOCK_BYTES),
+                              left + ((size_t)tm * a.kb + kpos) * A_BLOCK_BYTES, A_BLOCK_BYTES, bar);
+                ptx::bulk_g2s(ptx::smem_u32(sB + (size_t)stage * B_BLOCK_BYTES),
+                              right + ((size_t)tn * a.kb + kpos) * B_BLOCK_BYTES, B_BLOCK_BYTES, bar);
+                ++issued;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) {
+                // gave up: let the copies already in flight land before the CTA leaves
+                const int back = issued < STAGES ? issued : STAGES;
+                for (int j = 1; j <= back; ++j) {
+                    int s = stage - j;
+                    uint32_t ph = phase;
+                    if (s < 0) { s += STAGES; ph ^= 1u; }
+                    const long long t0 = clock64();
+                    while (!ptx::mbar_try_wait(ptx::smem_u32(&full_bar[s]), ph) && clock64() - t0 < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc0 = (2u << 4) | ((uint32_t)(BM >> 4) << 24);   // s32 accumulate, u8 x u8, K-major
+            int stage = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            long long u = u_begin;
+            while (u < u_end && ok) {
+                const long long tile = u / tile_units;
+                long long seg_end = (tile + 1) * tile_units;
+                if (seg_end > u_end) seg_end = u_end;
+                if (seg_end > u + MAX_SEGMENT_UNITS) seg_end = u + MAX_SEGMENT_UNITS;
+                ok = limb_wait(ptx::smem_u32(&accum_empty_bar), acc_phase ^ 1u, &abort_flag);
+                if (!ok) break;
+                ptx::fence_after_sync();
+                bool first = true;
+                for (; u < seg_end; ++u) {
+                    ok = limb_wait(ptx::smem_u32(&full_bar[stage]), phase, &abort_flag);
+                    if (!ok) break;
+                    ptx::fence_after_sync();
+                    const uint32_t a_addr = ptx::smem_u32(sA + (size_t)stage * A_BLOCK_BYTES);
+                    const uint32_t b_addr = ptx::smem_u32(sB + (size_t)stage * B_BLOCK_BYTES);
+                    const uint64_t bdesc0 = limb_smem_desc(b_addr);
+                    const uint64_t bdesc1 = limb_smem_desc(b_addr + 256 * KC);   // right-operand rows 256.. (planes 4..)
+#pragma unroll
+                    for (int p = 0; p < PLANES; ++p) {
+                        const uint64_t adesc = limb_smem_desc(a_addr + p * BM * KC);
+                        const int n_total = BN * (PLANES - p);
+                        const int n0 = n_total > 256 ? 256 : n_total;
+                        const uint32_t acc = (first && p == 0) ? 0u : 1u;
+                        ptx::mma_i8(tmem_base + BN * p, adesc, bdesc0, idesc0 | ((uint32_t)(n0 >> 3) << 17), acc);
+                        if (n_total > 256)
+                            ptx::mma_i8(tmem_base + BN * p + 256, adesc, bdesc1,
+                                        idesc0 | ((uint32_t)((n_total - 256) >> 3) << 17), acc);
+                    }
+                    ptx::mma_commit(ptx::smem_u32(&empty_bar[stage]));    // frees the stage once the MMAs have read it
+                    first = false;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                ptx::mma_commit(ptx::smem_u32(&accum_full_bar));
+                acc_phase ^= 1u;
+            }
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> red.add into Z ----------------
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        long long u = u_begin;
+        while (u < u_end && ok) {
+            const long long tile = u / tile_units;
+            long long seg_end = (tile + 1) * tile_units;
+            if (seg_end > u_end) seg_end = u_end;
+            if (seg_end > u + MAX_SEGMENT_UNITS) seg_end = u + MAX_SEGMENT_UNITS;
+            u = seg_end;
+            const int per_party = a.mt * a.nt;
+            const int party = (int)(tile / per_party);
+            const int t2 = (int)(tile - (long long)party * per_party);
+            const int tm = t2 / a.nt, tn = t2 - tm * a.nt;
+            ok = limb_wait(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
+            ok = __all_sync(0xffffffffu, ok);          // also reconverges the warp for the aligned TMEM loads
+            if (!ok) break;
+            ptx::fence_after_sync();
+            const int row = tm * BM + warp * 32 + lane;
+            u64* __restrict__ zrow = (party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N;
+            const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 8) {
+                uint32_t d[PLANES][8];
+#pragma unroll
+                for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c0, d[s]);
+                ptx::tmem_wait_ld();
+                const int col = tn * BN + c0;
+                if (row < a.M && col < a.N) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        u64 z = (u64)d[0][j];
+#pragma unroll
+                        for (int s = 1; s < PLANES; ++s) z += (u64)d[s][j] << (8 * s);
+                        atomicAdd(zrow + col + j, z);
+                    }
+                }
+            }
+            ptx::fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
+            acc_phase ^= 1u;
+        }
+    }
+
+    ptx::fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) *a.error_flag = 1;
+    if (warp == 0) {
+        ptx::fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace comet

@@ -20,17 +20,19 @@ def hz():
     return harness
 
 
-def _ok(report):
+def _ok(report, path=None):
     assert report["mismatches"] == 0, [c for c in report["compared"] if c[2]]
+    if path is not None:
+        assert report["path"] == path, "the requested matmul path did not run"
     return report
 
 
-PATHS = [1]   # COMET_PATH_SIMT
+PATHS = [1, 2]   # COMET_PATH_SIMT, COMET_PATH_LIMB
 
 
 @pytest.mark.parametrize("path", PATHS)
 def test_tiny_full(hz, path):
-    r = _ok(hz.run_and_compare_full(wl.CONFIGS["tiny"], seed=1, matmul_path=path))
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["tiny"], seed=1, matmul_path=path), path)
     assert r["n_active"] == 96 and r["up_reconstructs"]
     # 12 fractional bits, |w| <= 1, 96 active neurons: bounded by n * 2^-f, not by 2^-10
     assert r["float64_max_abs_err"] < 96 * 2.0 ** -12
@@ -38,14 +40,14 @@ def test_tiny_full(hz, path):
 
 @pytest.mark.parametrize("path", PATHS)
 def test_opt125m_full(hz, path):
-    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=2, matmul_path=path))
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=2, matmul_path=path), path)
     assert r["n_active"] == 320 and r["up_reconstructs"]
     assert r["float64_max_abs_err"] < 2.0 ** -10
 
 
 @pytest.mark.parametrize("path", PATHS)
 def test_opt13b_95_full(hz, path):
-    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt1.3b"], seed=3, sparsity=0.95, matmul_path=path))
+    r = _ok(hz.run_and_compare_full(wl.CONFIGS["opt1.3b"], seed=3, sparsity=0.95, matmul_path=path), path)
     assert r["n_active"] == 416 and r["up_reconstructs"]
     assert r["float64_max_abs_err"] < 2.0 ** -10
 
@@ -53,13 +55,13 @@ def test_opt13b_95_full(hz, path):
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("tokens", [1, 17, 130])
 def test_ragged_token_counts(hz, path, tokens):
-    _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=4, tokens=tokens, matmul_path=path, float_report=False))
+    _ok(hz.run_and_compare_full(wl.CONFIGS["opt125m"], seed=4, tokens=tokens, matmul_path=path, float_report=False), path)
 
 
 @pytest.mark.parametrize("path", PATHS)
 def test_gated_small(hz, path):
     cfg = wl.FFNConfig("gated-small", 40, 128, 512, 64, 16, True, 0.25, "uniform", "normal", "normal0.02")
-    r = _ok(hz.run_and_compare_full(cfg, seed=5, matmul_path=path))
+    r = _ok(hz.run_and_compare_full(cfg, seed=5, matmul_path=path), path)
     assert r["n_active"] == 128 and r["up_reconstructs"]
     assert r["float64_max_abs_err"] < 2.0 ** -10
 
@@ -67,7 +69,7 @@ def test_gated_small(hz, path):
 @pytest.mark.parametrize("path", PATHS)
 def test_all_ones_mask_is_the_dense_product(hz, path):
     cfg = wl.CONFIGS["tiny"]
-    r = _ok(hz.run_and_compare_full(cfg, seed=6, sparsity=0.0, matmul_path=path))
+    r = _ok(hz.run_and_compare_full(cfg, seed=6, sparsity=0.0, matmul_path=path), path)
     assert r["n_active"] == cfg.d_ff and r["up_reconstructs"]
 
 
@@ -77,19 +79,19 @@ def test_single_block_first_and_last(hz, path):
     for b in (0, cfg.n_blocks - 1):
         m = np.zeros(cfg.n_blocks, np.uint8)
         m[b] = 1
-        r = _ok(hz.run_and_compare_full(cfg, seed=7, mask=m, matmul_path=path, float_report=False))
+        r = _ok(hz.run_and_compare_full(cfg, seed=7, mask=m, matmul_path=path, float_report=False), path)
         assert r["n_active"] == cfg.block
 
 
 @pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("sparsity", [0.0, 0.5, 0.8, 0.9])
 def test_opt13b_sweep_sampled(hz, path, sparsity):
-    _ok(hz.run_and_compare_sampled(wl.CONFIGS["opt1.3b"], seed=8, sparsity=sparsity, matmul_path=path))
+    _ok(hz.run_and_compare_sampled(wl.CONFIGS["opt1.3b"], seed=8, sparsity=sparsity, matmul_path=path), path)
 
 
 @pytest.mark.parametrize("path", PATHS)
 def test_llama7b_sampled(hz, path):
-    r = _ok(hz.run_and_compare_sampled(wl.CONFIGS["llama7b"], seed=9, matmul_path=path))
+    r = _ok(hz.run_and_compare_sampled(wl.CONFIGS["llama7b"], seed=9, matmul_path=path), path)
     assert 23 * 64 <= r["n_active"] <= 26 * 64
 
 
@@ -101,7 +103,7 @@ def test_opt67b_decode_steps_sampled(hz, path):
     hz.load_weights(ctx, cfg, W)
     for step in (0, 1, 63):       # fresh mask, X and triples per step, weights loaded once
         r = _ok(hz.run_and_compare_sampled(cfg, seed=10, step=step, matmul_path=path, ctx=ctx, weights=W,
-                                           samples=256))
+                                           samples=256), path)
         assert r["n_active"] == 1312
     ctx.close()
 
