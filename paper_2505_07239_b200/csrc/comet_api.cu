@@ -277,7 +277,7 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
             if (c->cap_words[id] > 0)
                 ok = cudaMalloc((void**)&c->buf[p][id], (size_t)c->cap_words[id] * sizeof(u64)) == cudaSuccess;
     }
-    c->path = cfg->matmul_path == COMET_PATH_AUTO ? COMET_PATH_SIMT : cfg->matmul_path;
+    c->path = cfg->matmul_path == COMET_PATH_AUTO ? COMET_PATH_LIMB : cfg->matmul_path;
     if (c->path == COMET_PATH_LIMB) {
         namespace lb = comet::limb;
         const int d = cfg->d_model;
