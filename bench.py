@@ -249,8 +249,10 @@ def main():
     macs = ffn_macs(cfg, T, n)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     y_host = [torch.empty((T, d), dtype=torch.int64).pin_memory() for _ in (0, 1)]
-    UP_IDS = (cb.X, cb.A_UP, cb.B_UP, cb.C_UP)
-    DN_IDS = (cb.H, cb.A_DN, cb.B_DN, cb.C_DN)
+    # everything except the hidden state is known before the up-projection starts (the down-projection's
+    # triple included); H stands for the output of the activation step that sits between the projections
+    UP_IDS = (cb.X, cb.A_UP, cb.B_UP, cb.C_UP, cb.A_DN, cb.B_DN, cb.C_DN)
+    DN_IDS = (cb.H,)
 
     def ev():
         return torch.cuda.Event(enable_timing=True)

@@ -127,7 +127,10 @@ typedef struct {
 /* Create a context: validates the configuration, selects the device, and
  * allocates every buffer the later calls use (shares, triples, messages,
  * results) for the stated capacities.  `cuda_stream` is a cudaStream_t (NULL =
- * the default stream); the library never creates or destroys streams.
+ * the default stream) on which all calls are ordered.  The tensor-core path
+ * also owns one internal non-blocking stream, forked from and joined back into
+ * `cuda_stream` with events, on which comet_ffn_up opens the weight side of the
+ * down-projection early when W2 and B_DN are already loaded.
  * Errors: INVALID_ARG, SHAPE (divisibility rules above), OOM, CUDA. */
 int comet_init(const comet_config* config, void* cuda_stream, comet_ctx** out);
 

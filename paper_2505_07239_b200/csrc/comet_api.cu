@@ -28,10 +28,17 @@ struct comet_ctx {
     bool loaded[2][COMET_NUM_TENSORS];
     // limb path: blocked limb planes per party (left: E and V_i; right: B_i and F), and the device error flag
     int path;                     // COMET_PATH_SIMT or COMET_PATH_LIMB
-    uint8_t* planes_left[2][2];
-    uint8_t* planes_right[2][2];
-    size_t planes_left_bytes, planes_right_bytes;
-    int* d_error;
+    uint8_t* planes_left[2][2];       // [party][E, V_i]; shared by the two projections
+    uint8_t* planes_right_up[2][2];   // [party][B_i, F] of the up-projection
+    uint8_t* planes_right_dn[2][2];   // [party][B'_i, F'] of the down-projection
+    size_t planes_left_bytes, planes_right_up_bytes, planes_right_dn_bytes;
+    int* d_error;                     // = d_count + 1
+    // the weight side of the down-projection is opened on a second stream while the up-projection's
+    // tensor-core kernel runs (it only needs the mask, W2 and B'_i)
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_join;
+    bool side_pending;                // ev_join not yet waited for on the main stream
+    bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
     uint8_t* d_mask;
     int32_t* d_ids;
     int32_t* d_count;
@@ -137,44 +144,111 @@ cudaMemcpyKind copy_kind(int location, bool to_library) {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// Tensor-core path: Z <- C, blocked limb planes of (E, V_i) and (F, B_i), then the persistent stream-K kernel.
-int launch_combine_limb(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA, int idB, int idC, int idZ) {
-    namespace lb = comet::limb;
-    const int kb = ceil_div(K, lb::KC), mt = ceil_div(M, lb::BM), nt = ceil_div(N, lb::BN);
-    if ((size_t)mt * kb * lb::A_BLOCK_BYTES > c->planes_left_bytes ||
-        (size_t)nt * kb * lb::B_BLOCK_BYTES > c->planes_right_bytes)
-        return COMET_ERR_SHAPE;
-    {
-        PhaseTimer timer(c, COMET_PHASE_PREP, 3);
-        const int64_t pairs = (int64_t)M * N / 2;
-        comet::copy_pairs_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
-            c->buf[0][idC], c->buf[1][idC], c->buf[0][idZ], c->buf[1][idZ], pairs);
-        comet::PlanesArgs l;
-        l.in0 = c->buf[0][idE]; l.in1 = c->buf[1][idE];
-        l.rows = M; l.K = K; l.kblocks = kb; l.tile_rows = lb::BM;
-        comet::PlanesArgs r;
-        r.in0 = c->buf[0][idF]; r.in1 = c->buf[1][idF];
-        r.rows = N; r.K = K; r.kblocks = kb; r.tile_rows = lb::BN;
-        for (int p = 0; p < 2; ++p) {
-            l.in2[p] = c->buf[p][idA]; l.out_sum[p] = c->planes_left[p][0]; l.out_own[p] = c->planes_left[p][1];
-            l.add_sum[p] = p;                      // V_i = A_i + i*E
-            r.in2[p] = c->buf[p][idB]; r.out_sum[p] = c->planes_right[p][1]; r.out_own[p] = c->planes_right[p][0];
-            r.add_sum[p] = 0;                      // B_i as it is
-        }
-        comet::limb_planes_kernel<<<dim3(kb, ceil_div(M, lb::PREP_ROWS), 2), 256, 0, c->stream>>>(l);
-        comet::limb_planes_kernel<<<dim3(kb, ceil_div(N, lb::PREP_ROWS), 2), 256, 0, c->stream>>>(r);
+// One Pi_MatMul of the path: sizes and tensor ids.
+struct Proj {
+    int M, N, K;
+    int idX, idA, idE, idB, idF, idC, idZ;
+    bool down;
+};
+
+Proj proj_up(const comet_ctx* c, int tokens) {
+    return Proj{tokens, c->groups * c->n_active, c->cfg.d_model, COMET_X, COMET_A_UP, COMET_E_UP, COMET_B_UP,
+                COMET_F_UP, COMET_C_UP, COMET_Z_UP, false};
+}
+Proj proj_down(const comet_ctx* c, int tokens) {
+    return Proj{tokens, c->cfg.d_model, c->n_active, COMET_H, COMET_A_DN, COMET_E_DN, COMET_B_DN, COMET_F_DN,
+                COMET_C_DN, COMET_Y, true};
+}
+
+// Makes the main stream wait for the side stream's outstanding work (if any).
+int join_side(comet_ctx* c) {
+    if (c->side_pending) {
+        COMET_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_join, 0));
+        c->side_pending = false;
     }
-    c->stats.kernel_launches += 3;
+    return COMET_OK;
+}
+
+// Tensor-core path, before the exchange: E_i (left) and/or F_i + planes(B_i) (right), one launch.
+int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t stream) {
+    namespace lb = comet::limb;
+    comet::LimbOpenArgs a;
+    std::memset(&a, 0, sizeof(a));
+    const int kb = ceil_div(pr.K, lb::KC);
+    uint8_t* (*planes)[2] = pr.down ? c->planes_right_dn : c->planes_right_up;
+    for (int p = 0; p < 2; ++p) {
+        a.X[p] = c->buf[p][pr.idX];
+        a.A[p] = c->buf[p][pr.idA];
+        a.E[p] = c->buf[p][pr.idE];
+        a.W0[p] = pr.down ? c->buf[p][COMET_W2] : (c->groups == 2 ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1]);
+        a.W1[p] = c->buf[p][COMET_W1];
+        a.B[p] = c->buf[p][pr.idB];
+        a.F[p] = c->buf[p][pr.idF];
+        a.Bpl[p] = planes[p][0];
+    }
+    a.left_pairs = left ? (long long)pr.M * pr.K / 2 : 0;
+    a.left_blocks = left ? ew_grid(c, a.left_pairs, 256) : 0;
+    a.ids = c->d_ids;
+    a.n = c->n_active;
+    a.bs = c->cfg.block;
+    a.rows = pr.N;
+    a.K = pr.K;
+    a.ldw = pr.down ? c->cfg.d_ff : c->cfg.d_model;
+    a.kblocks = kb;
+    a.down = pr.down ? 1 : 0;
+    const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
+    if (a.left_blocks + right_tiles == 0) return COMET_OK;
+    comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
+    c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
+// Tensor-core path, after the exchange: planes(E), planes(V_i) (left), planes(F) (right), Z <- C, one launch.
+int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cudaStream_t stream) {
+    namespace lb = comet::limb;
+    comet::LimbPrepArgs a;
+    std::memset(&a, 0, sizeof(a));
+    const int kb = ceil_div(pr.K, lb::KC);
+    uint8_t* (*planes)[2] = pr.down ? c->planes_right_dn : c->planes_right_up;
+    a.E0 = c->buf[0][pr.idE]; a.E1 = c->buf[1][pr.idE];
+    a.F0 = c->buf[0][pr.idF]; a.F1 = c->buf[1][pr.idF];
+    for (int p = 0; p < 2; ++p) {
+        a.A[p] = c->buf[p][pr.idA];
+        a.Epl[p] = c->planes_left[p][0];
+        a.Vpl[p] = c->planes_left[p][1];
+        a.Fpl[p] = planes[p][1];
+        a.C[p] = c->buf[p][pr.idC];
+        a.Z[p] = c->buf[p][pr.idZ];
+    }
+    a.M = pr.M; a.N = pr.N; a.K = pr.K; a.kblocks = kb;
+    a.left_tiles = left ? kb * ceil_div(pr.M, lb::PREP_ROWS) : 0;
+    a.right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
+    a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
+    a.copy_blocks = copy ? ew_grid(c, a.copy_pairs, 256) : 0;
+    const int blocks = a.left_tiles + a.right_tiles + a.copy_blocks;
+    if (blocks == 0) return COMET_OK;
+    const size_t smem = (left ? 2 : 1) * sizeof(comet::LimbTile);
+    comet::limb_prep_kernel<<<dim3(blocks, 2), 256, smem, stream>>>(a);
+    c->stats.kernel_launches += 1;
+    COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
+// Tensor-core path: the persistent stream-K kernel over both parties' tiles.
+int limb_combine(comet_ctx* c, const Proj& pr) {
+    namespace lb = comet::limb;
+    const int kb = ceil_div(pr.K, lb::KC), mt = ceil_div(pr.M, lb::BM), nt = ceil_div(pr.N, lb::BN);
+    uint8_t* (*planes)[2] = pr.down ? c->planes_right_dn : c->planes_right_up;
     comet::LimbArgs a;
     for (int p = 0; p < 2; ++p) {
         a.Epl[p] = c->planes_left[p][0];
         a.Vpl[p] = c->planes_left[p][1];
-        a.Bpl[p] = c->planes_right[p][0];
-        a.Fpl[p] = c->planes_right[p][1];
-        a.Z[p] = c->buf[p][idZ];
+        a.Bpl[p] = planes[p][0];
+        a.Fpl[p] = planes[p][1];
+        a.Z[p] = c->buf[p][pr.idZ];
     }
-    a.M = M; a.N = N; a.mt = mt; a.nt = nt; a.kb = kb;
+    a.M = pr.M; a.N = pr.N; a.mt = mt; a.nt = nt; a.kb = kb;
     a.error_flag = c->d_error;
     const long long total_units = 2ll * mt * nt * 2 * kb;
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
@@ -188,8 +262,14 @@ int launch_combine_limb(comet_ctx* c, int M, int N, int K, int idE, int idF, int
     return COMET_OK;
 }
 
+bool limb_fits(const comet_ctx* c, const Proj& pr) {
+    namespace lb = comet::limb;
+    const size_t kb = ceil_div(pr.K, lb::KC), mt = ceil_div(pr.M, lb::BM), nt = ceil_div(pr.N, lb::BN);
+    return mt * kb * lb::A_BLOCK_BYTES <= c->planes_left_bytes &&
+           nt * kb * lb::B_BLOCK_BYTES <= (pr.down ? c->planes_right_dn_bytes : c->planes_right_up_bytes);
+}
+
 int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA, int idB, int idC, int idZ) {
-    if (c->path == COMET_PATH_LIMB) return launch_combine_limb(c, M, N, K, idE, idF, idA, idB, idC, idZ);
     comet::CombineArgs a;
     for (int p = 0; p < 2; ++p) {
         a.E[p] = c->buf[p][idE];
@@ -285,23 +365,27 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
         const int64_t kb_up = (d + lb::KC - 1) / lb::KC, kb_dn = (n + lb::KC - 1) / lb::KC;
         const int64_t kb_max = kb_up > kb_dn ? kb_up : kb_dn;
         const int64_t mt = (c->cap_T + lb::BM - 1) / lb::BM;
-        const int64_t right_up = ((gn + lb::BN - 1) / lb::BN) * kb_up, right_dn = ((d + lb::BN - 1) / lb::BN) * kb_dn;
         c->planes_left_bytes = (size_t)(mt * kb_max) * lb::A_BLOCK_BYTES;
-        c->planes_right_bytes = (size_t)(right_up > right_dn ? right_up : right_dn) * lb::B_BLOCK_BYTES;
+        c->planes_right_up_bytes = (size_t)(((gn + lb::BN - 1) / lb::BN) * kb_up) * lb::B_BLOCK_BYTES;
+        c->planes_right_dn_bytes = (size_t)(((d + lb::BN - 1) / lb::BN) * kb_dn) * lb::B_BLOCK_BYTES;
         for (int p = 0; p < 2 && ok; ++p)
             for (int w = 0; w < 2 && ok; ++w) {
                 ok = cudaMalloc((void**)&c->planes_left[p][w], c->planes_left_bytes) == cudaSuccess;
-                ok = ok && cudaMalloc((void**)&c->planes_right[p][w], c->planes_right_bytes) == cudaSuccess;
+                ok = ok && cudaMalloc((void**)&c->planes_right_up[p][w], c->planes_right_up_bytes) == cudaSuccess;
+                ok = ok && cudaMalloc((void**)&c->planes_right_dn[p][w], c->planes_right_dn_bytes) == cudaSuccess;
             }
         ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)lb::SMEM_BYTES) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     }
-    ok = ok && cudaMalloc((void**)&c->d_error, sizeof(int)) == cudaSuccess;
-    ok = ok && cudaMemset(c->d_error, 0, sizeof(int)) == cudaSuccess;
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_ids, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc((void**)&c->d_count, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_count, 2 * sizeof(int32_t)) == cudaSuccess;   // {count, error flag}
+    ok = ok && cudaMemset(c->d_count, 0, 2 * sizeof(int32_t)) == cudaSuccess;
+    if (ok) c->d_error = c->d_count + 1;
     ok = ok && cudaMallocHost((void**)&c->h_count, 2 * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -319,12 +403,16 @@ void comet_destroy(comet_ctx* c) {
     for (int id = 0; id < COMET_NUM_TENSORS; ++id)
         for (int p = 0; p < 2; ++p)
             if (c->buf[p][id]) cudaFree(c->buf[p][id]);
+    if (c->side) cudaStreamSynchronize(c->side);
     for (int p = 0; p < 2; ++p)
         for (int w = 0; w < 2; ++w) {
             if (c->planes_left[p][w]) cudaFree(c->planes_left[p][w]);
-            if (c->planes_right[p][w]) cudaFree(c->planes_right[p][w]);
+            if (c->planes_right_up[p][w]) cudaFree(c->planes_right_up[p][w]);
+            if (c->planes_right_dn[p][w]) cudaFree(c->planes_right_dn[p][w]);
         }
-    if (c->d_error) cudaFree(c->d_error);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
     if (c->d_mask) cudaFree(c->d_mask);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
@@ -356,6 +444,11 @@ int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* pt
     tensor_shape(c, tensor_id, rows, &er, &ec);
     if (rows != er || cols != ec) return COMET_ERR_SHAPE;
     if (rows * cols > c->cap_words[tensor_id]) return COMET_ERR_SHAPE;
+    if (tensor_id == COMET_W2 || tensor_id == COMET_B_DN) {
+        const int rc = join_side(c);       // the side stream may still be reading the old contents
+        if (rc != COMET_OK) return rc;
+        c->dn_right_ready = false;
+    }
     if (rows * cols > 0)
         COMET_CUDA(c, cudaMemcpyAsync(c->buf[party][tensor_id], ptr, (size_t)(rows * cols) * sizeof(u64),
                                       copy_kind(location, true), c->stream));
@@ -368,15 +461,24 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     if (!c || !block_mask || !n_active_out) return COMET_ERR_INVALID_ARG;
     if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
     if (n_blocks != c->cfg.d_ff / c->cfg.block) return COMET_ERR_SHAPE;
-    COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, block_mask, (size_t)n_blocks, copy_kind(location, true), c->stream));
+    {
+        const int rc = join_side(c);           // the side stream reads the index list
+        if (rc != COMET_OK) return rc;
+    }
+    c->dn_right_ready = false;
+    const uint8_t* dmask = block_mask;         // a device mask is read in place
+    if (location == COMET_HOST) {
+        COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, block_mask, (size_t)n_blocks, cudaMemcpyHostToDevice, c->stream));
+        dmask = c->d_mask;
+    }
     {
         PhaseTimer timer(c, COMET_PHASE_COMPACT, 1);
-        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_mask, n_blocks, c->d_ids, c->d_count);
+        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(dmask, n_blocks, c->d_ids, c->d_count);
     }
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
-    COMET_CUDA(c, cudaMemcpyAsync(c->h_count, c->d_count, sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
-    COMET_CUDA(c, cudaMemcpyAsync(c->h_count + 1, c->d_error, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    // one 8-byte copy: {count, error flag}
+    COMET_CUDA(c, cudaMemcpyAsync(c->h_count, c->d_count, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
     if (c->h_count[1] != 0) return COMET_ERR_TIMEOUT;     // an earlier kernel gave up on a bounded wait
     const int32_t blocks = *c->h_count;
@@ -414,6 +516,38 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
     c->up_tokens = tokens;
     c->up_done = true;
     if (n == 0) return COMET_OK;
+
+    if (c->path == COMET_PATH_LIMB) {
+        const Proj up = proj_up(c, tokens), dn = proj_down(c, tokens);
+        if (!limb_fits(c, up)) return COMET_ERR_SHAPE;
+        int rc = join_side(c);
+        if (rc != COMET_OK) return rc;
+        {
+            PhaseTimer timer(c, COMET_PHASE_OPEN, 1);
+            rc = limb_open(c, up, true, true, c->stream);
+        }
+        if (rc != COMET_OK) return rc;
+        {
+            PhaseTimer timer(c, COMET_PHASE_PREP, 1);
+            rc = limb_prep(c, up, true, true, true, c->stream);
+        }
+        if (rc != COMET_OK) return rc;
+        // The weight side of the down-projection depends only on the mask, W2 and B'_i: if those are loaded
+        // already, open it now on the side stream, under the tensor-core kernel that follows.
+        const bool early = !c->dn_right_ready && limb_fits(c, dn) && c->loaded[0][COMET_W2] &&
+                           c->loaded[1][COMET_W2] && c->loaded[0][COMET_B_DN] && c->loaded[1][COMET_B_DN];
+        if (early) {
+            COMET_CUDA(c, cudaEventRecord(c->ev_fork, c->stream));
+            COMET_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+            rc = limb_open(c, dn, false, true, c->side);
+            if (rc == COMET_OK) rc = limb_prep(c, dn, false, true, false, c->side);
+            if (rc != COMET_OK) return rc;
+            COMET_CUDA(c, cudaEventRecord(c->ev_join, c->side));
+            c->side_pending = true;
+            c->dn_right_ready = true;
+        }
+        return limb_combine(c, up);
+    }
 
     comet::PartyPtrs X, A, W0, W1, B;
     comet::PartyOut E, F;
@@ -461,6 +595,26 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
             COMET_CUDA(c, cudaMemsetAsync(c->buf[p][COMET_Y], 0, (size_t)tokens * d * sizeof(u64), c->stream));
         return COMET_OK;
     }
+    if (c->path == COMET_PATH_LIMB) {
+        const Proj dn = proj_down(c, tokens);
+        if (!limb_fits(c, dn)) return COMET_ERR_SHAPE;
+        const bool have_right = c->dn_right_ready;     // opened early, during the up-projection
+        int rc = join_side(c);
+        if (rc != COMET_OK) return rc;
+        {
+            PhaseTimer timer(c, COMET_PHASE_OPEN, 1);
+            rc = limb_open(c, dn, true, !have_right, c->stream);
+        }
+        if (rc != COMET_OK) return rc;
+        {
+            PhaseTimer timer(c, COMET_PHASE_PREP, 1);
+            rc = limb_prep(c, dn, true, !have_right, true, c->stream);
+        }
+        if (rc != COMET_OK) return rc;
+        c->dn_right_ready = false;                     // a triple serves one product
+        return limb_combine(c, dn);
+    }
+
     comet::PartyPtrs H, A, W, B;
     comet::PartyOut E, F;
     for (int p = 0; p < 2; ++p) {

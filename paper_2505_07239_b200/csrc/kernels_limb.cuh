@@ -33,9 +33,10 @@ constexpr int A_BLOCK_BYTES = PLANES * BM * KC;   // 32 KiB
 constexpr int B_BLOCK_BYTES = PLANES * BN * KC;   // 16 KiB
 constexpr int STAGES = 4;
 constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <= 3 below 2^32
-constexpr int THREADS = 192;                      // warps 0-3 epilogue, warp 4 copy producer, warp 5 MMA issuer
+constexpr int EPI_WARPS = 8;                      // warp w drains TMEM lanes 32*(w%4).., columns 32*(w/4)..
+constexpr int THREADS = 32 * (EPI_WARPS + 2);     // warps 0-7 epilogue, warp 8 copy producer, warp 9 MMA issuer
 constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
-constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + 1024;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + 128;
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s at 1.9 GHz: every wait gives up after this
 constexpr unsigned LBO_BYTES = 128, SBO_BYTES = 256;
 
@@ -46,23 +47,11 @@ __host__ __device__ __forceinline__ int block_offset(int rows, int p, int r, int
 }  // namespace limb
 
 // ---------------------------------------------------------------------------
-// Operand preparation after the exchange: blocked limb planes of
-//   S = in0 + in1              (the opened value E or F; identical for both parties, one copy each)
-//   W = in2 + (add_sum ? S : 0) (the party's own operand: V_i = A_i + i*E on the left, B_i on the right)
-// grid = (k-blocks, ceil(rows / 64), party); 256 threads; rows/k beyond the logical size are zero.
+// Blocked limb planes: helpers shared by the two memory-side kernels below.
+// A CTA tile is 64 rows x 32 contraction elements; words are staged in shared memory as [row][33] so that
+// the coalesced 16-byte global loads (16 threads per row) and the per-row 16-word reads of the byte
+// transposition are both conflict free.
 // ---------------------------------------------------------------------------
-struct PlanesArgs {
-    const u64* in0;          // message of party 0, [rows, K]
-    const u64* in1;          // message of party 1
-    const u64* in2[2];       // party's own share
-    uint8_t* out_sum[2];     // blocked planes of S, per party
-    uint8_t* out_own[2];     // blocked planes of W, per party
-    int add_sum[2];
-    int rows, K;             // logical sizes (K multiple of 16)
-    int kblocks;             // ceil(K / 32)
-    int tile_rows;           // 128 (left operand) or 64 (right operand)
-};
-
 __device__ __forceinline__ void limb_transpose4(unsigned x0, unsigned x1, unsigned x2, unsigned x3,
                                                 unsigned& p0, unsigned& p1, unsigned& p2, unsigned& p3) {
     const unsigned t0 = __byte_perm(x0, x1, 0x5140), t1 = __byte_perm(x2, x3, 0x5140);
@@ -73,19 +62,177 @@ __device__ __forceinline__ void limb_transpose4(unsigned x0, unsigned x1, unsign
     p3 = __byte_perm(t2, t3, 0x7632);
 }
 
-__global__ void __launch_bounds__(256)
-limb_planes_kernel(PlanesArgs a) {
-    using namespace limb;
-    __shared__ u64 sS[PREP_ROWS][KC + 1];
-    __shared__ u64 sW[PREP_ROWS][KC + 1];
-    const int party = blockIdx.z;
-    const int kb = blockIdx.x;
-    const int row0 = blockIdx.y * PREP_ROWS;
-    const int tid = threadIdx.x;
-    const u64* __restrict__ in2 = party ? a.in2[1] : a.in2[0];
-    const bool add = (party ? a.add_sum[1] : a.add_sum[0]) != 0;
+typedef u64 LimbTile[limb::PREP_ROWS][limb::KC + 1];
 
-    // phase 1: coalesced 16-byte loads, 16 threads per row
+// Split the 16 words src[r][16*half .. 16*half+15] into 8 limb planes of 16 bytes and store them at
+// (plane, row `rin`, k = 16*half) of the block `blk`, whose tiles have `tile_rows` rows.
+__device__ __forceinline__ void limb_emit_planes(const LimbTile& src, int r, int half, uint8_t* blk, int tile_rows,
+                                                 int rin) {
+    unsigned lo[16], hi[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const u64 v = src[r][half * 16 + j];
+        lo[j] = (unsigned)v;
+        hi[j] = (unsigned)(v >> 32);
+    }
+    uint4 plane[8];
+    limb_transpose4(lo[0], lo[1], lo[2], lo[3], plane[0].x, plane[1].x, plane[2].x, plane[3].x);
+    limb_transpose4(lo[4], lo[5], lo[6], lo[7], plane[0].y, plane[1].y, plane[2].y, plane[3].y);
+    limb_transpose4(lo[8], lo[9], lo[10], lo[11], plane[0].z, plane[1].z, plane[2].z, plane[3].z);
+    limb_transpose4(lo[12], lo[13], lo[14], lo[15], plane[0].w, plane[1].w, plane[2].w, plane[3].w);
+    limb_transpose4(hi[0], hi[1], hi[2], hi[3], plane[4].x, plane[5].x, plane[6].x, plane[7].x);
+    limb_transpose4(hi[4], hi[5], hi[6], hi[7], plane[4].y, plane[5].y, plane[6].y, plane[7].y);
+    limb_transpose4(hi[8], hi[9], hi[10], hi[11], plane[4].z, plane[5].z, plane[6].z, plane[7].z);
+    limb_transpose4(hi[12], hi[13], hi[14], hi[15], plane[4].w, plane[5].w, plane[6].w, plane[7].w);
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
+        *reinterpret_cast<uint4*>(blk + limb::block_offset(tile_rows, p, rin, half * 16)) = plane[p];
+}
+
+__device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows, int row, int kblocks, int kb,
+                                                   int* rin) {
+    const int tile = row / tile_rows;
+    *rin = row - tile * tile_rows;
+    return base + ((size_t)tile * kblocks + kb) * (size_t)(limb::PLANES * tile_rows * limb::KC);
+}
+
+// ---------------------------------------------------------------------------
+// Before the exchange (Section 2.1 "Multiplication"; Protocol 2 line 5, Protocol 3 line 9), one launch:
+//   left  blocks: E_i = X_i - A_i, elementwise;
+//   right tiles : F_i = gather(W_i) - B_i written as the message, and the blocked limb planes of the party's
+//                 own B_i (it is in registers anyway, so it is not read a second time later).
+// gather: up   (down = 0): row c of the right operand is row neuron(c) of W (whole rows of `ldw` words);
+//         down (down = 1): contraction index c is column neuron(c) of W (strips of `bs` words in every row).
+// grid = (left_blocks + kblocks * ceil(rows / 64), party), 256 threads.
+// ---------------------------------------------------------------------------
+struct LimbOpenArgs {
+    const u64* X[2];
+    const u64* A[2];
+    u64* E[2];
+    long long left_pairs;
+    int left_blocks;
+    const u64* W0[2];        // weights of group 0 (gate when gated, else the only matrix)
+    const u64* W1[2];        // weights of group 1 (up-projection of a gated FFN)
+    const u64* B[2];
+    u64* F[2];
+    uint8_t* Bpl[2];
+    const int32_t* ids;      // ascending active block ids
+    int n, bs;               // active neurons, neurons per block
+    int rows, K;             // logical size of the right operand [rows, K]
+    int ldw;                 // words per row of W
+    int kblocks, down;
+};
+
+__global__ void __launch_bounds__(256)
+limb_open_kernel(LimbOpenArgs a) {
+    using namespace limb;
+    const int party = blockIdx.y;
+    const int tid = threadIdx.x;
+    if ((int)blockIdx.x < a.left_blocks) {
+        const ulonglong2* __restrict__ x = reinterpret_cast<const ulonglong2*>(party ? a.X[1] : a.X[0]);
+        const ulonglong2* __restrict__ m = reinterpret_cast<const ulonglong2*>(party ? a.A[1] : a.A[0]);
+        ulonglong2* __restrict__ e = reinterpret_cast<ulonglong2*>(party ? a.E[1] : a.E[0]);
+        const long long stride = (long long)a.left_blocks * 256;
+        for (long long t = (long long)blockIdx.x * 256 + tid; t < a.left_pairs; t += stride) {
+            const ulonglong2 xv = __ldg(x + t), av = __ldg(m + t);
+            e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
+        }
+        return;
+    }
+    __shared__ LimbTile sB;
+    const int tile_id = blockIdx.x - a.left_blocks;
+    const int kb = tile_id % a.kblocks;
+    const int row0 = (tile_id / a.kblocks) * PREP_ROWS;
+    const u64* __restrict__ Bi = party ? a.B[1] : a.B[0];
+    u64* __restrict__ Fi = party ? a.F[1] : a.F[0];
+    {
+        const int kk = (tid & 15) * 2;
+        const int k = kb * KC + kk;
+        // down: the strip of W that holds compact contraction indices k, k+1
+        const int kcol = a.down && k < a.K ? a.ids[k / a.bs] * a.bs + (k % a.bs) : 0;
+#pragma unroll
+        for (int it = 0; it < PREP_ROWS / 16; ++it) {
+            const int r = it * 16 + (tid >> 4);
+            const int row = row0 + r;
+            u64 b0 = 0, b1 = 0;
+            if (row < a.rows && k < a.K) {
+                const u64* wsrc;
+                if (a.down) {
+                    wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
+                } else {
+                    const int grp = row / a.n, j = row - grp * a.n;
+                    const int neuron = a.ids[j / a.bs] * a.bs + (j % a.bs);
+                    wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0]) : (party ? a.W1[1] : a.W1[0])) +
+                           (size_t)neuron * a.ldw + k;
+                }
+                const size_t o = (size_t)row * a.K + k;
+                const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2*>(wsrc));
+                const ulonglong2 b = __ldg(reinterpret_cast<const ulonglong2*>(Bi + o));
+                *reinterpret_cast<ulonglong2*>(Fi + o) = make_ulonglong2(w.x - b.x, w.y - b.y);
+                b0 = b.x;
+                b1 = b.y;
+            }
+            sB[r][kk] = b0;
+            sB[r][kk + 1] = b1;
+        }
+    }
+    __syncthreads();
+    if (tid < 128) {
+        const int half = tid >> 6, r = tid & 63;
+        int rin;
+        uint8_t* blk = limb_block_ptr(party ? a.Bpl[1] : a.Bpl[0], BN, row0 + r, a.kblocks, kb, &rin);
+        limb_emit_planes(sB, r, half, blk, BN, rin);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// After the exchange, one launch: everything the tensor-core kernel needs, per party.
+//   left tiles : E = E_0 + E_1 -> planes(E);  V_i = A_i + i*E -> planes(V_i)      [M, K], 128-row blocks
+//   right tiles: F = F_0 + F_1 -> planes(F)                                      [N, K],  64-row blocks
+//   copy blocks: Z_i <- C_i (the accumulation target starts from the triple's C share)
+// grid = (kblocks * (ceil(M/64) + ceil(N/64)) + copy_blocks, party), 256 threads.  Any part may be empty.
+// ---------------------------------------------------------------------------
+struct LimbPrepArgs {
+    const u64* E0; const u64* E1;
+    const u64* A[2];
+    uint8_t* Epl[2];
+    uint8_t* Vpl[2];
+    int M, left_tiles;       // left_tiles = kblocks * ceil(M / 64), or 0
+    const u64* F0; const u64* F1;
+    uint8_t* Fpl[2];
+    int N, right_tiles;      // right_tiles = kblocks * ceil(N / 64), or 0
+    int K, kblocks;
+    const u64* C[2];
+    u64* Z[2];
+    long long copy_pairs;
+    int copy_blocks;
+};
+
+__global__ void __launch_bounds__(256)
+limb_prep_kernel(LimbPrepArgs a) {
+    using namespace limb;
+    const int party = blockIdx.y;
+    const int tid = threadIdx.x;
+    int id = blockIdx.x;
+    if (id >= a.left_tiles + a.right_tiles) {
+        id -= a.left_tiles + a.right_tiles;
+        const ulonglong2* __restrict__ s = reinterpret_cast<const ulonglong2*>(party ? a.C[1] : a.C[0]);
+        ulonglong2* __restrict__ d = reinterpret_cast<ulonglong2*>(party ? a.Z[1] : a.Z[0]);
+        const long long stride = (long long)a.copy_blocks * 256;
+        for (long long t = (long long)id * 256 + tid; t < a.copy_pairs; t += stride) d[t] = __ldg(s + t);
+        return;
+    }
+    extern __shared__ __align__(16) uint8_t prep_smem[];     // one tile (right/copy only) or two (left present)
+    LimbTile& sS = *reinterpret_cast<LimbTile*>(prep_smem);
+    LimbTile& sW = *reinterpret_cast<LimbTile*>(prep_smem + sizeof(LimbTile));
+    const bool left = id < a.left_tiles;
+    if (!left) id -= a.left_tiles;
+    const int kb = id % a.kblocks;
+    const int row0 = (id / a.kblocks) * PREP_ROWS;
+    const int rows = left ? a.M : a.N;
+    const u64* __restrict__ in0 = left ? a.E0 : a.F0;
+    const u64* __restrict__ in1 = left ? a.E1 : a.F1;
+    const u64* __restrict__ own = party ? a.A[1] : a.A[0];
     {
         const int kk = (tid & 15) * 2;
         const int k = kb * KC + kk;
@@ -94,64 +241,36 @@ limb_planes_kernel(PlanesArgs a) {
             const int r = it * 16 + (tid >> 4);
             const int row = row0 + r;
             u64 s0 = 0, s1 = 0, w0 = 0, w1 = 0;
-            if (row < a.rows && k < a.K) {
+            if (row < rows && k < a.K) {
                 const size_t o = (size_t)row * a.K + k;
-                const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(a.in0 + o));
-                const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(a.in1 + o));
-                const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(in2 + o));
-                s0 = x.x + y.x;
+                const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(in0 + o));
+                const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(in1 + o));
+                s0 = x.x + y.x;                       // the exchange: both messages summed
                 s1 = x.y + y.y;
-                w0 = z.x + (add ? s0 : 0ull);
-                w1 = z.y + (add ? s1 : 0ull);
+                if (left) {
+                    const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(own + o));
+                    w0 = z.x + (party ? s0 : 0ull);   // V_i = A_i + i*E
+                    w1 = z.y + (party ? s1 : 0ull);
+                }
             }
             sS[r][kk] = s0;
             sS[r][kk + 1] = s1;
-            sW[r][kk] = w0;
-            sW[r][kk + 1] = w1;
+            if (left) {
+                sW[r][kk] = w0;
+                sW[r][kk + 1] = w1;
+            }
         }
     }
     __syncthreads();
-
-    // phase 2: one thread per (output, 16-k half, row): split 16 words into 8 limb planes of 16 bytes
-    {
-        const int which = tid >> 7;              // 0: S, 1: W
-        const int half = (tid >> 6) & 1;
-        const int r = tid & 63;
-        const u64(*src)[KC + 1] = which ? sW : sS;
-        unsigned lo[16], hi[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const u64 v = src[r][half * 16 + j];
-            lo[j] = (unsigned)v;
-            hi[j] = (unsigned)(v >> 32);
-        }
-        uint4 plane[8];
-        limb_transpose4(lo[0], lo[1], lo[2], lo[3], plane[0].x, plane[1].x, plane[2].x, plane[3].x);
-        limb_transpose4(lo[4], lo[5], lo[6], lo[7], plane[0].y, plane[1].y, plane[2].y, plane[3].y);
-        limb_transpose4(lo[8], lo[9], lo[10], lo[11], plane[0].z, plane[1].z, plane[2].z, plane[3].z);
-        limb_transpose4(lo[12], lo[13], lo[14], lo[15], plane[0].w, plane[1].w, plane[2].w, plane[3].w);
-        limb_transpose4(hi[0], hi[1], hi[2], hi[3], plane[4].x, plane[5].x, plane[6].x, plane[7].x);
-        limb_transpose4(hi[4], hi[5], hi[6], hi[7], plane[4].y, plane[5].y, plane[6].y, plane[7].y);
-        limb_transpose4(hi[8], hi[9], hi[10], hi[11], plane[4].z, plane[5].z, plane[6].z, plane[7].z);
-        limb_transpose4(hi[12], hi[13], hi[14], hi[15], plane[4].w, plane[5].w, plane[6].w, plane[7].w);
-
-        const int row = row0 + r;
-        const int tile = row / a.tile_rows, rin = row - tile * a.tile_rows;
-        uint8_t* base = which ? (party ? a.out_own[1] : a.out_own[0]) : (party ? a.out_sum[1] : a.out_sum[0]);
-        uint8_t* blk = base + ((size_t)tile * a.kblocks + kb) * (size_t)(PLANES * a.tile_rows * KC);
-#pragma unroll
-        for (int p = 0; p < 8; ++p)
-            *reinterpret_cast<uint4*>(blk + block_offset(a.tile_rows, p, rin, half * 16)) = plane[p];
-    }
-}
-
-// Z_i <- C_i (the accumulation target of the tensor-core kernel starts from the triple's C share)
-__global__ void __launch_bounds__(256)
-copy_pairs_kernel(const u64* s0, const u64* s1, u64* d0, u64* d1, int64_t pairs) {
-    const ulonglong2* __restrict__ s = reinterpret_cast<const ulonglong2*>(blockIdx.y ? s1 : s0);
-    ulonglong2* __restrict__ d = reinterpret_cast<ulonglong2*>(blockIdx.y ? d1 : d0);
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < pairs; t += stride) d[t] = __ldg(s + t);
+    const int which = tid >> 7;                       // 0: the summed message, 1: the party's own operand
+    if (which == 1 && !left) return;
+    const int half = (tid >> 6) & 1, r = tid & 63;
+    const int tile_rows = left ? BM : BN;
+    uint8_t* base = left ? (which ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]))
+                         : (party ? a.Fpl[1] : a.Fpl[0]);
+    int rin;
+    uint8_t* blk = limb_block_ptr(base, tile_rows, row0 + r, a.kblocks, kb, &rin);
+    limb_emit_planes(which ? sW : sS, r, half, blk, tile_rows, rin);
 }
 
 // ---------------------------------------------------------------------------
@@ -257,7 +376,7 @@ combine_limb_kernel(LimbArgs a) {
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     uint8_t* sA = smem;
     uint8_t* sB = smem + (size_t)STAGES * A_BLOCK_BYTES;
 
@@ -273,7 +392,7 @@ combine_limb_kernel(LimbArgs a) {
             ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), 1);
         }
         ptx::mbar_init(ptx::smem_u32(&accum_full_bar), 1);
-        ptx::mbar_init(ptx::smem_u32(&accum_empty_bar), 128);
+        ptx::mbar_init(ptx::smem_u32(&accum_empty_bar), 32 * EPI_WARPS);
         abort_flag = 0;
         ptx::fence_barrier_init();
     }
@@ -286,7 +405,7 @@ combine_limb_kernel(LimbArgs a) {
     ptx::fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
 
-    if (warp == 4) {
+    if (warp == EPI_WARPS) {
         // ---------------- producer: one bulk copy per operand block ----------------
         if (lane == 0) {
             int stage = 0;
@@ -327,7 +446,7 @@ combine_limb_kernel(LimbArgs a) {
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == EPI_WARPS + 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc0 = (2u << 4) | ((uint32_t)(BM >> 4) << 24);   // s32 accumulate, u8 x u8, K-major
@@ -373,7 +492,7 @@ combine_limb_kernel(LimbArgs a) {
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> red.add into Z ----------------
+        // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> release TMEM -> red.add into Z --------
         uint32_t acc_phase = 0;
         bool ok = true;
         long long u = u_begin;
@@ -391,28 +510,39 @@ combine_limb_kernel(LimbArgs a) {
             ok = __all_sync(0xffffffffu, ok);          // also reconverges the warp for the aligned TMEM loads
             if (!ok) break;
             ptx::fence_after_sync();
-            const int row = tm * BM + warp * 32 + lane;
-            u64* __restrict__ zrow = (party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N;
-            const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 8) {
+            const int quarter = warp & 3, chalf = warp >> 2;
+            const int row = tm * BM + quarter * 32 + lane;
+            const int col0 = tn * BN + chalf * 32;
+            const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + chalf * 32;
+            u64 z[32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint32_t d[PLANES][8];
 #pragma unroll
-                for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c0, d[s]);
+                for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c * 8, d[s]);
                 ptx::tmem_wait_ld();
-                const int col = tn * BN + c0;
-                if (row < a.M && col < a.N) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        u64 z = (u64)d[0][j];
+                for (int j = 0; j < 8; ++j) {
+                    u64 v = (u64)d[0][j];
 #pragma unroll
-                        for (int s = 1; s < PLANES; ++s) z += (u64)d[s][j] << (8 * s);
-                        atomicAdd(zrow + col + j, z);
+                    for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
+                    z[c * 8 + j] = v;
+                }
+            }
+            // the accumulators are in registers: hand TMEM back before the (slow) global atomics
+            ptx::fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
+            if (row < a.M) {
+                u64* __restrict__ zrow = (party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int col = col0 + c * 8;
+                    if (col < a.N) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) atomicAdd(zrow + col + j, z[c * 8 + j]);
                     }
                 }
             }
-            ptx::fence_before_sync();
-            ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
             acc_phase ^= 1u;
         }
     }

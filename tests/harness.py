@@ -154,7 +154,7 @@ def sample_positions(rng, rows, cols, count):
 
 
 def run_and_compare_sampled(cfg, seed, sparsity=None, tokens=None, step=0, matmul_path=cb.PATH_AUTO,
-                            samples=512, ctx=None, weights=None):
+                            samples=512, ctx=None, weights=None, early_down=True):
     """Full-size check: messages E, F compared in full (they are cheap on the
     CPU), the products compared at sampled output positions computed one by
     one by the oracle from Eq. 1.  Up and down projections are exercised
@@ -180,6 +180,11 @@ def run_and_compare_sampled(cfg, seed, sparsity=None, tokens=None, step=0, matmu
 
     tri = wl.dealer_triple(seed, f"{cfg.name}/up/step{step}", T, d, g * n, valid=False)
     load_triple_up(ctx, tri)
+    trd = wl.dealer_triple(seed, f"{cfg.name}/down/step{step}", T, n, d, valid=False)
+    if early_down:
+        # the down-projection's triple is already there when ffn_up runs, so the library may open its
+        # weight side early (the full-chain tests load it late and cover the other order)
+        load_triple_down(ctx, trd)
     ctx.ffn_up(T)
     report["path"] = ctx.stats().matmul_path
     Zg = [ctx.get(party, cb.Z_UP, (T, g * n)) for party in (0, 1)]
@@ -200,8 +205,8 @@ def run_and_compare_sampled(cfg, seed, sparsity=None, tokens=None, step=0, matmu
     _, H0, H1 = wl.hidden_shares(cfg, seed, n, step=step, tokens=T)
     for party, Hs in ((0, H0), (1, H1)):
         ctx.load_shares(party, cb.H, cb.to_device(Hs))
-    trd = wl.dealer_triple(seed, f"{cfg.name}/down/step{step}", T, n, d, valid=False)
-    load_triple_down(ctx, trd)
+    if not early_down:
+        load_triple_down(ctx, trd)
     ctx.ffn_down(T)
     Yg = [ctx.get(party, cb.Y, (T, d)) for party in (0, 1)]
     ctx.truncate(cb.Y)
