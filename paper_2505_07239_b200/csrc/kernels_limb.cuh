@@ -31,12 +31,13 @@ namespace limb {
 constexpr int BM = 128, BN = 64, KC = 32, PLANES = 8;
 constexpr int A_BLOCK_BYTES = PLANES * BM * KC;   // 32 KiB
 constexpr int B_BLOCK_BYTES = PLANES * BN * KC;   // 16 KiB
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;
 constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <= 3 below 2^32
 constexpr int EPI_WARPS = 8;                      // warp w drains TMEM lanes 32*(w%4).., columns 32*(w/4)..
 constexpr int THREADS = 32 * (EPI_WARPS + 2);     // warps 0-7 epilogue, warp 8 copy producer, warp 9 MMA issuer
 constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
-constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + 128;
+constexpr int OUT_ROW_BYTES = 32 * 8 + 16;        // one staged output row of 32 words, padded against bank conflicts
+constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + (size_t)EPI_WARPS * 32 * OUT_ROW_BYTES + 128;
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s at 1.9 GHz: every wait gives up after this
 constexpr unsigned LBO_BYTES = 128, SBO_BYTES = 256;
 
@@ -303,6 +304,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// shared -> global bulk reduction: 64-bit integer add of `bytes` (multiple of 16) contiguous bytes
+__device__ __forceinline__ void bulk_reduce_add_u64(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.u64 [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
 }
@@ -314,13 +324,23 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
+// D[tmem] (+)= A[smem desc] * B[smem desc], u8 x u8 -> s32.  The descriptors are passed as (low, high) words: only
+// the low word (the shared-memory address field) changes between instructions.
+#define COMET_MMA_I8(NAME, QUAL)                                                                                   \
+    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,            \
+                                         uint32_t b_hi, uint32_t idesc, uint32_t acc) {                           \
+        asm volatile(                                                                                              \
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"                                                           \
+            "setp.ne.b32 p, %6, 0;\n\t"                                                                            \
+            "mov.b64 da, {%1, %2};\n\t"                                                                            \
+            "mov.b64 db, {%3, %4};\n\t"                                                                            \
+            "tcgen05.mma.cta_group::1.kind::i8" QUAL " [%0], da, db, %5, p;\n\t}"                                  \
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc) : "memory");          \
+    }
+COMET_MMA_I8(mma_i8, "")                               // A operand fetched for this instruction only
+COMET_MMA_I8(mma_i8_keep_a, ".collector::a::fill")     // A operand kept in the collector for the next instruction
+COMET_MMA_I8(mma_i8_reuse_a, ".collector::a::lastuse") // A operand taken from the collector, then dropped
+#undef COMET_MMA_I8
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -337,16 +357,14 @@ struct LimbArgs {
     const uint8_t* Vpl[2];   // left planes of V_i = A_i + i*E
     const uint8_t* Bpl[2];   // right planes of B_i: [n-tile][k-block][16 KiB]
     const uint8_t* Fpl[2];   // right planes of F = F_0 + F_1
-    u64* Z[2];               // [M, N], pre-loaded with C_i; partial sums are added atomically
-    int M, N;
+    u64* Z[2];               // [M, N], pre-loaded with C_i; partial sums are added with bulk reductions
+    int M, N;                // N a multiple of 16
     int mt, nt, kb;          // tiles and k-blocks per operand pair; one tile runs over 2*kb blocks
     int* error_flag;         // set to 1 if a bounded wait ran out
 };
 
-// Bounded wait: false (and the CTA-wide abort flag raised) if the barrier did not flip in time or another
-// role already gave up.
-__device__ __forceinline__ bool limb_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+// Slow path of a bounded wait, kept out of line so that the polling loops of the three roles stay short.
+__device__ __noinline__ bool limb_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 128; ++i)
@@ -359,12 +377,44 @@ __device__ __forceinline__ bool limb_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-__device__ __forceinline__ uint64_t limb_smem_desc(uint32_t addr) {
-    // K-major, no swizzle: bits 0-13 address>>4, 16-29 leading byte offset>>4 (between the two 16-byte K
-    // halves), 32-45 stride byte offset>>4 (between 8-row groups), 46-47 descriptor version 1
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(limb::LBO_BYTES >> 4) << 16) |
-           ((uint64_t)(limb::SBO_BYTES >> 4) << 32) | (1ull << 46);
+// Bounded wait: false (and the CTA-wide abort flag raised) if the barrier did not flip in time or another
+// role already gave up.
+__device__ __forceinline__ bool limb_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    return limb_wait_slow(bar, parity, abort_flag);
 }
+
+// One contiguous piece of a CTA's share of the (party, tile, k-block) space: a run of k-blocks of one tile.
+struct LimbSegment {
+    int party, tm, tn;
+    int kpos;        // first k-block, in [0, 2*kb): blocks [0,kb) pair E with B_i, [kb,2kb) pair V_i with F
+    int count;       // k-blocks in this segment, <= MAX_SEGMENT_UNITS
+};
+
+__device__ __forceinline__ LimbSegment limb_segment(const LimbArgs& a, long long u, long long u_end) {
+    const long long tile_units = 2ll * a.kb;
+    const long long tile = u / tile_units;
+    long long seg_end = (tile + 1) * tile_units;
+    if (seg_end > u_end) seg_end = u_end;
+    if (seg_end > u + limb::MAX_SEGMENT_UNITS) seg_end = u + limb::MAX_SEGMENT_UNITS;
+    const int per_party = a.mt * a.nt;
+    LimbSegment s;
+    s.party = (int)(tile / per_party);
+    const int t2 = (int)(tile - (long long)s.party * per_party);
+    s.tm = t2 / a.nt;
+    s.tn = t2 - s.tm * a.nt;
+    s.kpos = (int)(u - tile * tile_units);
+    s.count = (int)(seg_end - u);
+    return s;
+}
+
+// Low / high word of a shared-memory matrix descriptor, K-major, no swizzle: bits 0-13 address>>4, 16-29 leading
+// byte offset>>4 (between the two 16-byte K halves), 32-45 stride byte offset>>4 (between 8-row groups), 46-47
+// descriptor version 1.
+__device__ __forceinline__ uint32_t limb_desc_lo(uint32_t addr) {
+    return ((addr & 0x3FFFFu) >> 4) | ((uint32_t)(limb::LBO_BYTES >> 4) << 16);
+}
+constexpr uint32_t LIMB_DESC_HI = (uint32_t)(limb::SBO_BYTES >> 4) | (1u << 14);
 
 __global__ void __launch_bounds__(limb::THREADS, 1)
 combine_limb_kernel(LimbArgs a) {
@@ -379,10 +429,10 @@ combine_limb_kernel(LimbArgs a) {
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     uint8_t* sA = smem;
     uint8_t* sB = smem + (size_t)STAGES * A_BLOCK_BYTES;
+    uint8_t* sOut = sB + (size_t)STAGES * B_BLOCK_BYTES;      // EPI_WARPS x 32 rows x OUT_ROW_BYTES
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long tile_units = 2ll * a.kb;
-    const long long total_units = 2ll * a.mt * a.nt * tile_units;
+    const long long total_units = 2ll * a.mt * a.nt * 2ll * a.kb;
     const long long u_begin = total_units * blockIdx.x / gridDim.x;
     const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
 
@@ -412,27 +462,37 @@ combine_limb_kernel(LimbArgs a) {
             uint32_t phase = 0;
             int issued = 0;
             bool ok = true;
-            for (long long u = u_begin; u < u_end && ok; ++u) {
-                ok = limb_wait(ptx::smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag);
-                if (!ok) break;
-                const long long tile = u / tile_units;
-                int kpos = (int)(u - tile * tile_units);
-                const int per_party = a.mt * a.nt;
-                const int party = (int)(tile / per_party);
-                const int t2 = (int)(tile - (long long)party * per_party);
-                const int tm = t2 / a.nt, tn = t2 - tm * a.nt;
-                const bool second = kpos >= a.kb;
+            const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
+            const uint32_t sA0 = ptx::smem_u32(sA), sB0 = ptx::smem_u32(sB);
+            for (long long u = u_begin; u < u_end && ok;) {
+                const LimbSegment sg = limb_segment(a, u, u_end);
+                u += sg.count;
+                int kpos = sg.kpos;
+                bool second = kpos >= a.kb;
                 if (second) kpos -= a.kb;
-                const uint8_t* left = second ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]);
-                const uint8_t* right = second ? (party ? a.Fpl[1] : a.Fpl[0]) : (party ? a.Bpl[1] : a.Bpl[0]);
-                const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
-                ptx::mbar_expect_tx(bar, A_BLOCK_BYTES + B_BLOCK_BYTES);
-                ptx::bulk_g2s(ptx::smem_u32(sA + (size_t)stage * A_BLOCK_BYTES),
-                              left + ((size_t)tm * a.kb + kpos) * A_BLOCK_BYTES, A_BLOCK_BYTES, bar);
-                ptx::bulk_g2s(ptx::smem_u32(sB + (size_t)stage * B_BLOCK_BYTES),
-                              right + ((size_t)tn * a.kb + kpos) * B_BLOCK_BYTES, B_BLOCK_BYTES, bar);
-                ++issued;
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                const uint8_t* left = (second ? (sg.party ? a.Vpl[1] : a.Vpl[0]) : (sg.party ? a.Epl[1] : a.Epl[0])) +
+                                      ((size_t)sg.tm * a.kb + kpos) * A_BLOCK_BYTES;
+                const uint8_t* right = (second ? (sg.party ? a.Fpl[1] : a.Fpl[0]) : (sg.party ? a.Bpl[1] : a.Bpl[0])) +
+                                       ((size_t)sg.tn * a.kb + kpos) * B_BLOCK_BYTES;
+                for (int it = 0; it < sg.count; ++it) {
+                    ok = limb_wait(empty0 + 8 * stage, phase ^ 1u, &abort_flag);
+                    if (!ok) break;
+                    const uint32_t bar = full0 + 8 * stage;
+                    ptx::mbar_expect_tx(bar, A_BLOCK_BYTES + B_BLOCK_BYTES);
+                    ptx::bulk_g2s(sA0 + stage * A_BLOCK_BYTES, left, A_BLOCK_BYTES, bar);
+                    ptx::bulk_g2s(sB0 + stage * B_BLOCK_BYTES, right, B_BLOCK_BYTES, bar);
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    left += A_BLOCK_BYTES;
+                    right += B_BLOCK_BYTES;
+                    if (++kpos == a.kb && !second) {
+                        // the tile's first product (E with B_i) is done: go on with the second (V_i with F)
+                        second = true;
+                        kpos = 0;
+                        left = (sg.party ? a.Vpl[1] : a.Vpl[0]) + (size_t)sg.tm * a.kb * A_BLOCK_BYTES;
+                        right = (sg.party ? a.Fpl[1] : a.Fpl[0]) + (size_t)sg.tn * a.kb * B_BLOCK_BYTES;
+                    }
+                }
             }
             if (!ok) {
                 // gave up: let the copies already in flight land before the CTA leaves
@@ -447,104 +507,108 @@ combine_limb_kernel(LimbArgs a) {
             }
         }
     } else if (warp == EPI_WARPS + 1) {
-        // ---------------- MMA issuer ----------------
+        // ---------------- MMA issuer: 12 instructions per k-block, as little else as possible ----------------
         if (lane == 0) {
-            const uint32_t idesc0 = (2u << 4) | ((uint32_t)(BM >> 4) << 24);   // s32 accumulate, u8 x u8, K-major
+            // instruction descriptor: s32 accumulate, u8 x u8, both K-major, M = 128, N filled in per instruction
+            constexpr uint32_t IDESC = (2u << 4) | ((uint32_t)(BM >> 4) << 24);
+            const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
+            const uint32_t accum_full = ptx::smem_u32(&accum_full_bar), accum_empty = ptx::smem_u32(&accum_empty_bar);
+            const uint32_t a_lo0 = limb_desc_lo(ptx::smem_u32(sA)), b_lo0 = limb_desc_lo(ptx::smem_u32(sB));
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            long long u = u_begin;
-            while (u < u_end && ok) {
-                const long long tile = u / tile_units;
-                long long seg_end = (tile + 1) * tile_units;
-                if (seg_end > u_end) seg_end = u_end;
-                if (seg_end > u + MAX_SEGMENT_UNITS) seg_end = u + MAX_SEGMENT_UNITS;
-                ok = limb_wait(ptx::smem_u32(&accum_empty_bar), acc_phase ^ 1u, &abort_flag);
+            for (long long u = u_begin; u < u_end && ok;) {
+                const LimbSegment sg = limb_segment(a, u, u_end);
+                u += sg.count;
+                ok = limb_wait(accum_empty, acc_phase ^ 1u, &abort_flag);
                 if (!ok) break;
                 ptx::fence_after_sync();
-                bool first = true;
-                for (; u < seg_end; ++u) {
-                    ok = limb_wait(ptx::smem_u32(&full_bar[stage]), phase, &abort_flag);
+                uint32_t acc = 0;                         // the segment's first block overwrites the accumulators
+                for (int it = 0; it < sg.count; ++it) {
+                    ok = limb_wait(full0 + 8 * stage, phase, &abort_flag);
                     if (!ok) break;
                     ptx::fence_after_sync();
-                    const uint32_t a_addr = ptx::smem_u32(sA + (size_t)stage * A_BLOCK_BYTES);
-                    const uint32_t b_addr = ptx::smem_u32(sB + (size_t)stage * B_BLOCK_BYTES);
-                    const uint64_t bdesc0 = limb_smem_desc(b_addr);
-                    const uint64_t bdesc1 = limb_smem_desc(b_addr + 256 * KC);   // right-operand rows 256.. (planes 4..)
+                    const uint32_t a_lo = a_lo0 + stage * (A_BLOCK_BYTES >> 4);
+                    const uint32_t b_lo = b_lo0 + stage * (B_BLOCK_BYTES >> 4);
+                    const uint32_t b_lo_hi = b_lo + ((256 * KC) >> 4);         // right-operand rows 256.. (planes 4..7)
+                    // Left plane p meets right planes 0..7-p, whose products land in accumulators D_p..D_7: one
+                    // instruction of N = 64*(8-p), cut at 256.  When a plane issues two instructions the second
+                    // takes the left operand from the collector instead of shared memory.
 #pragma unroll
                     for (int p = 0; p < PLANES; ++p) {
-                        const uint64_t adesc = limb_smem_desc(a_addr + p * BM * KC);
+                        const uint32_t ap = a_lo + ((p * BM * KC) >> 4);
                         const int n_total = BN * (PLANES - p);
-                        const int n0 = n_total > 256 ? 256 : n_total;
-                        const uint32_t acc = (first && p == 0) ? 0u : 1u;
-                        ptx::mma_i8(tmem_base + BN * p, adesc, bdesc0, idesc0 | ((uint32_t)(n0 >> 3) << 17), acc);
-                        if (n_total > 256)
-                            ptx::mma_i8(tmem_base + BN * p + 256, adesc, bdesc1,
-                                        idesc0 | ((uint32_t)((n_total - 256) >> 3) << 17), acc);
+                        const uint32_t acc_p = p == 0 ? acc : 1u;
+                        if (n_total > 256) {
+                            ptx::mma_i8_keep_a(tmem_base + BN * p, ap, LIMB_DESC_HI, b_lo, LIMB_DESC_HI,
+                                               IDESC | ((uint32_t)(256 >> 3) << 17), acc_p);
+                            ptx::mma_i8_reuse_a(tmem_base + BN * p + 256, ap, LIMB_DESC_HI, b_lo_hi, LIMB_DESC_HI,
+                                                IDESC | ((uint32_t)((n_total - 256) >> 3) << 17), acc_p);
+                        } else {
+                            ptx::mma_i8(tmem_base + BN * p, ap, LIMB_DESC_HI, b_lo, LIMB_DESC_HI,
+                                        IDESC | ((uint32_t)(n_total >> 3) << 17), acc_p);
+                        }
                     }
-                    ptx::mma_commit(ptx::smem_u32(&empty_bar[stage]));    // frees the stage once the MMAs have read it
-                    first = false;
+                    ptx::mma_commit(empty0 + 8 * stage);    // frees the stage once the MMAs have read it
+                    acc = 1u;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                ptx::mma_commit(ptx::smem_u32(&accum_full_bar));
+                ptx::mma_commit(accum_full);
                 acc_phase ^= 1u;
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> release TMEM -> red.add into Z --------
+        // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> release TMEM ->
+        //                  stage the rows in shared memory -> one bulk add-reduction per row into Z ----------------
         uint32_t acc_phase = 0;
         bool ok = true;
-        long long u = u_begin;
-        while (u < u_end && ok) {
-            const long long tile = u / tile_units;
-            long long seg_end = (tile + 1) * tile_units;
-            if (seg_end > u_end) seg_end = u_end;
-            if (seg_end > u + MAX_SEGMENT_UNITS) seg_end = u + MAX_SEGMENT_UNITS;
-            u = seg_end;
-            const int per_party = a.mt * a.nt;
-            const int party = (int)(tile / per_party);
-            const int t2 = (int)(tile - (long long)party * per_party);
-            const int tm = t2 / a.nt, tn = t2 - tm * a.nt;
+        const int quarter = warp & 3, chalf = warp >> 2;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + chalf * 32;
+        uint8_t* my_row = sOut + ((size_t)warp * 32 + lane) * OUT_ROW_BYTES;
+        const uint32_t my_row_s = ptx::smem_u32(my_row);
+        for (long long u = u_begin; u < u_end && ok;) {
+            const LimbSegment sg = limb_segment(a, u, u_end);
+            u += sg.count;
             ok = limb_wait(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);          // also reconverges the warp for the aligned TMEM loads
             if (!ok) break;
             ptx::fence_after_sync();
-            const int quarter = warp & 3, chalf = warp >> 2;
-            const int row = tm * BM + quarter * 32 + lane;
-            const int col0 = tn * BN + chalf * 32;
-            const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + chalf * 32;
-            u64 z[32];
+            ptx::bulk_wait_group_read0();              // the previous segment's reductions have read this row
+            const int row = sg.tm * BM + quarter * 32 + lane;
+            const int col0 = sg.tn * BN + chalf * 32;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t d[PLANES][8];
 #pragma unroll
                 for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c * 8, d[s]);
                 ptx::tmem_wait_ld();
+                u64 z[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     u64 v = (u64)d[0][j];
 #pragma unroll
                     for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
-                    z[c * 8 + j] = v;
+                    z[j] = v;
                 }
+#pragma unroll
+                for (int j = 0; j < 8; j += 2)
+                    *reinterpret_cast<ulonglong2*>(my_row + (c * 8 + j) * 8) = make_ulonglong2(z[j], z[j + 1]);
             }
-            // the accumulators are in registers: hand TMEM back before the (slow) global atomics
+            // the accumulators have left TMEM: hand it back before the reduction traffic starts
             ptx::fence_before_sync();
             ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
-            if (row < a.M) {
-                u64* __restrict__ zrow = (party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int col = col0 + c * 8;
-                    if (col < a.N) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) atomicAdd(zrow + col + j, z[c * 8 + j]);
-                    }
-                }
+            int cols = a.N - col0;
+            if (cols > 32) cols = 32;
+            if (row < a.M && cols > 0) {
+                ptx::fence_proxy_async_smem();         // this thread's row, written above, is read by the copy engine
+                ptx::bulk_reduce_add_u64((sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0, my_row_s,
+                                         (uint32_t)cols * 8u);
             }
+            ptx::bulk_commit_group();
             acc_phase ^= 1u;
         }
+        ptx::bulk_wait_group0();                       // every reduction of this thread has completed
     }
 
     ptx::fence_before_sync();
