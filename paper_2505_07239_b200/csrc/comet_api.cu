@@ -41,8 +41,9 @@ struct comet_ctx {
     bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
     uint8_t* d_mask;
     int32_t* d_ids;
-    int32_t* d_count;
-    int32_t* h_count;             // pinned
+    int32_t* d_count;             // {count, error flag of the bounded waits}
+    int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
+    int32_t* h_count_dev;         // device-side address of h_count
     bool mask_set;
     int32_t n_active, n_active_blocks;
     int32_t tokens;               // T fixed by the last load of X / A_UP / H
@@ -376,6 +377,14 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
             }
         ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)lb::SMEM_BYTES) == cudaSuccess;
+        // the memory-side kernels may share an SM with a resident tensor-core CTA (which forces the largest
+        // shared-memory carve-out), so they ask for the same carve-out
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::limb_open_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::limb_prep_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
@@ -386,7 +395,8 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     ok = ok && cudaMalloc((void**)&c->d_count, 2 * sizeof(int32_t)) == cudaSuccess;   // {count, error flag}
     ok = ok && cudaMemset(c->d_count, 0, 2 * sizeof(int32_t)) == cudaSuccess;
     if (ok) c->d_error = c->d_count + 1;
-    ok = ok && cudaMallocHost((void**)&c->h_count, 2 * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_count, 2 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer((void**)&c->h_count_dev, c->h_count, 0) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         comet_destroy(c);
@@ -473,12 +483,11 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     }
     {
         PhaseTimer timer(c, COMET_PHASE_COMPACT, 1);
-        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(dmask, n_blocks, c->d_ids, c->d_count);
+        // the kernel reports {count, error flag} straight into mapped host memory: no copy to enqueue
+        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(dmask, n_blocks, c->d_ids, c->d_count, c->h_count_dev);
     }
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
-    // one 8-byte copy: {count, error flag}
-    COMET_CUDA(c, cudaMemcpyAsync(c->h_count, c->d_count, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
     if (c->h_count[1] != 0) return COMET_ERR_TIMEOUT;     // an earlier kernel gave up on a bounded wait
     const int32_t blocks = *c->h_count;

@@ -36,7 +36,8 @@ constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <
 constexpr int EPI_WARPS = 8;                      // warp w drains TMEM lanes 32*(w%4).., columns 32*(w/4)..
 constexpr int THREADS = 32 * (EPI_WARPS + 2);     // warps 0-7 epilogue, warp 8 copy producer, warp 9 MMA issuer
 constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
-constexpr int OUT_ROW_BYTES = 32 * 8 + 16;        // one staged output row of 32 words, padded against bank conflicts
+constexpr int OUT_COLS = 16;                      // words per staged output row (a thread's 32 go in two rounds)
+constexpr int OUT_ROW_BYTES = OUT_COLS * 8 + 16;  // padded against bank conflicts
 constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + (size_t)EPI_WARPS * 32 * OUT_ROW_BYTES + 128;
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s at 1.9 GHz: every wait gives up after this
 constexpr unsigned LBO_BYTES = 128, SBO_BYTES = 256;
@@ -574,38 +575,42 @@ combine_limb_kernel(LimbArgs a) {
             ok = __all_sync(0xffffffffu, ok);          // also reconverges the warp for the aligned TMEM loads
             if (!ok) break;
             ptx::fence_after_sync();
-            ptx::bulk_wait_group_read0();              // the previous segment's reductions have read this row
             const int row = sg.tm * BM + quarter * 32 + lane;
             const int col0 = sg.tn * BN + chalf * 32;
+            u64 z[32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t d[PLANES][8];
 #pragma unroll
                 for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c * 8, d[s]);
                 ptx::tmem_wait_ld();
-                u64 z[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     u64 v = (u64)d[0][j];
 #pragma unroll
                     for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
-                    z[j] = v;
+                    z[c * 8 + j] = v;
                 }
-#pragma unroll
-                for (int j = 0; j < 8; j += 2)
-                    *reinterpret_cast<ulonglong2*>(my_row + (c * 8 + j) * 8) = make_ulonglong2(z[j], z[j + 1]);
             }
-            // the accumulators have left TMEM: hand it back before the reduction traffic starts
+            // the accumulators are in registers: hand TMEM back before the reduction traffic starts
             ptx::fence_before_sync();
             ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
-            int cols = a.N - col0;
-            if (cols > 32) cols = 32;
-            if (row < a.M && cols > 0) {
-                ptx::fence_proxy_async_smem();         // this thread's row, written above, is read by the copy engine
-                ptx::bulk_reduce_add_u64((sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0, my_row_s,
-                                         (uint32_t)cols * 8u);
+            u64* zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0;
+#pragma unroll
+            for (int h = 0; h < 32 / OUT_COLS; ++h) {
+                ptx::bulk_wait_group_read0();          // the previous reduction has read this thread's staging row
+#pragma unroll
+                for (int j = 0; j < OUT_COLS; j += 2)
+                    *reinterpret_cast<ulonglong2*>(my_row + j * 8) =
+                        make_ulonglong2(z[h * OUT_COLS + j], z[h * OUT_COLS + j + 1]);
+                int cols = a.N - col0 - h * OUT_COLS;
+                if (cols > OUT_COLS) cols = OUT_COLS;
+                if (row < a.M && cols > 0) {
+                    ptx::fence_proxy_async_smem();     // this thread's row, written above, is read by the copy engine
+                    ptx::bulk_reduce_add_u64(zrow + h * OUT_COLS, my_row_s, (uint32_t)cols * 8u);
+                }
+                ptx::bulk_commit_group();
             }
-            ptx::bulk_commit_group();
             acc_phase ^= 1u;
         }
         ptx::bulk_wait_group0();                       // every reduction of this thread has completed

@@ -22,9 +22,12 @@ struct PartyOut {
 // One CTA of 1024 threads walks the mask 1024 blocks at a time: a warp ballot
 // ranks each active block inside its warp, a shuffle scan over the 32 warp
 // totals gives each warp's base, and a running base carries across chunks.
+// `count` points at two words {count, error flag}; both are also written to
+// `host_report` (mapped host memory) so that the host needs no copy.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
-compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids, int32_t* __restrict__ count) {
+compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids, int32_t* __restrict__ count,
+                    int32_t* __restrict__ host_report) {
     __shared__ int warp_excl[32];
     __shared__ int chunk_total;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -52,7 +55,13 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
         running += chunk_total;
         __syncthreads();                   // warp_excl / chunk_total are rewritten next round
     }
-    if (threadIdx.x == 0) *count = running;
+    if (threadIdx.x == 0) {
+        *count = running;
+        // {count, error flag raised by an earlier kernel's bounded wait} for the host, in mapped pinned memory
+        host_report[0] = running;
+        host_report[1] = count[1];
+        __threadfence_system();
+    }
 }
 
 // ---------------------------------------------------------------------------
