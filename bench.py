@@ -32,6 +32,30 @@ METRIC = "sparse shared-FFN Z_2^64 MACs/s"
 UNIT = "MAC64/s"
 L2_FLUSH_BYTES = 512 << 20
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the tensor-core combine kernel on the
+# default workload, from the ncu capture summarised in profiles/combine_limb__opt1.3b_s90.md (average of the
+# up- and the down-projection launch).  Valid only for the kernel source it was taken on: keyed by its SHA-256.
+COMBINE_LIMB_TRAFFIC = {
+    "workload": ("opt1.3b", 0.9),
+    "kernel_sha256": "bde0e5c18ff3d9f03566223900c7a4b121d6c7b98a99ee579388baee226720f5",
+    "bytes_per_launch": 116595456,
+}
+
+
+def combine_traffic(workload, sparsity, used_path):
+    """The stored ncu DRAM traffic of the dominant kernel, or None when it does not apply any more."""
+    import hashlib
+
+    if used_path != "limb" or (workload, round(sparsity, 4)) != COMBINE_LIMB_TRAFFIC["workload"]:
+        return None
+    src = os.path.join(ROOT, "paper_2505_07239_b200", "csrc", "kernels_limb.cuh")
+    try:
+        with open(src, "rb") as fh:
+            digest = hashlib.sha256(fh.read()).hexdigest()
+    except OSError:
+        return None
+    return COMBINE_LIMB_TRAFFIC["bytes_per_launch"] if digest == COMBINE_LIMB_TRAFFIC["kernel_sha256"] else None
+
 
 def ffn_macs(cfg, T, n):
     """Algorithmic ring MACs of one step, both parties: 2*T*K*N per party per product."""
@@ -381,7 +405,11 @@ def main():
                     "peak_source": "148 SM x 64 int32 mul-add lanes/clk x 1.965 GHz / 4 issue slots per 64-bit MAC"}
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["kernel"] = "combine_" + used_path
-        roof["traffic"] = None
+        roof["traffic"] = combine_traffic(args.workload, sparsity, used_path)
+        roof["traffic_unit"] = "bytes per launch (ncu dram read+write); algorithmic: planes once + Z read-modify-write"
+        # per party: planes of both operand pairs read once, Z read and written once; averaged over the two launches
+        roof["algorithmic_bytes_per_launch"] = 8 * ((2 * T * d + 2 * d * g * n + 2 * T * g * n) +
+                                                    (2 * T * n + 2 * n * d + 2 * T * d))
         t_roof = max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (roof["peak"] * 1e12))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -10,12 +10,13 @@ from __future__ import annotations
 
 import ctypes
 import os
+import subprocess
 from typing import Optional
 
 import numpy as np
 import torch
 
-from .build import LIB_PATH
+from .build import LIB_PATH, build_library, is_current
 
 OK = 0
 DEVICE, HOST = 0, 1
@@ -55,10 +56,14 @@ class CometError(RuntimeError):
 
 
 def _load():
-    if not os.path.exists(LIB_PATH):
-        raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2505_07239_b200.build` "
-            "(there is no CPU fallback)")
+    if not is_current():
+        # missing, or built from other sources than the ones in the tree: rebuild rather than run stale kernels
+        try:
+            build_library()
+        except (OSError, subprocess.CalledProcessError) as exc:
+            raise ImportError(
+                f"{LIB_PATH} is missing or stale and could not be rebuilt ({exc}); build it with "
+                "`python -m paper_2505_07239_b200.build` (there is no CPU fallback)") from exc
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     lib.comet_init.argtypes = [ctypes.POINTER(CometConfig), vp, ctypes.POINTER(vp)]
