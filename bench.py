@@ -26,6 +26,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2505_07239_b200 import ranks  # noqa: E402
 from paper_2505_07239_b200 import workloads as wl  # noqa: E402
 
 METRIC = "sparse shared-FFN Z_2^64 MACs/s"
@@ -177,9 +178,9 @@ def time_oracle(cfg, seed, sparsity, budget_s=15.0):
 
 
 def run_reference(args, cfg, sparsity):
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = ranks.rank_world_local()
     if rank != 0:
-        return
+        return          # under a multi-process launch rank 0 alone times the oracle; the others leave with status 0
     steps = max(1, args.steps)
     per = max(2.0, min(30.0, 120.0 / (steps + args.warmup)))
     vals = []
@@ -234,16 +235,14 @@ def main():
 
     from paper_2505_07239_b200 import binding as cb
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = ranks.rank_world_local()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
     T, d, g = cfg.tokens, cfg.d_model, cfg.groups
-    seed = 1000 + rank          # every rank runs its own independent FFN problem (weak scaling, no collective)
+    seed = ranks.rank_seed(1000, rank)   # every rank runs its own independent FFN problems (weak scaling, no collective)
     path = {"auto": cb.PATH_AUTO, "simt": cb.PATH_SIMT, "limb": cb.PATH_LIMB}[args.path]
     stream = torch.cuda.Stream(device=dev)
     n_cap = cfg.n_active_blocks(sparsity) * cfg.block
@@ -371,14 +370,11 @@ def main():
     h2d = sum(t.numel() * 8 for p in (0, 1) for t in sets[0]["pinned"][p].values()) + sets[0]["mask_host"].numel()
     d2h = 2 * T * d * 8 + 4
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = t.tolist()
+    total_ms, e2e_ms = ranks.max_over_ranks([total_ms, e2e_ms], dev)
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
-        value = world * macs / (ms_per_step * 1e-3)
+        value = ranks.whole_job_throughput(macs, world, args.steps, total_ms)
         phase = {name: {"ms_per_step": stats.phase_ms[k] / prof_steps, "launches_per_step":
                         stats.phase_launches[k] / prof_steps} for k, name in enumerate(cb.PHASE_NAMES)}
         comb_launch_ms = stats.phase_ms[3] / max(1, stats.phase_launches[3])
@@ -421,7 +417,7 @@ def main():
                        "parallelism": f"independent FFN per GPU x{world}"},
             "gpu_launches": int(launches),
             "clocks": clocks,
-            "e2e": {"value": world * macs / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+            "e2e": {"value": ranks.whole_job_throughput(macs, world, args.steps, e2e_ms), "unit": UNIT,
                     "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "roofline": roof,
             "path_roofline": {"algorithmic_bytes": ffn_bytes(cfg, T, n), "algorithmic_macs": macs,
