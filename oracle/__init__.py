@@ -178,3 +178,68 @@ def truncate(party: int, Z, frac_bits: int):
     out = np.empty_like(Z)
     lib().orc_truncate(ctypes.c_int(party), _p(Z), _p(out), ctypes.c_size_t(Z.size), ctypes.c_int(frac_bits))
     return out
+
+
+# ---------------------------------------------------------------------------
+# Oblivious shuffle (Protocol 1).  Permutations are int32 index arrays acting on
+# the rows of [rows, cols] uint64 matrices: (pi(x))[j] = x[pi[j]].
+# ---------------------------------------------------------------------------
+def _perm(p) -> np.ndarray:
+    p = np.ascontiguousarray(p, dtype=np.int32)
+    assert p.ndim == 1
+    return p
+
+
+def _rows2d(x) -> np.ndarray:
+    x = _u64(x)
+    return x.reshape(x.shape[0], -1)
+
+
+def apply_permutation(perm, x):
+    perm, x2 = _perm(perm), _rows2d(x)
+    out = np.empty_like(x2)
+    lib().orc_apply_permutation(_p(perm), _p(x2), _p(out), ctypes.c_int(x2.shape[0]), ctypes.c_int(x2.shape[1]))
+    return out.reshape(np.shape(x))
+
+
+def compose_permutations(p, q):
+    """p o q as operators: (p o q)(x) = p(q(x))."""
+    p, q = _perm(p), _perm(q)
+    out = np.empty_like(p)
+    lib().orc_compose_permutations(_p(p), _p(q), _p(out), ctypes.c_int(p.size))
+    return out
+
+
+def invert_permutation(p):
+    p = _perm(p)
+    out = np.empty_like(p)
+    lib().orc_invert_permutation(_p(p), _p(out), ctypes.c_int(p.size))
+    return out
+
+
+def shuffle_offline(pi, tau, a, c):
+    """Offline stage: tau = (tau_0, tau_1), a = (a_0, a_1), c the dealer's random
+    matrix.  Returns rho = (rho_0, rho_1), b = (b_0, b_1)."""
+    pi, t0, t1 = _perm(pi), _perm(tau[0]), _perm(tau[1])
+    a0, a1, c2 = _rows2d(a[0]), _rows2d(a[1]), _rows2d(c)
+    rows, cols = a0.shape
+    r0, r1 = np.empty_like(pi), np.empty_like(pi)
+    b0, b1 = np.empty_like(a0), np.empty_like(a0)
+    lib().orc_shuffle_offline(ctypes.c_int(rows), ctypes.c_int(cols), _p(pi), _p(t0), _p(t1), _p(a0), _p(a1), _p(c2),
+                              _p(r0), _p(r1), _p(b0), _p(b1))
+    shape = np.shape(a[0])
+    return (r0, r1), (b0.reshape(shape), b1.reshape(shape))
+
+
+def shuffle_online(x, tau, rho, a, b):
+    """Online stage for both parties.  Returns messages y = (y_0, y_1) and results z = (z_0, z_1)."""
+    x0, x1 = _rows2d(x[0]), _rows2d(x[1])
+    rows, cols = x0.shape
+    arrs = [_perm(tau[0]), _perm(tau[1]), _perm(rho[0]), _perm(rho[1]),
+            _rows2d(a[0]), _rows2d(a[1]), _rows2d(b[0]), _rows2d(b[1])]
+    outs = [np.empty_like(x0) for _ in range(4)]
+    lib().orc_shuffle_online(ctypes.c_int(rows), ctypes.c_int(cols), _p(x0), _p(x1), *[_p(v) for v in arrs],
+                             *[_p(o) for o in outs])
+    shape = np.shape(x[0])
+    y0, y1, z0, z1 = (o.reshape(shape) for o in outs)
+    return (y0, y1), (z0, z1)

@@ -17,6 +17,10 @@
 // closed forms and the {0,1}-ulp invariant; hand-computed fixtures.
 // Parity unpinned: the individual share values Z_i (as opposed to their sum)
 // are fixed only by Eq. 1 itself plus this repository's seeded inputs.
+// Oblivious shuffle (Protocol 1): pinned by the paper's worked permutation
+// example, by z_1 + z_2 = pi(x) against numpy indexing, by the operator
+// identities rho_1 o tau_2 = rho_2 o tau_1 = pi, by exhaustive permutations of
+// three elements and by unshuffle(shuffle(x)) = x.
 
 #include <cstddef>
 #include <cstdint>
@@ -217,6 +221,67 @@ void orc_truncate(int party, const u64* in, u64* out, size_t count, int f) {
     for (size_t t = 0; t < count; ++t) {
         if (party == 0) out[t] = in[t] >> f;
         else out[t] = (u64)0 - (((u64)0 - in[t]) >> f);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Section 4.2, "Oblivious shuffle".  A permutation pi acts on a vector as the
+// paper's example fixes it: pi = [2,1,3] gives pi(x) = [x_2, x_1, x_3], i.e.
+// (pi(x))_j = x_{pi_j} (indices 0-based here).  The shuffled objects are the
+// `rows` rows of a [rows, cols] matrix of ring words.
+// ---------------------------------------------------------------------------
+void orc_apply_permutation(const int32_t* perm, const u64* x, u64* out, int rows, int cols) {
+    for (int j = 0; j < rows; ++j)
+        for (int c = 0; c < cols; ++c) out[(size_t)j * cols + c] = x[(size_t)perm[j] * cols + c];
+}
+
+// p o q as an operator: (p o q)(x) = p(q(x)).  (p(q(x)))_j = (q(x))_{p_j} = x_{q_{p_j}}.
+void orc_compose_permutations(const int32_t* p, const int32_t* q, int32_t* out, int rows) {
+    for (int j = 0; j < rows; ++j) out[j] = q[p[j]];
+}
+
+void orc_invert_permutation(const int32_t* p, int32_t* out, int rows) {
+    for (int j = 0; j < rows; ++j) out[p[j]] = j;
+}
+
+// Protocol 1, offline stage (the trusted third party): given pi, tau_1, tau_2 and the
+// random a_1, a_2, c it derives rho_1 = pi o tau_2^{-1}, rho_2 = pi o tau_1^{-1},
+// b_1 = rho_1(a_2) + c and b_2 = rho_2(a_1) - c.  Party index 0/1 = the paper's 1/2.
+void orc_shuffle_offline(int rows, int cols, const int32_t* pi, const int32_t* tau0, const int32_t* tau1,
+                         const u64* a0, const u64* a1, const u64* c,
+                         int32_t* rho0, int32_t* rho1, u64* b0, u64* b1) {
+    std::vector<int32_t> inv(rows);
+    orc_invert_permutation(tau1, inv.data(), rows);
+    orc_compose_permutations(pi, inv.data(), rho0, rows);
+    orc_invert_permutation(tau0, inv.data(), rows);
+    orc_compose_permutations(pi, inv.data(), rho1, rows);
+    const size_t count = (size_t)rows * cols;
+    orc_apply_permutation(rho0, a1, b0, rows, cols);
+    orc_apply_permutation(rho1, a0, b1, rows, cols);
+    for (size_t t = 0; t < count; ++t) {
+        b0[t] = b0[t] + c[t];
+        b1[t] = b1[t] - c[t];
+    }
+}
+
+// Protocol 1, online stage, both parties: [y]_i = tau_i([x]_i) + a_i is sent to the
+// other party, which computes [z]_i = rho_i([y]_{other}) - b_i.
+void orc_shuffle_online(int rows, int cols, const u64* x0, const u64* x1,
+                        const int32_t* tau0, const int32_t* tau1, const int32_t* rho0, const int32_t* rho1,
+                        const u64* a0, const u64* a1, const u64* b0, const u64* b1,
+                        u64* y0, u64* y1, u64* z0, u64* z1) {
+    const size_t count = (size_t)rows * cols;
+    orc_apply_permutation(tau0, x0, y0, rows, cols);
+    orc_apply_permutation(tau1, x1, y1, rows, cols);
+    for (size_t t = 0; t < count; ++t) {
+        y0[t] = y0[t] + a0[t];
+        y1[t] = y1[t] + a1[t];
+    }
+    orc_apply_permutation(rho0, y1, z0, rows, cols);      // party 0 works on what party 1 sent
+    orc_apply_permutation(rho1, y0, z1, rows, cols);
+    for (size_t t = 0; t < count; ++t) {
+        z0[t] = z0[t] - b0[t];
+        z1[t] = z1[t] - b1[t];
     }
 }
 

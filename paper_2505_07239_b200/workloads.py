@@ -283,6 +283,42 @@ def dealer_triple(seed: int, stream: str, rows: int, inner: int, cols: int, vali
     return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1)}
 
 
+def random_permutation(seed: int, stream: str, count: int) -> np.ndarray:
+    """Seeded uniform permutation of range(count) (rank of random keys), int32."""
+    keys = random_u64(seed, stream, count)
+    return np.argsort(keys, kind="stable").astype(np.int32)
+
+
+def dealer_shuffle(seed: int, stream: str, rows: int, cols: int, inverse_of: Optional[dict] = None) -> dict:
+    """What the trusted dealer hands out for one oblivious shuffle of the rows of a
+    [rows, cols] matrix (Protocol 1, offline stage): pi, (tau_0, tau_1), (rho_0, rho_1)
+    with pi = rho_0 o tau_1 = rho_1 o tau_0, masks (a_0, a_1), (b_0, b_1).
+    A permutation p acts as (p(x))[j] = x[p[j]].
+
+    With `inverse_of` (the material of an earlier shuffle) the sub-permutations are the
+    ones each party derives locally to undo that shuffle, tau'_i = rho_i^{-1} and
+    rho'_i = tau_i^{-1}; the masks are fresh.
+    """
+    def inv(p):
+        out = np.empty_like(p)
+        out[p] = np.arange(p.size, dtype=np.int32)
+        return out
+
+    if inverse_of is None:
+        pi = random_permutation(seed, stream + "/pi", rows)
+        tau = (random_permutation(seed, stream + "/tau0", rows), random_permutation(seed, stream + "/tau1", rows))
+        # rho_0 = pi o tau_1^{-1}: (p o q)[j] = q[p[j]]
+        rho = (inv(tau[1])[pi], inv(tau[0])[pi])
+    else:
+        tau = (inv(inverse_of["rho"][0]), inv(inverse_of["rho"][1]))
+        rho = (inv(inverse_of["tau"][0]), inv(inverse_of["tau"][1]))
+        pi = inv(inverse_of["pi"])
+    a = tuple(random_u64(seed, stream + f"/a{i}", rows * cols).reshape(rows, cols) for i in (0, 1))
+    c = random_u64(seed, stream + "/c", rows * cols).reshape(rows, cols)
+    b = (a[1][rho[0]] + c, a[0][rho[1]] - c)
+    return {"pi": pi, "tau": tau, "rho": rho, "a": a, "b": b, "c": c}
+
+
 def reshare(value: np.ndarray, seed: int, stream: str):
     """Fresh uniform sharing of a ring tensor (used after the activation functionality)."""
     return split_shares(value, seed, stream)
