@@ -205,6 +205,44 @@ const char* comet_strerror(int code);
 int comet_last_cuda_error(comet_ctx* ctx);
 
 /* ---------------------------------------------------------------------------
+ * Oblivious shuffle, Section 4.2, Protocol 1, online stage, for both parties.
+ * It is the step on either side of the sparse FFN: the input matrix is shuffled
+ * into the secret order of the revealed sparsity distribution before the
+ * up-projection, and the output is unshuffled after the down-projection.
+ *
+ * A permutation p acts on the ROWS of a [rows, cols] matrix of ring words as the
+ * paper's example fixes it, (p(x))[j] = x[p[j]] (0-based).  Party i holds its
+ * share X[i], its sub-permutations tau[i], rho[i] (int32, `rows` entries each,
+ * with pi = rho_0 o tau_1 = rho_1 o tau_0) and the dealer's masks a[i], b[i]
+ * ([rows, cols]; b_0 = rho_0(a_1) + c, b_1 = rho_1(a_0) - c).  The call computes
+ *     Y[i] = tau_i(X[i]) + a[i]          (the message party i sends), then
+ *     Z[i] = rho_i(Y[1-i]) - b[i]        (party i's share of pi(x)).
+ * Unshuffle is the same call with the sub-permutations each party derives
+ * locally, tau'_i = rho_i^{-1} and rho'_i = tau_i^{-1} (comet_invert_permutation),
+ * and fresh masks.
+ *
+ * Stateless: no context and no memory of the library's own.  Every pointer is a
+ * DEVICE pointer on the current device, owned by the caller; X, a, b are only
+ * read, Y and Z are overwritten and must not overlap any other argument.  Two
+ * kernels are enqueued on `cuda_stream` (NULL = default stream); the call does
+ * not wait for them.  16-byte accesses are used when cols is even and X, a, b,
+ * Y, Z are 16-byte aligned, 8-byte accesses otherwise.
+ * A permutation entry outside [0, rows) is never followed: the row it would
+ * have fetched counts as zero and, if `bad_index_flag` (device int32, may be
+ * NULL) is given, it is set to 1.  The caller clears the flag.
+ * Errors: INVALID_ARG (null pointer), SHAPE (rows or cols < 1 or >= 2^31), CUDA. */
+int comet_shuffle(void* cuda_stream, const uint64_t* const X[2], const int32_t* const tau[2],
+                  const int32_t* const rho[2], const uint64_t* const a[2], const uint64_t* const b[2],
+                  uint64_t* const Y[2], uint64_t* const Z[2], int64_t rows, int64_t cols, int32_t* bad_index_flag);
+
+/* inverse[perm[j]] = j for j in [0, rows): the local step by which a party turns
+ * its (rho_i, tau_i) into the sub-permutations of the unshuffle (Section 4.2,
+ * remark (ii)).  Device pointers; entries outside [0, rows) are skipped and
+ * reported through `bad_index_flag` as above. */
+int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* inverse, int64_t rows,
+                             int32_t* bad_index_flag);
+
+/* ---------------------------------------------------------------------------
  * Allocation-free Pi_MatMul.  (The paper has no counterpart; this exists for
  * deployment reasons only.)
  *

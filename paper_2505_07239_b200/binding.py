@@ -29,7 +29,7 @@ NUM_TENSORS = 17
 EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
-    "comet_set_profiling", "comet_beaver_matmul_static",
+    "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -83,6 +83,8 @@ def _load():
     lib.comet_set_profiling.argtypes = [vp, ctypes.c_int]
     pair = ctypes.c_void_p * 2
     lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
+    lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
+    lib.comet_invert_permutation.argtypes = [vp, vp, vp, i64, vp]
     return lib
 
 
@@ -230,3 +232,46 @@ def beaver_matmul_static(X, A, Y, B, C, Z, stream: Optional[torch.cuda.Stream] =
     sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
     return _lib.comet_beaver_matmul_static(sp, ptrs(X, (T, K)), ptrs(A, (T, K)), ptrs(Y, (N, K)), ptrs(B, (N, K)),
                                            ptrs(C, (T, N)), ptrs(Z, (T, N)), T, K, N)
+
+
+def _pair(ts, shape=None, dtype=None):
+    for t in ts:
+        assert t.is_cuda and t.is_contiguous()
+        assert shape is None or tuple(t.shape) == tuple(shape)
+        assert dtype is None or t.dtype == dtype
+    return (ctypes.c_void_p * 2)(ts[0].data_ptr(), ts[1].data_ptr())
+
+
+def shuffle(X, tau, rho, a, b, stream: Optional[torch.cuda.Stream] = None, bad_index_flag=None):
+    """Oblivious shuffle of the rows of a shared matrix (comet_shuffle), both parties.
+
+    Each argument is a pair (party 0, party 1) of CUDA tensors: X, a, b of 8-byte
+    words with the same shape [rows, ...]; tau, rho int32 of length rows.
+    Returns (Y, Z): the two messages and the two shares of pi(x).  Only the
+    output tensors are allocated here (torch); the arithmetic is the library's.
+    """
+    rows = X[0].shape[0]
+    cols = X[0].numel() // rows
+    Y = [torch.empty_like(X[0]) for _ in (0, 1)]
+    Z = [torch.empty_like(X[0]) for _ in (0, 1)]
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    flag = ctypes.c_void_p(bad_index_flag.data_ptr() if bad_index_flag is not None else 0)
+    for t in (*X, *a, *b):
+        assert t.element_size() == 8
+    code = _lib.comet_shuffle(sp, _pair(X), _pair(tau, (rows,), torch.int32), _pair(rho, (rows,), torch.int32),
+                              _pair(a, X[0].shape), _pair(b, X[0].shape), _pair(Y), _pair(Z), rows, cols, flag)
+    if code != OK:
+        raise CometError(code, "comet_shuffle")
+    return Y, Z
+
+
+def invert_permutation(perm, stream: Optional[torch.cuda.Stream] = None, bad_index_flag=None):
+    """inverse[perm[j]] = j on the device (comet_invert_permutation)."""
+    assert perm.is_cuda and perm.dtype == torch.int32 and perm.is_contiguous()
+    out = torch.empty_like(perm)
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    flag = ctypes.c_void_p(bad_index_flag.data_ptr() if bad_index_flag is not None else 0)
+    code = _lib.comet_invert_permutation(sp, perm.data_ptr(), out.data_ptr(), perm.numel(), flag)
+    if code != OK:
+        raise CometError(code, "comet_invert_permutation")
+    return out

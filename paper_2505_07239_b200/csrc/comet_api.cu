@@ -13,6 +13,7 @@
 
 #include "kernels_limb.cuh"
 #include "kernels_open.cuh"
+#include "kernels_shuffle.cuh"
 #include "kernels_simt.cuh"
 
 using comet::u64;
@@ -817,4 +818,74 @@ extern "C" int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* con
     comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, stream>>>(args);
     if (cudaGetLastError() != cudaSuccess) return COMET_ERR_CUDA;
     return COMET_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Oblivious shuffle (Protocol 1), online stage.  Stateless: no context, no
+// memory of its own.
+// ---------------------------------------------------------------------------
+namespace {
+
+int shuffle_grid(long long items) {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    long long want = (items + 255) / 256, cap = (long long)sms * 16;
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// out_i = in_i[perm_i] +/- mask_i for both parties, one launch
+int launch_shuffle_step(cudaStream_t stream, const uint64_t* const in[2], const int32_t* const perm[2],
+                        const uint64_t* const mask[2], uint64_t* const out[2], int64_t rows, int64_t cols,
+                        int subtract, int32_t* bad) {
+    comet::ShuffleArgs a;
+    bool vec = (cols % 2) == 0;
+    for (int p = 0; p < 2; ++p) {
+        a.in[p] = reinterpret_cast<const u64*>(in[p]);
+        a.perm[p] = perm[p];
+        a.mask[p] = reinterpret_cast<const u64*>(mask[p]);
+        a.out[p] = reinterpret_cast<u64*>(out[p]);
+        vec = vec && aligned16(in[p]) && aligned16(mask[p]) && aligned16(out[p]);
+    }
+    a.rows = rows;
+    a.pieces = (int)(vec ? cols / 2 : cols);
+    a.subtract = subtract;
+    a.bad_index = bad;
+    const int grid = shuffle_grid(rows * a.pieces);
+    const long long stride = (long long)grid * 256;
+    a.stride_rows = stride / a.pieces;
+    a.stride_pieces = (int)(stride % a.pieces);
+    if (vec) comet::shuffle_rows_kernel<ulonglong2><<<dim3(grid, 2), 256, 0, stream>>>(a);
+    else comet::shuffle_rows_kernel<u64><<<dim3(grid, 2), 256, 0, stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" int comet_shuffle(void* cuda_stream, const uint64_t* const X[2], const int32_t* const tau[2],
+                             const int32_t* const rho[2], const uint64_t* const a[2], const uint64_t* const b[2],
+                             uint64_t* const Y[2], uint64_t* const Z[2], int64_t rows, int64_t cols,
+                             int32_t* bad_index_flag) {
+    if (!X || !tau || !rho || !a || !b || !Y || !Z) return COMET_ERR_INVALID_ARG;
+    for (int p = 0; p < 2; ++p)
+        if (!X[p] || !tau[p] || !rho[p] || !a[p] || !b[p] || !Y[p] || !Z[p]) return COMET_ERR_INVALID_ARG;
+    if (rows < 1 || cols < 1 || rows > 0x7fffffffll || cols > 0x7fffffffll) return COMET_ERR_SHAPE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // [y]_i = tau_i([x]_i) + a_i
+    int rc = launch_shuffle_step(stream, X, tau, a, Y, rows, cols, 0, bad_index_flag);
+    if (rc != COMET_OK) return rc;
+    // the exchange: party i reads what the other party wrote.  [z]_i = rho_i([y]_other) - b_i
+    const uint64_t* const received[2] = {Y[1], Y[0]};
+    return launch_shuffle_step(stream, received, rho, b, Z, rows, cols, 1, bad_index_flag);
+}
+
+extern "C" int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* inverse, int64_t rows,
+                                        int32_t* bad_index_flag) {
+    if (!perm || !inverse) return COMET_ERR_INVALID_ARG;
+    if (rows < 1 || rows > 0x7fffffffll) return COMET_ERR_SHAPE;
+    comet::invert_permutation_kernel<<<shuffle_grid(rows), 256, 0, (cudaStream_t)cuda_stream>>>(perm, inverse, rows,
+                                                                                                  bad_index_flag);
+    return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
 }
