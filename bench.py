@@ -209,6 +209,73 @@ def workload_name(cfg, sparsity):
             f"block={cfg.block} sparsity={sparsity:.2f} n_active={n}")
 
 
+# --------------------------------------------------------------------------- oblivious shuffle (secondary line)
+def run_shuffle(args, cfg):
+    """`--op shuffle`: the online stage of the oblivious shuffle (Protocol 1) on the workload's activation matrix
+    [tokens, d_model], both parties, against the HBM roofline.  Algorithmic bytes per party: read x, a, the
+    received y and b, write y and z = 48 bytes per word, plus the two index arrays."""
+    import torch
+
+    from paper_2505_07239_b200 import binding as cb
+
+    rank, world, local = ranks.rank_world_local()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    rows, cols = cfg.tokens, cfg.d_model
+    if args.shuffle_rows:
+        rows = args.shuffle_rows
+    seed = ranks.rank_seed(2000, rank)
+    sets = max(4, int((2 * L2_FLUSH_BYTES) // (6 * 8 * rows * cols)) + 1)      # rotating sets well beyond L2
+    sets = min(sets, 64)
+    data = []
+    for s in range(sets):
+        m = wl.dealer_shuffle(seed, f"bench/shuffle/{s % 4}", rows, cols)      # 4 distinct draws, copied to fresh memory
+        x = wl.random_u64(seed, f"bench/shuffle/x/{s % 4}", rows * cols).reshape(rows, cols)
+        xs = wl.split_shares(x, seed, f"bench/shuffle/x/{s % 4}")
+        d64 = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int64)).to(dev)   # noqa: E731
+        d32 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)                  # noqa: E731
+        data.append(([d64(v) for v in xs], [d32(v) for v in m["tau"]], [d32(v) for v in m["rho"]],
+                     [d64(v) for v in m["a"]], [d64(v) for v in m["b"]]))
+    stream = torch.cuda.Stream(device=dev)
+    bytes_step = 2 * (48 * rows * cols + 8 * rows)
+    for s in range(max(3, args.warmup)):
+        cb.shuffle(*data[s % sets], stream=stream)
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    evs = []
+    for s in range(args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        cb.shuffle(*data[s % sets], stream=stream)
+        e1.record(stream)
+        evs.append((e0, e1))
+    torch.cuda.synchronize(dev)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = float(sum(a.elapsed_time(b) for a, b in evs))
+    (total_ms,) = ranks.max_over_ranks([total_ms], dev)
+    if rank != 0:
+        return
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    hbm = peaks.get("hbm_gbs", 6650.0)
+    gbs = ranks.whole_job_throughput(bytes_step, world, args.steps, total_ms) / 1e9
+    print(json.dumps({
+        "metric": "oblivious shuffle online stage, algorithmic GB/s", "value": gbs, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": f"rows={rows} cols={cols} (activation matrix of {cfg.name}), both parties",
+                   "l2": f"{sets} rotating input sets, {sets * 6 * 8 * rows * cols >> 20} MiB in total"},
+        "gpu_launches": 2 * args.steps, "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": gbs / world, "peak": hbm, "unit": "GB/s",
+                     "frac": gbs / world / hbm, "traffic": None, "kernel": "shuffle_rows_kernel (2 launches per step)",
+                     "peak_source": "measured" if peaks else "fallback"}}))
+
+
 # --------------------------------------------------------------------------- GPU leg
 def main():
     ap = argparse.ArgumentParser()
@@ -220,6 +287,9 @@ def main():
     ap.add_argument("--sparsity", type=float, default=None)
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "limb"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle"],
+                    help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage")
+    ap.add_argument("--shuffle-rows", type=int, default=0, help="--op shuffle: rows instead of the workload's tokens")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
     sparsity = args.sparsity
@@ -227,6 +297,8 @@ def main():
         sparsity = 0.9 if args.workload == "opt1.3b" else 1.0 - cfg.active_fraction
     if args.impl == "reference":
         return run_reference(args, cfg, sparsity)
+    if args.op == "shuffle":
+        return run_shuffle(args, cfg)
     if args.warmup < 3:
         args.warmup = 3
 
