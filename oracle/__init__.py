@@ -243,3 +243,15 @@ def shuffle_online(x, tau, rho, a, b):
     shape = np.shape(x[0])
     y0, y1, z0, z1 = (o.reshape(shape) for o in outs)
     return (y0, y1), (z0, z1)
+
+
+def beaver_mul(x, y, a, b, c):
+    """Element-wise Beaver product of Eq. 1 for both parties.  Every argument is a pair of
+    equally shaped uint64 arrays.  Returns dict with the messages D, E and the result Z (pairs)."""
+    arrs = _pairs(x, y, a, b, c)
+    shape = arrs[0].shape
+    for v in arrs:
+        assert v.shape == shape
+    outs = [np.empty(shape, U64) for _ in range(6)]
+    lib().orc_beaver_mul(ctypes.c_size_t(arrs[0].size), *[_p(v) for v in arrs], *[_p(o) for o in outs])
+    return {"D": (outs[0], outs[1]), "E": (outs[2], outs[3]), "Z": (outs[4], outs[5])}

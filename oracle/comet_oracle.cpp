@@ -285,4 +285,32 @@ void orc_shuffle_online(int rows, int cols, const u64* x0, const u64* x1,
     }
 }
 
+// ---------------------------------------------------------------------------
+// Section 2.1, "Multiplication", Eq. 1 taken element by element (the product
+// ReLU(gate) * up of a gated FFN is of this kind): for every element,
+// [d]_i = [x]_i - [a]_i and [e]_i = [y]_i - [b]_i are exchanged, d and e
+// reconstructed, and [z]_i = [c]_i + d*[b]_i + e*[a]_i + i*d*e.
+// ---------------------------------------------------------------------------
+void orc_beaver_mul(size_t count, const u64* x0, const u64* x1, const u64* y0, const u64* y1,
+                    const u64* a0, const u64* a1, const u64* b0, const u64* b1, const u64* c0, const u64* c1,
+                    u64* d0, u64* d1, u64* e0, u64* e1, u64* z0, u64* z1) {
+    const u64* xs[2] = {x0, x1};
+    const u64* ys[2] = {y0, y1};
+    const u64* as[2] = {a0, a1};
+    const u64* bs[2] = {b0, b1};
+    const u64* cs[2] = {c0, c1};
+    u64* ds[2] = {d0, d1};
+    u64* es[2] = {e0, e1};
+    u64* zs[2] = {z0, z1};
+    for (int i = 0; i < 2; ++i)
+        for (size_t t = 0; t < count; ++t) {
+            ds[i][t] = xs[i][t] - as[i][t];
+            es[i][t] = ys[i][t] - bs[i][t];
+        }
+    for (size_t t = 0; t < count; ++t) {
+        const u64 d = d0[t] + d1[t], e = e0[t] + e1[t];
+        for (int i = 0; i < 2; ++i) zs[i][t] = cs[i][t] + d * bs[i][t] + e * as[i][t] + (u64)i * (d * e);
+    }
+}
+
 }  // extern "C"

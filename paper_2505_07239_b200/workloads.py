@@ -283,6 +283,18 @@ def dealer_triple(seed: int, stream: str, rows: int, inner: int, cols: int, vali
     return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1)}
 
 
+def dealer_triple_elementwise(seed: int, stream: str, shape) -> dict:
+    """Element-wise Beaver triple: a, b uniform, c = a * b mod 2^64 element by element, each split into two
+    uniform shares.  Returns {"a": (a, a0, a1), "b": ..., "c": ...}."""
+    count = int(np.prod(shape))
+    a = random_u64(seed, stream + "/a", count).reshape(shape)
+    b = random_u64(seed, stream + "/b", count).reshape(shape)
+    with np.errstate(over="ignore"):
+        c = a * b
+    return {"a": (a, *split_shares(a, seed, stream + "/a")), "b": (b, *split_shares(b, seed, stream + "/b")),
+            "c": (c, *split_shares(c, seed, stream + "/c"))}
+
+
 def random_permutation(seed: int, stream: str, count: int) -> np.ndarray:
     """Seeded uniform permutation of range(count) (rank of random keys), int32."""
     keys = random_u64(seed, stream, count)
