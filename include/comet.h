@@ -243,6 +243,21 @@ int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* in
                              int32_t* bad_index_flag);
 
 /* ---------------------------------------------------------------------------
+ * Element-wise Beaver product, Section 2.1 "Multiplication", Eq. 1 applied to
+ * every element (in a gated FFN: ReLU(gate) times up), for both parties:
+ *     D[i] = X[i] - A[i],  E[i] = Y[i] - B[i]            (the two messages), then
+ *     Z[i] = C[i] + d*B[i] + e*A[i] + i*d*e,  d = D[0]+D[1], e = E[0]+E[1],
+ * element by element mod 2^64, with an element-wise triple c = a*b.  The result
+ * is at scale 2f when both factors are at scale f; truncate it afterwards.
+ * Stateless; all pointers are DEVICE pointers on the current device to `count`
+ * words each, owned by the caller; D, E, Z are overwritten and must not overlap
+ * the inputs.  Two kernels are enqueued on `cuda_stream`; the call does not wait.
+ * Errors: INVALID_ARG (null pointer), SHAPE (count < 1), CUDA. */
+int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], const uint64_t* const Y[2],
+                     const uint64_t* const A[2], const uint64_t* const B[2], const uint64_t* const C[2],
+                     uint64_t* const D[2], uint64_t* const E[2], uint64_t* const Z[2], int64_t count);
+
+/* ---------------------------------------------------------------------------
  * Allocation-free Pi_MatMul.  (The paper has no counterpart; this exists for
  * deployment reasons only.)
  *

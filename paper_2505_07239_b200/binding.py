@@ -30,6 +30,7 @@ EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
+    "comet_beaver_mul",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -85,6 +86,7 @@ def _load():
     lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
     lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
     lib.comet_invert_permutation.argtypes = [vp, vp, vp, i64, vp]
+    lib.comet_beaver_mul.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, pair, i64]
     return lib
 
 
@@ -275,3 +277,21 @@ def invert_permutation(perm, stream: Optional[torch.cuda.Stream] = None, bad_ind
     if code != OK:
         raise CometError(code, "comet_invert_permutation")
     return out
+
+
+def beaver_mul(X, Y, A, B, C, stream: Optional[torch.cuda.Stream] = None):
+    """Element-wise Beaver product of two shared tensors (comet_beaver_mul), both parties.
+    Every argument is a pair of equally shaped CUDA tensors of 8-byte words.
+    Returns (D, E, Z): the messages x - a and y - b, and the shares of x * y."""
+    shape = X[0].shape
+    for t in (*X, *Y, *A, *B, *C):
+        assert t.element_size() == 8 and t.shape == shape
+    D = [torch.empty_like(X[0]) for _ in (0, 1)]
+    E = [torch.empty_like(X[0]) for _ in (0, 1)]
+    Z = [torch.empty_like(X[0]) for _ in (0, 1)]
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    code = _lib.comet_beaver_mul(sp, _pair(X), _pair(Y), _pair(A), _pair(B), _pair(C), _pair(D), _pair(E), _pair(Z),
+                                 X[0].numel())
+    if code != OK:
+        raise CometError(code, "comet_beaver_mul")
+    return D, E, Z

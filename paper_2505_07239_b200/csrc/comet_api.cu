@@ -12,6 +12,7 @@
 #include <cuda_runtime.h>
 
 #include "kernels_limb.cuh"
+#include "kernels_mul.cuh"
 #include "kernels_open.cuh"
 #include "kernels_shuffle.cuh"
 #include "kernels_simt.cuh"
@@ -887,5 +888,39 @@ extern "C" int comet_invert_permutation(void* cuda_stream, const int32_t* perm, 
     if (rows < 1 || rows > 0x7fffffffll) return COMET_ERR_SHAPE;
     comet::invert_permutation_kernel<<<shuffle_grid(rows), 256, 0, (cudaStream_t)cuda_stream>>>(perm, inverse, rows,
                                                                                                   bad_index_flag);
+    return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
+// Element-wise Beaver product (Eq. 1 element by element).  Stateless.
+// ---------------------------------------------------------------------------
+extern "C" int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], const uint64_t* const Y[2],
+                                const uint64_t* const A[2], const uint64_t* const B[2], const uint64_t* const C[2],
+                                uint64_t* const D[2], uint64_t* const E[2], uint64_t* const Z[2], int64_t count) {
+    if (!X || !Y || !A || !B || !C || !D || !E || !Z) return COMET_ERR_INVALID_ARG;
+    for (int p = 0; p < 2; ++p)
+        if (!X[p] || !Y[p] || !A[p] || !B[p] || !C[p] || !D[p] || !E[p] || !Z[p]) return COMET_ERR_INVALID_ARG;
+    if (count < 1) return COMET_ERR_SHAPE;
+    comet::MulArgs g;
+    bool vec = (count % 2) == 0;
+    for (int p = 0; p < 2; ++p) {
+        g.x[p] = reinterpret_cast<const u64*>(X[p]); g.y[p] = reinterpret_cast<const u64*>(Y[p]);
+        g.a[p] = reinterpret_cast<const u64*>(A[p]); g.b[p] = reinterpret_cast<const u64*>(B[p]);
+        g.c[p] = reinterpret_cast<const u64*>(C[p]);
+        g.d[p] = reinterpret_cast<u64*>(D[p]); g.e[p] = reinterpret_cast<u64*>(E[p]);
+        g.z[p] = reinterpret_cast<u64*>(Z[p]);
+        vec = vec && aligned16(X[p]) && aligned16(Y[p]) && aligned16(A[p]) && aligned16(B[p]) && aligned16(C[p]) &&
+              aligned16(D[p]) && aligned16(E[p]) && aligned16(Z[p]);
+    }
+    g.pieces = vec ? count / 2 : count;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const dim3 grid(shuffle_grid(g.pieces), 2);
+    if (vec) {
+        comet::beaver_mul_open_kernel<ulonglong2><<<grid, 256, 0, stream>>>(g);
+        comet::beaver_mul_combine_kernel<ulonglong2><<<grid, 256, 0, stream>>>(g);      // after the exchange
+    } else {
+        comet::beaver_mul_open_kernel<u64><<<grid, 256, 0, stream>>>(g);
+        comet::beaver_mul_combine_kernel<u64><<<grid, 256, 0, stream>>>(g);
+    }
     return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
 }
