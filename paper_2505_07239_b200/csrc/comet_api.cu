@@ -41,6 +41,7 @@ struct comet_ctx {
     cudaEvent_t ev_fork, ev_join;
     bool side_pending;                // ev_join not yet waited for on the main stream
     bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
+    bool dn_right_few;                // ... and were laid out for the few-token kernel (128-row tiles)
     uint8_t* d_mask;
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
@@ -163,6 +164,9 @@ Proj proj_down(const comet_ctx* c, int tokens) {
                 COMET_C_DN, COMET_Y, true};
 }
 
+// The few-token kernel (operand roles exchanged) serves products with at most 32 token rows.
+inline bool limb_few(const Proj& pr) { return pr.M <= comet::limb_few::BT; }
+
 // Makes the main stream wait for the side stream's outstanding work (if any).
 int join_side(comet_ctx* c) {
     if (c->side_pending) {
@@ -199,6 +203,7 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.ldw = pr.down ? c->cfg.d_ff : c->cfg.d_model;
     a.kblocks = kb;
     a.down = pr.down ? 1 : 0;
+    a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
@@ -225,6 +230,8 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
         a.Z[p] = c->buf[p][pr.idZ];
     }
     a.M = pr.M; a.N = pr.N; a.K = pr.K; a.kblocks = kb;
+    a.left_tile_rows = limb_few(pr) ? comet::limb_few::BT : lb::BM;
+    a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
     a.left_tiles = left ? kb * ceil_div(pr.M, lb::PREP_ROWS) : 0;
     a.right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
@@ -238,10 +245,14 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
     return COMET_OK;
 }
 
-// Tensor-core path: the persistent stream-K kernel over both parties' tiles.
+// Tensor-core path: the persistent stream-K kernel over both parties' tiles (the few-token variant when the
+// product has at most 32 token rows).
 int limb_combine(comet_ctx* c, const Proj& pr) {
     namespace lb = comet::limb;
-    const int kb = ceil_div(pr.K, lb::KC), mt = ceil_div(pr.M, lb::BM), nt = ceil_div(pr.N, lb::BN);
+    namespace lf = comet::limb_few;
+    const bool few = limb_few(pr);
+    const int kb = ceil_div(pr.K, lb::KC);
+    const int mt = few ? 1 : ceil_div(pr.M, lb::BM), nt = few ? ceil_div(pr.N, lf::BW) : ceil_div(pr.N, lb::BN);
     uint8_t* (*planes)[2] = pr.down ? c->planes_right_dn : c->planes_right_up;
     comet::LimbArgs a;
     for (int p = 0; p < 2; ++p) {
@@ -257,7 +268,8 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
         PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
-        comet::combine_limb_kernel<<<grid, lb::THREADS, lb::SMEM_BYTES, c->stream>>>(a);
+        if (few) comet::combine_limb_few_kernel<<<grid, lf::THREADS, lf::SMEM_BYTES, c->stream>>>(a);
+        else comet::combine_limb_kernel<<<grid, lb::THREADS, lb::SMEM_BYTES, c->stream>>>(a);
     }
     c->stats.kernel_launches += 1;
     c->stats.matmul_path = COMET_PATH_LIMB;
@@ -267,7 +279,9 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
 
 bool limb_fits(const comet_ctx* c, const Proj& pr) {
     namespace lb = comet::limb;
-    const size_t kb = ceil_div(pr.K, lb::KC), mt = ceil_div(pr.M, lb::BM), nt = ceil_div(pr.N, lb::BN);
+    // the few-token layout (32-row token tiles, 128-row weight tiles) never needs more than the ordinary one
+    // plus one 64-row tile of the right operand, which the allocation includes
+    const size_t kb = ceil_div(pr.K, lb::KC), mt = ceil_div(pr.M, lb::BM), nt = ceil_div(pr.N, lb::BN) + 1;
     return mt * kb * lb::A_BLOCK_BYTES <= c->planes_left_bytes &&
            nt * kb * lb::B_BLOCK_BYTES <= (pr.down ? c->planes_right_dn_bytes : c->planes_right_up_bytes);
 }
@@ -369,8 +383,8 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
         const int64_t kb_max = kb_up > kb_dn ? kb_up : kb_dn;
         const int64_t mt = (c->cap_T + lb::BM - 1) / lb::BM;
         c->planes_left_bytes = (size_t)(mt * kb_max) * lb::A_BLOCK_BYTES;
-        c->planes_right_up_bytes = (size_t)(((gn + lb::BN - 1) / lb::BN) * kb_up) * lb::B_BLOCK_BYTES;
-        c->planes_right_dn_bytes = (size_t)(((d + lb::BN - 1) / lb::BN) * kb_dn) * lb::B_BLOCK_BYTES;
+        c->planes_right_up_bytes = (size_t)(((gn + lb::BN - 1) / lb::BN + 1) * kb_up) * lb::B_BLOCK_BYTES;
+        c->planes_right_dn_bytes = (size_t)(((d + lb::BN - 1) / lb::BN + 1) * kb_dn) * lb::B_BLOCK_BYTES;
         for (int p = 0; p < 2 && ok; ++p)
             for (int w = 0; w < 2 && ok; ++w) {
                 ok = cudaMalloc((void**)&c->planes_left[p][w], c->planes_left_bytes) == cudaSuccess;
@@ -381,6 +395,10 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
                                         (int)lb::SMEM_BYTES) == cudaSuccess;
         // the memory-side kernels may share an SM with a resident tensor-core CTA (which forces the largest
         // shared-memory carve-out), so they ask for the same carve-out
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_few_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)comet::limb_few::SMEM_BYTES) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_few_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::limb_open_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -556,6 +574,7 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
             COMET_CUDA(c, cudaEventRecord(c->ev_join, c->side));
             c->side_pending = true;
             c->dn_right_ready = true;
+            c->dn_right_few = limb_few(dn);
         }
         return limb_combine(c, up);
     }
@@ -609,7 +628,8 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
     if (c->path == COMET_PATH_LIMB) {
         const Proj dn = proj_down(c, tokens);
         if (!limb_fits(c, dn)) return COMET_ERR_SHAPE;
-        const bool have_right = c->dn_right_ready;     // opened early, during the up-projection
+        // opened early, during the up-projection, and in the plane layout this token count needs
+        const bool have_right = c->dn_right_ready && c->dn_right_few == limb_few(dn);
         int rc = join_side(c);
         if (rc != COMET_OK) return rc;
         {

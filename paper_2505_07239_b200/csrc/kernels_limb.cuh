@@ -123,6 +123,7 @@ struct LimbOpenArgs {
     int rows, K;             // logical size of the right operand [rows, K]
     int ldw;                 // words per row of W
     int kblocks, down;
+    int right_tile_rows;     // rows per plane tile of the right operand: 64, or 128 for the few-token kernel
 };
 
 __global__ void __launch_bounds__(256)
@@ -182,8 +183,8 @@ limb_open_kernel(LimbOpenArgs a) {
     if (tid < 128) {
         const int half = tid >> 6, r = tid & 63;
         int rin;
-        uint8_t* blk = limb_block_ptr(party ? a.Bpl[1] : a.Bpl[0], BN, row0 + r, a.kblocks, kb, &rin);
-        limb_emit_planes(sB, r, half, blk, BN, rin);
+        uint8_t* blk = limb_block_ptr(party ? a.Bpl[1] : a.Bpl[0], a.right_tile_rows, row0 + r, a.kblocks, kb, &rin);
+        limb_emit_planes(sB, r, half, blk, a.right_tile_rows, rin);
     }
 }
 
@@ -204,6 +205,7 @@ struct LimbPrepArgs {
     uint8_t* Fpl[2];
     int N, right_tiles;      // right_tiles = kblocks * ceil(N / 64), or 0
     int K, kblocks;
+    int left_tile_rows, right_tile_rows;   // rows per plane tile: 128 / 64, or 32 / 128 for the few-token kernel
     const u64* C[2];
     u64* Z[2];
     long long copy_pairs;
@@ -267,7 +269,7 @@ limb_prep_kernel(LimbPrepArgs a) {
     const int which = tid >> 7;                       // 0: the summed message, 1: the party's own operand
     if (which == 1 && !left) return;
     const int half = (tid >> 6) & 1, r = tid & 63;
-    const int tile_rows = left ? BM : BN;
+    const int tile_rows = left ? a.left_tile_rows : a.right_tile_rows;
     uint8_t* base = left ? (which ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]))
                          : (party ? a.Fpl[1] : a.Fpl[0]);
     int rin;
@@ -622,6 +624,217 @@ combine_limb_kernel(LimbArgs a) {
     if (warp == 0) {
         ptx::fence_after_sync();
         ptx::tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Few tokens (M <= 32, the decode step): the roles of the two operands are exchanged.  The weight-side operand
+// (B_i, then F) supplies the 128 rows of the MMA, one limb plane per instruction, and the token-side operand
+// (E, then V_i) is the one whose planes are stacked along N: 32 token rows per plane, so right plane q meets
+// left planes 0..7-q in one instruction of N = 32*(8-q) <= 256, 8 instructions per 32-deep step, and the eight
+// accumulators D_s (128 neurons x 32 tokens) take 256 TMEM columns.  A 128-row tile of the ordinary kernel would
+// spend three quarters of its tensor work on padding rows here.  Every weight plane is used by exactly one tile,
+// so the kernel streams them once; it is bound by that traffic, not by the tensor pipe.
+// Plane layouts: token side [k-block][8 planes x 32 rows x 32 B] (8 KiB blocks), weight side
+// [n-tile of 128][k-block][32 KiB].  The output tile Z^T (neurons x tokens) is transposed through shared memory
+// so that each bulk reduction adds 32 consecutive neurons of one token row.
+// ---------------------------------------------------------------------------
+namespace limb_few {
+constexpr int BW = 128, BT = 32, KC = limb::KC, PLANES = limb::PLANES;
+constexpr int W_BLOCK_BYTES = PLANES * BW * KC;   // 32 KiB
+constexpr int T_BLOCK_BYTES = PLANES * BT * KC;   // 8 KiB
+constexpr int STAGES = 4;
+constexpr int EPI_WARPS = 8;                      // warp w: neurons 32*(w%4).., tokens 16*(w/4)..
+constexpr int THREADS = 32 * (EPI_WARPS + 2);
+constexpr int OUT_BYTES_PER_WARP = 16 * 32 * 8;   // 16 token rows x 32 neurons
+constexpr int TMEM_COLS = PLANES * BT;            // 256
+constexpr size_t SMEM_BYTES = (size_t)STAGES * (W_BLOCK_BYTES + T_BLOCK_BYTES) + (size_t)EPI_WARPS * OUT_BYTES_PER_WARP + 128;
+}  // namespace limb_few
+
+// LimbArgs as for combine_limb_kernel with Epl/Vpl = token-side planes, Bpl/Fpl = weight-side planes, mt = 1,
+// nt = ceil(N / 128), M <= 32.
+__global__ void __launch_bounds__(limb_few::THREADS, 1)
+combine_limb_few_kernel(LimbArgs a) {
+    using namespace limb_few;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[STAGES];
+    __shared__ __align__(8) uint64_t empty_bar[STAGES];
+    __shared__ __align__(8) uint64_t accum_full_bar, accum_empty_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    uint8_t* sW = smem;
+    uint8_t* sT = smem + (size_t)STAGES * W_BLOCK_BYTES;
+    uint8_t* sOut = sT + (size_t)STAGES * T_BLOCK_BYTES;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long total_units = 2ll * a.mt * a.nt * 2ll * a.kb;
+    const long long u_begin = total_units * blockIdx.x / gridDim.x;
+    const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_u32(&accum_full_bar), 1);
+        ptx::mbar_init(ptx::smem_u32(&accum_empty_bar), 32 * EPI_WARPS);
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    if (warp == 0) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::fence_before_sync();
+    __syncthreads();
+    ptx::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == EPI_WARPS) {
+        // ---------------- producer: one bulk copy per operand block ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int issued = 0;
+            bool ok = true;
+            const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
+            const uint32_t sW0 = ptx::smem_u32(sW), sT0 = ptx::smem_u32(sT);
+            for (long long u = u_begin; u < u_end && ok;) {
+                const LimbSegment sg = limb_segment(a, u, u_end);
+                u += sg.count;
+                int kpos = sg.kpos;
+                bool second = kpos >= a.kb;
+                if (second) kpos -= a.kb;
+                const uint8_t* tok = (second ? (sg.party ? a.Vpl[1] : a.Vpl[0]) : (sg.party ? a.Epl[1] : a.Epl[0])) +
+                                     (size_t)kpos * T_BLOCK_BYTES;
+                const uint8_t* wgt = (second ? (sg.party ? a.Fpl[1] : a.Fpl[0]) : (sg.party ? a.Bpl[1] : a.Bpl[0])) +
+                                     ((size_t)sg.tn * a.kb + kpos) * W_BLOCK_BYTES;
+                for (int it = 0; it < sg.count; ++it) {
+                    ok = limb_wait(empty0 + 8 * stage, phase ^ 1u, &abort_flag);
+                    if (!ok) break;
+                    const uint32_t bar = full0 + 8 * stage;
+                    ptx::mbar_expect_tx(bar, W_BLOCK_BYTES + T_BLOCK_BYTES);
+                    ptx::bulk_g2s(sW0 + stage * W_BLOCK_BYTES, wgt, W_BLOCK_BYTES, bar);
+                    ptx::bulk_g2s(sT0 + stage * T_BLOCK_BYTES, tok, T_BLOCK_BYTES, bar);
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    tok += T_BLOCK_BYTES;
+                    wgt += W_BLOCK_BYTES;
+                    if (++kpos == a.kb && !second) {
+                        second = true;
+                        kpos = 0;
+                        tok = (sg.party ? a.Vpl[1] : a.Vpl[0]);
+                        wgt = (sg.party ? a.Fpl[1] : a.Fpl[0]) + (size_t)sg.tn * a.kb * W_BLOCK_BYTES;
+                    }
+                }
+            }
+            if (!ok) {
+                const int back = issued < STAGES ? issued : STAGES;
+                for (int j = 1; j <= back; ++j) {
+                    int s = stage - j;
+                    uint32_t ph = phase;
+                    if (s < 0) { s += STAGES; ph ^= 1u; }
+                    const long long t0 = clock64();
+                    while (!ptx::mbar_try_wait(ptx::smem_u32(&full_bar[s]), ph) && clock64() - t0 < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == EPI_WARPS + 1) {
+        // ---------------- MMA issuer: weight plane q against token planes 0..7-q ----------------
+        if (lane == 0) {
+            constexpr uint32_t IDESC = (2u << 4) | ((uint32_t)(BW >> 4) << 24);
+            const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
+            const uint32_t accum_full = ptx::smem_u32(&accum_full_bar), accum_empty = ptx::smem_u32(&accum_empty_bar);
+            const uint32_t w_lo0 = limb_desc_lo(ptx::smem_u32(sW)), t_lo0 = limb_desc_lo(ptx::smem_u32(sT));
+            int stage = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (long long u = u_begin; u < u_end && ok;) {
+                const LimbSegment sg = limb_segment(a, u, u_end);
+                u += sg.count;
+                ok = limb_wait(accum_empty, acc_phase ^ 1u, &abort_flag);
+                if (!ok) break;
+                ptx::fence_after_sync();
+                uint32_t acc = 0;
+                for (int it = 0; it < sg.count; ++it) {
+                    ok = limb_wait(full0 + 8 * stage, phase, &abort_flag);
+                    if (!ok) break;
+                    ptx::fence_after_sync();
+                    const uint32_t w_lo = w_lo0 + stage * (W_BLOCK_BYTES >> 4);
+                    const uint32_t t_lo = t_lo0 + stage * (T_BLOCK_BYTES >> 4);
+#pragma unroll
+                    for (int q = 0; q < PLANES; ++q)
+                        ptx::mma_i8(tmem_base + BT * q, w_lo + ((q * BW * KC) >> 4), LIMB_DESC_HI, t_lo, LIMB_DESC_HI,
+                                    IDESC | ((uint32_t)((BT * (PLANES - q)) >> 3) << 17), q == 0 ? acc : 1u);
+                    ptx::mma_commit(empty0 + 8 * stage);
+                    acc = 1u;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                ptx::mma_commit(accum_full);
+                acc_phase ^= 1u;
+            }
+        }
+    } else {
+        // ---------------- epilogue: lane = neuron, registers = tokens; transpose through shared memory ----------------
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        const int quarter = warp & 3, thalf = warp >> 2;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + thalf * 16;
+        u64* stage_out = reinterpret_cast<u64*>(sOut + (size_t)warp * OUT_BYTES_PER_WARP);   // [16 tokens][32 neurons]
+        for (long long u = u_begin; u < u_end && ok;) {
+            const LimbSegment sg = limb_segment(a, u, u_end);
+            u += sg.count;
+            ok = limb_wait(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ptx::fence_after_sync();
+            u64 z[16];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t d[PLANES][8];
+#pragma unroll
+                for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BT * s + c * 8, d[s]);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    u64 v = (u64)d[0][j];
+#pragma unroll
+                    for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
+                    z[c * 8 + j] = v;
+                }
+            }
+            ptx::fence_before_sync();
+            ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
+            if (lane < 16) ptx::bulk_wait_group_read0();       // this lane's previous reduction has read its row
+            __syncwarp();
+#pragma unroll
+            for (int t = 0; t < 16; ++t) stage_out[t * 32 + lane] = z[t];
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            const int token = thalf * 16 + lane;               // lanes 0..15 each own one token row of the piece
+            const int col0 = sg.tn * BW + quarter * 32;
+            int cols = a.N - col0;
+            if (cols > 32) cols = 32;
+            if (lane < 16) {
+                if (token < a.M && cols > 0)
+                    ptx::bulk_reduce_add_u64((sg.party ? a.Z[1] : a.Z[0]) + (size_t)token * a.N + col0,
+                                             ptx::smem_u32(stage_out + lane * 32), (uint32_t)cols * 8u);
+                ptx::bulk_commit_group();
+            }
+            acc_phase ^= 1u;
+        }
+        if (lane < 16) ptx::bulk_wait_group0();
+    }
+
+    ptx::fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) *a.error_flag = 1;
+    if (warp == 0) {
+        ptx::fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, limb_few::TMEM_COLS);
     }
 }
 
