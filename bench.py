@@ -461,24 +461,32 @@ def main():
         bf16 = peaks.get("bf16_tflops", 1590.0)
         src = "measured" if peaks else "fallback"
         achieved = comb_macs_per_launch / (comb_launch_ms * 1e-3) / 1e12
+        # per launch, both parties: planes of both operand pairs read once, Z read and written once (average of the
+        # up- and the down-projection launch)
+        comb_bytes_per_launch = 8 * ((2 * T * d + 2 * d * g * n + 2 * T * g * n) + (2 * T * n + 2 * n * d + 2 * T * d))
         if used_path == "limb":
             # int8 tensor peak = measured bf16 peak x nominal ratio 2, in MAC/s, over 36 limb products per ring MAC
             peak = bf16 * 1e12 / 2 * 2 / 36 / 1e12
-            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
-                    "peak_source": f"{src} bf16 GEMM peak x2 (int8 nominal ratio), as MAC/s, / 36 limb products"}
+            t_tensor = comb_macs_per_launch / (peak * 1e12)
+            t_hbm = comb_bytes_per_launch / (hbm * 1e9)
+            if t_hbm > t_tensor:
+                # few tokens: the kernel streams the weight-side planes once and is bound by that traffic
+                roof = {"bound": "hbm", "achieved": comb_bytes_per_launch / (comb_launch_ms * 1e-3) / 1e9, "peak": hbm,
+                        "unit": "GB/s", "peak_source": f"{src} HBM copy peak"}
+            else:
+                roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
+                        "peak_source": f"{src} bf16 GEMM peak x2 (int8 nominal ratio), as MAC/s, / 36 limb products"}
         else:
             # 148 SMs x 64 32-bit integer multiply-add lanes per clock x max SM clock / 4 issue slots per ring MAC
             peak = 148 * 64 * 1.965e9 / 4 / 1e12
             roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
                     "peak_source": "148 SM x 64 int32 mul-add lanes/clk x 1.965 GHz / 4 issue slots per 64-bit MAC"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["kernel"] = "combine_" + used_path
+        roof["kernel"] = "combine_" + used_path + ("_few" if used_path == "limb" and T <= 32 else "")
         roof["traffic"] = combine_traffic(args.workload, sparsity, used_path)
         roof["traffic_unit"] = "bytes per launch (ncu dram read+write); algorithmic: planes once + Z read-modify-write"
-        # per party: planes of both operand pairs read once, Z read and written once; averaged over the two launches
-        roof["algorithmic_bytes_per_launch"] = 8 * ((2 * T * d + 2 * d * g * n + 2 * T * g * n) +
-                                                    (2 * T * n + 2 * n * d + 2 * T * d))
-        t_roof = max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (roof["peak"] * 1e12))
+        roof["algorithmic_bytes_per_launch"] = comb_bytes_per_launch
+        t_roof = max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (peak * 1e12))     # peak: the multiply pipe's, T MAC64/s
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

@@ -173,6 +173,25 @@ def simm(X, Y, I, A, B, C):
     return {"E": (E0, E1), "F": (F0, F1), "Z": (Z0, Z1)}
 
 
+def simm_rowsets(X, Y, I, S, A, B, C):
+    """Protocol 3 with per-column row sets: S is the [T, n] sparsity distribution of the compact X
+    (non-zero = present).  Returns E [T,n] (zero off the support), F [n,N], Z [T,N] and the number of
+    masked entries of X."""
+    X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1 = _pairs(X, Y, A, B, C)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    S = np.ascontiguousarray(S, dtype=np.uint8)
+    T, n = X0.shape
+    _, N = Y0.shape
+    assert I.size == n and S.shape == (T, n) and A0.shape == (T, n) and B0.shape == (n, N) and C0.shape == (T, N)
+    E0, E1 = np.empty((T, n), U64), np.empty((T, n), U64)
+    F0, F1 = np.empty((n, N), U64), np.empty((n, N), U64)
+    Z0, Z1 = np.empty((T, N), U64), np.empty((T, N), U64)
+    lib().orc_simm_rowsets.restype = ctypes.c_longlong
+    masked = lib().orc_simm_rowsets(ctypes.c_int(T), ctypes.c_int(n), ctypes.c_int(N), _p(I), _p(S),
+                                    *[_p(a) for a in (X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, Z0, Z1)])
+    return {"E": (E0, E1), "F": (F0, F1), "Z": (Z0, Z1), "masked": int(masked)}
+
+
 def truncate(party: int, Z, frac_bits: int):
     Z = _u64(Z)
     out = np.empty_like(Z)

@@ -17,6 +17,9 @@
 // closed forms and the {0,1}-ulp invariant; hand-computed fixtures.
 // Parity unpinned: the individual share values Z_i (as opposed to their sum)
 // are fixed only by Eq. 1 itself plus this repository's seeded inputs.
+// SIMM with per-column row sets R_j (Protocol 3 in general): pinned by the masked
+// plaintext product, by its reduction to the token-shared case under an
+// all-ones distribution, and by the counts of Theorem 2.
 // Oblivious shuffle (Protocol 1): pinned by the paper's worked permutation
 // example, by z_1 + z_2 = pi(x) against numpy indexing, by the operator
 // identities rho_1 o tau_2 = rho_2 o tau_1 = pi, by exhaustive permutations of
@@ -210,6 +213,67 @@ void orc_simm(int T, int n, int N, const int32_t* I,
                 }
             }
     }
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 3 (SIMM) with a sparsity distribution S of X that differs from row
+// to row: S is [T, n] over the compact columns (non-zero byte = X[r, c] is a
+// non-zero), so R_j of compact column c is {r : S[r, c] != 0} (lines 1-5).
+// A column with empty R_j is not a "nonzero column": nothing of it is masked,
+// sent or multiplied, and its message rows stay zero.  For the others, only the
+// entries of x'' = X[R_j, j] are masked and sent (E is zero off the support),
+// row I[c] of Y is masked once, and the outer product of Eq. 1 is added into the
+// rows in R_j (Merge&Sum).  a_j lives in A'[R_j, c] (whatever A' holds off the
+// support is ignored); the dealer's C' is the sum over j of a_j b_j^T scattered
+// to the rows R_j.  Returns the number of masked entries of X (the nnz of S).
+// ---------------------------------------------------------------------------
+long long orc_simm_rowsets(int T, int n, int N, const int32_t* I, const uint8_t* S,
+                           const u64* X0, const u64* X1, const u64* Y0, const u64* Y1,
+                           const u64* A0, const u64* A1, const u64* B0, const u64* B1,
+                           const u64* C0, const u64* C1,
+                           u64* E0, u64* E1, u64* F0, u64* F1, u64* Z0, u64* Z1) {
+    const u64* Xs[2] = {X0, X1};
+    const u64* Ys[2] = {Y0, Y1};
+    const u64* As[2] = {A0, A1};
+    const u64* Bs[2] = {B0, B1};
+    const u64* Cs[2] = {C0, C1};
+    u64* Es[2] = {E0, E1};
+    u64* Fs[2] = {F0, F1};
+    u64* Zs[2] = {Z0, Z1};
+    for (int i = 0; i < 2; ++i) {
+        for (size_t t = 0; t < (size_t)T * N; ++t) Zs[i][t] = Cs[i][t];
+        for (size_t t = 0; t < (size_t)T * n; ++t) Es[i][t] = 0;
+        for (size_t t = 0; t < (size_t)n * N; ++t) Fs[i][t] = 0;
+    }
+    long long masked = 0;
+    std::vector<int> R;
+    std::vector<u64> e, f(N);
+    for (int c = 0; c < n; ++c) {
+        R.clear();
+        for (int r = 0; r < T; ++r)
+            if (S[(size_t)r * n + c] != 0) R.push_back(r);         // line 3: R_j
+        if (R.empty()) continue;                                    // not a nonzero column
+        const int j = I[c];
+        masked += (long long)R.size();
+        e.assign(R.size(), 0);
+        for (int i = 0; i < 2; ++i) {
+            for (size_t k = 0; k < R.size(); ++k)                   // lines 7-8 + masking of x''
+                Es[i][(size_t)R[k] * n + c] = Xs[i][(size_t)R[k] * n + c] - As[i][(size_t)R[k] * n + c];
+            for (int q = 0; q < N; ++q)                             // line 9 + masking of y
+                Fs[i][(size_t)c * N + q] = Ys[i][(size_t)j * N + q] - Bs[i][(size_t)c * N + q];
+        }
+        for (size_t k = 0; k < R.size(); ++k) e[k] = E0[(size_t)R[k] * n + c] + E1[(size_t)R[k] * n + c];
+        for (int q = 0; q < N; ++q) f[q] = F0[(size_t)c * N + q] + F1[(size_t)c * N + q];
+        for (int i = 0; i < 2; ++i)                                 // line 10 and the sum of line 12
+            for (size_t k = 0; k < R.size(); ++k) {
+                const u64 a = As[i][(size_t)R[k] * n + c];
+                for (int q = 0; q < N; ++q) {
+                    const u64 b = Bs[i][(size_t)c * N + q];
+                    Zs[i][(size_t)R[k] * N + q] += e[k] * b + a * f[q] + (u64)i * (e[k] * f[q]);
+                }
+            }
+    }
+    return masked;
 }
 
 // ---------------------------------------------------------------------------

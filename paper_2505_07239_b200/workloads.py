@@ -283,6 +283,35 @@ def dealer_triple(seed: int, stream: str, rows: int, inner: int, cols: int, vali
     return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1)}
 
 
+def token_block_masks(seed: int, stream: str, tokens: int, n_blocks: int, p_token: float) -> np.ndarray:
+    """Per-token 0/1 masks over `n_blocks` active blocks, each entry Bernoulli(p_token), repaired so that every
+    block keeps at least one token (the block mask is the union of the token masks) and every token at least one
+    block.  uint8 [tokens, n_blocks]."""
+    u = random_unit(seed, stream, tokens * n_blocks).reshape(tokens, n_blocks)
+    m = (np.abs(u) < p_token).astype(np.uint8)
+    pick_t = random_u64(seed, stream + "/fix_t", n_blocks) % np.uint64(tokens)
+    pick_b = random_u64(seed, stream + "/fix_b", tokens) % np.uint64(max(1, n_blocks))
+    for b in np.nonzero(m.sum(axis=0) == 0)[0]:
+        m[int(pick_t[b]), b] = 1
+    for t in np.nonzero(m.sum(axis=1) == 0)[0]:
+        m[t, int(pick_b[t])] = 1
+    return m
+
+
+def dealer_triple_rowsets(seed: int, stream: str, S: np.ndarray, cols: int) -> dict:
+    """Triple of a SIMM product whose left operand has the sparsity distribution S [rows, inner]: A' and B' uniform,
+    C' = (S * A') B' (only the entries of A' on the support take part), each split into two uniform shares.  The A'
+    shares are left uniformly random OFF the support too: whoever uses them has to ignore those words."""
+    rows, inner = S.shape
+    A = random_u64(seed, stream + "/A", rows * inner).reshape(rows, inner)
+    B = random_u64(seed, stream + "/B", inner * cols).reshape(inner, cols)
+    A0, A1 = split_shares(A, seed, stream + "/A")
+    B0, B1 = split_shares(B, seed, stream + "/B")
+    C = ring_matmul(np.where(S != 0, A, U64(0)), B)
+    C0, C1 = split_shares(C, seed, stream + "/C")
+    return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1)}
+
+
 def dealer_triple_elementwise(seed: int, stream: str, shape) -> dict:
     """Element-wise Beaver triple: a, b uniform, c = a * b mod 2^64 element by element, each split into two
     uniform shares.  Returns {"a": (a, a0, a1), "b": ..., "c": ...}."""
