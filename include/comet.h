@@ -166,6 +166,27 @@ int comet_set_mask(comet_ctx* ctx, const uint8_t* block_mask, int location, int3
  * nothing. */
 int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
 
+/* Protocol 3 (SIMM) in general, lines 1-5: the sparsity distribution of the hidden
+ * state may differ from token to token.  `token_mask` is [tokens, n_active_blocks]
+ * bytes, row-major; byte (t, b) non-zero means that the neurons of the b-th ACTIVE
+ * block (in the ascending order of comet_get_index) are non-zeros of token t, so
+ * R_j = {t : token_mask[t, block(j)] != 0}.  It refines the block mask of
+ * comet_set_mask (which must precede it and should be the union of the token
+ * masks) and applies to the comet_ffn_down calls that follow, until the next
+ * comet_set_mask or until it is cleared with token_mask = NULL, tokens = 0,
+ * n_active_blocks = 0.  Under a token mask comet_ffn_down opens only the
+ * non-zero entries (E'_i is zero elsewhere: those words are not part of the
+ * message) and ignores whatever COMET_H and COMET_A_DN hold off the support;
+ * the dealer's C' is sum_j a_j b_j^T scattered to the rows R_j, i.e.
+ * (mask * A') B'.  The products themselves are still evaluated densely over
+ * [tokens, n] on the tensor cores: communication is Theorem 2's minimum, the
+ * multiply count is not.  *masked_out (may be NULL) receives the number of
+ * non-zero entries (neurons, summed over tokens); one 8-byte device-to-host
+ * report and a stream synchronise.  Errors: STATE (no block mask yet), SHAPE
+ * (tokens out of range, n_active_blocks not the current count), INVALID_ARG. */
+int comet_set_token_mask(comet_ctx* ctx, const uint8_t* token_mask, int location, int32_t tokens,
+                         int32_t n_active_blocks, int64_t* masked_out);
+
 /* Protocol 3 (SIMM) with R_j = all tokens for every active column j, so that
  * Merge&Sum of the per-column products is one matmul with inner size n:
  * E'_i = H_i - A'_i, F'_i = W2_i[I, :] - B'_i, Y_i = C'_i + E' B'_i + A'_i F' +

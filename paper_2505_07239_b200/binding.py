@@ -30,7 +30,7 @@ EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
-    "comet_beaver_mul",
+    "comet_beaver_mul", "comet_set_token_mask",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -72,6 +72,7 @@ def _load():
     lib.comet_destroy.restype = None
     lib.comet_load_shares.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64, i64]
     lib.comet_set_mask.argtypes = [vp, vp, ctypes.c_int, i32, ctypes.POINTER(i32)]
+    lib.comet_set_token_mask.argtypes = [vp, vp, ctypes.c_int, i32, i32, ctypes.POINTER(i64)]
     lib.comet_ffn_up.argtypes = [vp, i32]
     lib.comet_ffn_down.argtypes = [vp, i32]
     lib.comet_truncate.argtypes = [vp, ctypes.c_int]
@@ -162,6 +163,24 @@ class Comet:
         self._check(_lib.comet_set_mask(self._h, ptr, loc, nb, ctypes.byref(n)), "comet_set_mask")
         self.n_active = n.value
         return n.value
+
+    def set_token_mask(self, mask) -> int:
+        """Per-token mask over the active blocks, [tokens, n_active_blocks] uint8 (numpy or torch), or None to
+        clear it.  Returns the number of non-zero entries of the hidden state under it."""
+        masked = ctypes.c_int64(0)
+        if mask is None:
+            self._check(_lib.comet_set_token_mask(self._h, None, DEVICE, 0, 0, ctypes.byref(masked)),
+                        "comet_set_token_mask")
+            return 0
+        if isinstance(mask, np.ndarray):
+            assert mask.dtype == np.uint8 and mask.flags["C_CONTIGUOUS"] and mask.ndim == 2
+            ptr, loc = mask.ctypes.data, HOST
+        else:
+            assert mask.dtype == torch.uint8 and mask.is_contiguous() and mask.dim() == 2
+            ptr, loc = mask.data_ptr(), (DEVICE if mask.is_cuda else HOST)
+        self._check(_lib.comet_set_token_mask(self._h, ptr, loc, mask.shape[0], mask.shape[1], ctypes.byref(masked)),
+                    "comet_set_token_mask")
+        return masked.value
 
     def ffn_up(self, tokens: int):
         self._check(_lib.comet_ffn_up(self._h, tokens), "comet_ffn_up")

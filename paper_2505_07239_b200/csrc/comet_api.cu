@@ -43,6 +43,12 @@ struct comet_ctx {
     bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
     bool dn_right_few;                // ... and were laid out for the few-token kernel (128-row tiles)
     uint8_t* d_mask;
+    uint8_t* d_tmask;             // per-token mask over the active blocks, [cap_T, d_ff / block] capacity
+    bool tmask_set;
+    int32_t tmask_tokens;
+    int64_t tmask_masked;         // non-zero entries of the hidden state under the token mask (neurons, not blocks)
+    long long* h_masked;          // pinned and mapped: the count reported by count_mask_kernel
+    long long* h_masked_dev;
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
     int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
@@ -204,6 +210,8 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.kblocks = kb;
     a.down = pr.down ? 1 : 0;
     a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
+    a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
+    a.tmask_ld = c->n_active_blocks;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
@@ -232,6 +240,9 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
     a.M = pr.M; a.N = pr.N; a.K = pr.K; a.kblocks = kb;
     a.left_tile_rows = limb_few(pr) ? comet::limb_few::BT : lb::BM;
     a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
+    a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
+    a.tmask_ld = c->n_active_blocks;
+    a.bs = c->cfg.block;
     a.left_tiles = left ? kb * ceil_div(pr.M, lb::PREP_ROWS) : 0;
     a.right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
@@ -297,6 +308,9 @@ int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA,
         a.Z[p] = c->buf[p][idZ];
     }
     a.M = M; a.N = N; a.K = K;
+    a.tmask = (idZ == COMET_Y && c->tmask_set) ? c->d_tmask : nullptr;
+    a.tmask_ld = c->n_active_blocks;
+    a.bs = c->cfg.block;
     dim3 grid((N + comet::simt::BN - 1) / comet::simt::BN, (M + comet::simt::BM - 1) / comet::simt::BM, 2);
     PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
     comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, c->stream>>>(a);
@@ -411,6 +425,9 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     }
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_tmask, (size_t)nb * (size_t)c->cap_T) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_masked, sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostGetDevicePointer((void**)&c->h_masked_dev, c->h_masked, 0) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_ids, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_count, 2 * sizeof(int32_t)) == cudaSuccess;   // {count, error flag}
     ok = ok && cudaMemset(c->d_count, 0, 2 * sizeof(int32_t)) == cudaSuccess;
@@ -444,6 +461,8 @@ void comet_destroy(comet_ctx* c) {
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
     if (c->d_mask) cudaFree(c->d_mask);
+    if (c->d_tmask) cudaFree(c->d_tmask);
+    if (c->h_masked) cudaFreeHost(c->h_masked);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
     if (c->h_count) cudaFreeHost(c->h_count);
@@ -519,12 +538,40 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     c->n_active_blocks = blocks;
     c->n_active = (int32_t)n;
     c->mask_set = true;
+    c->tmask_set = false;             // a token mask refines one block mask
     c->up_done = c->down_done = false;
     for (int p = 0; p < 2; ++p)
         for (int id = COMET_A_UP; id <= COMET_C_DN; ++id) c->loaded[p][id] = false;
     c->stats.n_active = c->n_active;
     c->stats.n_active_blocks = blocks;
     *n_active_out = c->n_active;
+    return COMET_OK;
+}
+
+int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, int32_t tokens,
+                         int32_t n_active_blocks, int64_t* masked_out) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    if (!c->mask_set) return COMET_ERR_STATE;
+    if (!token_mask) {                         // back to "every token uses every active neuron"
+        if (tokens != 0 || n_active_blocks != 0) return COMET_ERR_INVALID_ARG;
+        c->tmask_set = false;
+        if (masked_out) *masked_out = 0;
+        return COMET_OK;
+    }
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (tokens < 1 || tokens > c->cap_T || n_active_blocks != c->n_active_blocks || n_active_blocks < 1)
+        return COMET_ERR_SHAPE;
+    if ((int64_t)tokens * c->n_active < 0 || (int64_t)tokens * c->n_active > 0x7fffffffll) return COMET_ERR_SHAPE;
+    const size_t bytes = (size_t)tokens * (size_t)n_active_blocks;
+    COMET_CUDA(c, cudaMemcpyAsync(c->d_tmask, token_mask, bytes, copy_kind(location, true), c->stream));
+    comet::count_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, (long long)bytes, c->h_masked_dev);
+    c->stats.kernel_launches += 1;
+    COMET_CUDA(c, cudaGetLastError());
+    COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+    c->tmask_masked = (int64_t)*c->h_masked * c->cfg.block;
+    c->tmask_tokens = tokens;
+    c->tmask_set = true;
+    if (masked_out) *masked_out = c->tmask_masked;
     return COMET_OK;
 }
 
@@ -593,7 +640,8 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
     const int64_t pairs = (int64_t)tokens * d / 2;
     {
         PhaseTimer timer(c, COMET_PHASE_OPEN, 2);
-        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(X, A, E, pairs);
+        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(X, A, E, pairs, nullptr,
+                                                                                              0, d, bs);
         int rows_grid = g * n < c->sm_count * 8 ? g * n : c->sm_count * 8;
         comet::open_weight_rows_kernel<<<dim3(rows_grid, 2), 256, 0, c->stream>>>(W0, W1, B, F, c->d_ids, n, g, bs,
                                                                                    d);
@@ -614,8 +662,10 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
         if (n > 0 && (!c->loaded[p][COMET_H] || !c->loaded[p][COMET_A_DN] || !c->loaded[p][COMET_B_DN]))
             return COMET_ERR_STATE;
     }
+    if (c->tmask_set && c->tmask_tokens != tokens) return COMET_ERR_SHAPE;   // the token mask was given for another T
     c->stats.tokens = tokens;
-    c->stats.message_bytes = 2ll * 8 * ((int64_t)tokens * n + (int64_t)n * d);
+    // with a token mask only the non-zero entries of the hidden state are opened (Theorem 2's communication)
+    c->stats.message_bytes = 2ll * 8 * ((c->tmask_set ? c->tmask_masked : (int64_t)tokens * n) + (int64_t)n * d);
     c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)n * d;
     c->down_tokens = tokens;
     c->down_done = true;
@@ -659,7 +709,8 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
     const int64_t pairs = (int64_t)tokens * n / 2;
     {
         PhaseTimer timer(c, COMET_PHASE_OPEN, 2);
-        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(H, A, E, pairs);
+        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
+            H, A, E, pairs, c->tmask_set ? c->d_tmask : nullptr, c->n_active_blocks, n, bs);
         const int64_t wpairs = (int64_t)d * n / 2;
         comet::open_weight_strips_kernel<<<dim3(ew_grid(c, wpairs, 256), 2), 256, 0, c->stream>>>(
             W, B, F, c->d_ids, n, bs, d, D);
@@ -832,9 +883,10 @@ extern "C" int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* con
         args.Z[p] = reinterpret_cast<u64*>(Z[p]);
     }
     args.M = T; args.N = N; args.K = K;
+    args.tmask = nullptr; args.tmask_ld = 0; args.bs = 1;
     auto blocks = [](int64_t pairs) { return (unsigned)((pairs + 255) / 256 < 1184 ? (pairs + 255) / 256 : 1184); };
-    comet::open_activation_kernel<<<dim3(blocks(left / 2), 2), 256, 0, stream>>>(x, a, e, left / 2);
-    comet::open_activation_kernel<<<dim3(blocks(right / 2), 2), 256, 0, stream>>>(y, b, f, right / 2);
+    comet::open_activation_kernel<<<dim3(blocks(left / 2), 2), 256, 0, stream>>>(x, a, e, left / 2, nullptr, 0, K, 1);
+    comet::open_activation_kernel<<<dim3(blocks(right / 2), 2), 256, 0, stream>>>(y, b, f, right / 2, nullptr, 0, K, 1);
     dim3 grid((N + comet::simt::BN - 1) / comet::simt::BN, (T + comet::simt::BM - 1) / comet::simt::BM, 2);
     comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, stream>>>(args);
     if (cudaGetLastError() != cudaSuccess) return COMET_ERR_CUDA;

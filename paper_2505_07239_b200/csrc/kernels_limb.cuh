@@ -124,6 +124,10 @@ struct LimbOpenArgs {
     int ldw;                 // words per row of W
     int kblocks, down;
     int right_tile_rows;     // rows per plane tile of the right operand: 64, or 128 for the few-token kernel
+    // Protocol 3 with per-column row sets: per-token mask over the active blocks, [rows of X, tmask_ld] bytes, or
+    // null.  Where it is zero the entry of X is no non-zero: it is not opened and E_i is zero there.
+    const uint8_t* tmask;
+    int tmask_ld;
 };
 
 __global__ void __launch_bounds__(256)
@@ -137,6 +141,13 @@ limb_open_kernel(LimbOpenArgs a) {
         ulonglong2* __restrict__ e = reinterpret_cast<ulonglong2*>(party ? a.E[1] : a.E[0]);
         const long long stride = (long long)a.left_blocks * 256;
         for (long long t = (long long)blockIdx.x * 256 + tid; t < a.left_pairs; t += stride) {
+            if (a.tmask) {
+                const unsigned word = (unsigned)(2 * t), row = word / (unsigned)a.K, col = word - row * (unsigned)a.K;
+                if (a.tmask[(size_t)row * a.tmask_ld + col / (unsigned)a.bs] == 0) {
+                    e[t] = make_ulonglong2(0ull, 0ull);
+                    continue;
+                }
+            }
             const ulonglong2 xv = __ldg(x + t), av = __ldg(m + t);
             e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
         }
@@ -206,6 +217,8 @@ struct LimbPrepArgs {
     int N, right_tiles;      // right_tiles = kblocks * ceil(N / 64), or 0
     int K, kblocks;
     int left_tile_rows, right_tile_rows;   // rows per plane tile: 128 / 64, or 32 / 128 for the few-token kernel
+    const uint8_t* tmask;    // per-token mask over the active blocks (see LimbOpenArgs), or null: where it is zero
+    int tmask_ld, bs;        // the party's A_i is no part of the triple and counts as zero
     const u64* C[2];
     u64* Z[2];
     long long copy_pairs;
@@ -251,7 +264,7 @@ limb_prep_kernel(LimbPrepArgs a) {
                 const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(in1 + o));
                 s0 = x.x + y.x;                       // the exchange: both messages summed
                 s1 = x.y + y.y;
-                if (left) {
+                if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + k / a.bs] != 0)) {
                     const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(own + o));
                     w0 = z.x + (party ? s0 : 0ull);   // V_i = A_i + i*E
                     w1 = z.y + (party ? s1 : 0ull);

@@ -68,16 +68,45 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
 // K2: E_i = X_i - A_i  (Section 2.1 "Multiplication": [d]_i = [x]_i - [a]_i).
 // `pairs` = number of 16-byte word pairs per party.
 // ---------------------------------------------------------------------------
+// With `tmask` (per-token mask over the active blocks, [rows, tmask_ld] bytes; Protocol 3 with per-column row
+// sets) an entry whose mask byte is zero is no non-zero of X: it is not opened and E_i is zero there.
 __global__ void __launch_bounds__(256)
-open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs) {
+open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, const uint8_t* __restrict__ tmask,
+                       int tmask_ld, int K, int bs) {
     const int party = blockIdx.y;
     const ulonglong2* __restrict__ x = reinterpret_cast<const ulonglong2*>((party ? X.p[1] : X.p[0]));
     const ulonglong2* __restrict__ a = reinterpret_cast<const ulonglong2*>((party ? A.p[1] : A.p[0]));
     ulonglong2* __restrict__ e = reinterpret_cast<ulonglong2*>((party ? E.p[1] : E.p[0]));
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < pairs; t += stride) {
+        if (tmask) {
+            const unsigned word = (unsigned)(2 * t), row = word / (unsigned)K, col = word - row * (unsigned)K;
+            if (tmask[(size_t)row * tmask_ld + col / (unsigned)bs] == 0) {
+                e[t] = make_ulonglong2(0ull, 0ull);
+                continue;
+            }
+        }
         const ulonglong2 xv = __ldg(x + t), av = __ldg(a + t);
         e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
+    }
+}
+
+// Number of non-zero bytes of a mask, written to `out` (mapped host memory) as a 64-bit count.
+__global__ void __launch_bounds__(1024)
+count_mask_kernel(const uint8_t* __restrict__ mask, long long count, long long* out) {
+    __shared__ long long partial[32];
+    long long mine = 0;
+    for (long long t = threadIdx.x; t < count; t += 1024) mine += mask[t] != 0;
+    for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
+    if ((threadIdx.x & 31) == 0) partial[threadIdx.x >> 5] = mine;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        long long v = partial[threadIdx.x];
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+        if (threadIdx.x == 0) {
+            *out = v;
+            __threadfence_system();
+        }
     }
 }
 

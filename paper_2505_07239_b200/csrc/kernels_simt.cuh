@@ -23,6 +23,10 @@ struct CombineArgs {
     const u64* C[2];   // triple shares, [M, N]
     u64* Z[2];         // result shares, [M, N]
     int M, N, K;       // K multiple of 8, N multiple of 4
+    // Protocol 3 with per-column row sets: per-token mask over the active blocks of the contraction index,
+    // [M, tmask_ld] bytes, or null; where it is zero A_i is no part of the triple and counts as zero.
+    const uint8_t* tmask;
+    int tmask_ld, bs;
 };
 
 namespace simt {
@@ -68,7 +72,8 @@ combine_simt_kernel(CombineArgs a) {
         for (int h = 0; h < 2; ++h) {
             ge0[h] = lok ? ldg2(E0 + loff + k0 + 2 * h) : zero2;
             ge1[h] = lok ? ldg2(E1 + loff + k0 + 2 * h) : zero2;
-            ga[h] = lok ? ldg2(Ai + loff + k0 + 2 * h) : zero2;
+            ga[h] = (lok && (!a.tmask || a.tmask[(size_t)(m0 + lrow) * a.tmask_ld + (k0 + lk + 2 * h) / a.bs] != 0))
+                        ? ldg2(Ai + loff + k0 + 2 * h) : zero2;
         }
         gf0 = rok ? ldg2(F0 + roff + k0) : zero2;
         gf1 = rok ? ldg2(F1 + roff + k0) : zero2;

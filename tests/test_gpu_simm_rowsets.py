@@ -1,0 +1,109 @@
+"""GPU parity of the down-projection under a per-token mask (Protocol 3 with per-column row sets R_j,
+comet_set_token_mask + comet_ffn_down through the C ABI) against the CPU oracle, bit for bit."""
+import ctypes
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+import oracle  # noqa: E402
+from paper_2505_07239_b200 import workloads as wl  # noqa: E402
+
+
+def _run(cfg, seed, tokens, sparsity, p_token, path, clear_after=False):
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    T, d, f = tokens, cfg.d_model, cfg.frac_bits
+    W = wl.model_shares(cfg, seed, plain=False)
+    mask = wl.block_mask(cfg, seed, sparsity)
+    I = oracle.index_set(mask, cfg.block, 1)
+    n, nab = I.size, int(mask.sum())
+    tm = wl.token_block_masks(seed, "tm", T, nab, p_token)
+    S = np.repeat(tm, cfg.block, axis=1)                       # element-level distribution over the compact columns
+    _, H0, H1 = wl.hidden_shares(cfg, seed, n, tokens=T)       # uniform words everywhere, also off the support
+    tri = wl.dealer_triple_rowsets(seed, "down", S, d)
+
+    ctx = hz.make_context(cfg, T, path)
+    hz.load_weights(ctx, cfg, W)
+    assert ctx.set_mask(mask) == n
+    masked = ctx.set_token_mask(tm)
+    assert masked == int(S.sum())
+    for p, Hs in ((0, H0), (1, H1)):
+        ctx.load_shares(p, cb.H, cb.to_device(Hs))
+    hz.load_triple_down(ctx, tri)
+    ctx.ffn_down(T)
+    st = ctx.stats()
+    assert st.matmul_path == path
+    assert st.message_bytes == 2 * 8 * (masked + n * d)        # only the non-zeros of the hidden state are sent
+    ref = oracle.simm_rowsets((H0, H1), W["W2"][1:], I, S, tri["A"][1:], tri["B"][1:], tri["C"][1:])
+    assert ref["masked"] == masked
+    bad = 0
+    for p in (0, 1):
+        bad += int((ctx.get(p, cb.E_DN, (T, n)) != ref["E"][p]).sum())
+        bad += int((ctx.get(p, cb.F_DN, (d, n)).T != ref["F"][p]).sum())
+        bad += int((ctx.get(p, cb.Y, (T, d)) != ref["Z"][p]).sum())
+    ctx.truncate(cb.Y)
+    for p in (0, 1):
+        bad += int((ctx.get(p, cb.Y, (T, d)) != oracle.truncate(p, ref["Z"][p], f)).sum())
+    if clear_after:
+        # cleared: the next product is the token-shared one again
+        assert ctx.set_token_mask(None) == 0
+        full = wl.dealer_triple(seed, "down/full", T, n, d, valid=False)
+        for p, Hs in ((0, H0), (1, H1)):
+            ctx.load_shares(p, cb.H, cb.to_device(Hs))
+        hz.load_triple_down(ctx, full)
+        ctx.ffn_down(T)
+        ref2 = oracle.simm((H0, H1), W["W2"][1:], I, full["A"][1:], full["B"][1:], full["C"][1:])
+        for p in (0, 1):
+            bad += int((ctx.get(p, cb.Y, (T, d)) != ref2["Z"][p]).sum())
+            bad += int((ctx.get(p, cb.E_DN, (T, n)) != ref2["E"][p]).sum())
+    ctx.close()
+    return bad
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("tokens", [16, 40, 130])          # few-token kernel, one ragged tile, two tiles
+def test_token_masked_down_projection_small(path, tokens):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-small", tokens, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    assert _run(cfg, 61 + tokens, tokens, 0.5, 0.3, path, clear_after=True) == 0
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_token_masked_down_projection_opt125m(path):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    assert _run(wl.CONFIGS["opt125m"], 71, 128, None, 0.25, path) == 0
+
+
+def test_token_masked_down_projection_llama_shape_blocks_of_64():
+    """Config 4's structure: 64-neuron blocks, block mask = union of sparse per-token masks."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-b64", 96, 256, 2048, 64, 16, True, 0.25, "uniform", "normal", "normal0.02")
+    assert _run(cfg, 73, 96, 0.75, 0.05, 2) == 0
+
+
+def test_token_mask_errors():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    cfg = wl.CONFIGS["tiny"]
+    ctx = hz.make_context(cfg, cfg.tokens)
+    lib, h = cb.library(), ctx._h
+    m = torch.ones((cfg.tokens, 3), dtype=torch.uint8, device="cuda")
+    out = ctypes.c_int64(0)
+    assert lib.comet_set_token_mask(h, m.data_ptr(), 0, cfg.tokens, 3, ctypes.byref(out)) == -3     # no block mask yet
+    assert ctx.set_mask(wl.block_mask(cfg, 1)) == 96
+    assert lib.comet_set_token_mask(h, m.data_ptr(), 0, cfg.tokens, 4, ctypes.byref(out)) == -2     # 3 active blocks
+    assert lib.comet_set_token_mask(h, m.data_ptr(), 0, cfg.tokens + 1, 3, ctypes.byref(out)) == -2
+    assert lib.comet_set_token_mask(h, None, 0, 5, 3, ctypes.byref(out)) == -1
+    assert lib.comet_set_token_mask(h, m.data_ptr(), 0, cfg.tokens, 3, ctypes.byref(out)) == 0
+    assert out.value == cfg.tokens * 96
+    ctx.close()
