@@ -173,6 +173,39 @@ def simm(X, Y, I, A, B, C):
     return {"E": (E0, E1), "F": (F0, F1), "Z": (Z0, Z1)}
 
 
+def components_dfs(S):
+    """Connected components of the bipartite graph of S [T, n] (Protocol 2 line 1).
+    Returns (row_comp [T], col_comp [n], L); -1 marks a node without an edge."""
+    S = np.ascontiguousarray(S, dtype=np.uint8)
+    T, n = S.shape
+    rc, cc = np.empty(T, np.int32), np.empty(n, np.int32)
+    L = lib().orc_components_dfs(ctypes.c_int(T), ctypes.c_int(n), _p(S), _p(rc), _p(cc))
+    return rc, cc, int(L)
+
+
+def somm_components(X, Y, I, S, A, B, C):
+    """Protocol 2 over the connected components of S [T, n].  Y pair is [K, Dy]; I maps compact columns to
+    columns of Y; A [T,K], B [K,n], C [T,n] hold the per-component triples stacked.  Returns compact E [T,K],
+    F [K,n], Z [T,n] (zero outside the component blocks), the partition and the cost counters."""
+    X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1 = _pairs(X, Y, A, B, C)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    S = np.ascontiguousarray(S, dtype=np.uint8)
+    T, K = X0.shape
+    _, Dy = Y0.shape
+    n = I.size
+    assert S.shape == (T, n) and A0.shape == (T, K) and B0.shape == (K, n) and C0.shape == (T, n)
+    E0, E1 = np.empty((T, K), U64), np.empty((T, K), U64)
+    F0, F1 = np.empty((K, n), U64), np.empty((K, n), U64)
+    R0, R1 = np.empty((T, n), U64), np.empty((T, n), U64)
+    rc, cc = np.empty(T, np.int32), np.empty(n, np.int32)
+    cost = np.zeros(2, np.int64)
+    L = lib().orc_somm_components(ctypes.c_int(T), ctypes.c_int(K), ctypes.c_int(Dy), _p(I), ctypes.c_int(n), _p(S),
+                                  *[_p(a) for a in (X0, X1, Y0, Y1, A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, R0, R1)],
+                                  _p(rc), _p(cc), _p(cost))
+    return {"E": (E0, E1), "F": (F0, F1), "Z": (R0, R1), "row_comp": rc, "col_comp": cc, "L": int(L),
+            "masked_nodes": int(cost[0]), "dot_products": int(cost[1])}
+
+
 def simm_rowsets(X, Y, I, S, A, B, C):
     """Protocol 3 with per-column row sets: S is the [T, n] sparsity distribution of the compact X
     (non-zero = present).  Returns E [T,n] (zero off the support), F [n,N], Z [T,N] and the number of

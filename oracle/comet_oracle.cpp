@@ -17,6 +17,10 @@
 // closed forms and the {0,1}-ulp invariant; hand-computed fixtures.
 // Parity unpinned: the individual share values Z_i (as opposed to their sum)
 // are fixed only by Eq. 1 itself plus this repository's seeded inputs.
+// SOMM over connected components (Protocol 2 in general): the partition is
+// pinned by a library routine for connected components and by hand-made graphs,
+// the result by the plaintext product on the component blocks, the costs by the
+// counts of Theorem 1, and the whole by its reduction to the token-shared case.
 // SIMM with per-column row sets R_j (Protocol 3 in general): pinned by the masked
 // plaintext product, by its reduction to the token-shared case under an
 // all-ones distribution, and by the counts of Theorem 2.
@@ -167,6 +171,127 @@ void orc_somm(int T, int K, int Dy, const int32_t* I, int n,
     orc_index_cols(Y1, K, Dy, I, n, Yt1.data());
     orc_pi_matmul(T, K, n, X0, X1, Yt0.data(), Yt1.data(), // line 6
                   A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, R0, R1);
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 2 line 1: the connected components {G_t} of the bipartite graph whose
+// nodes are the T rows of X and the n (compact) columns of Y and whose edges are
+// the non-zeros of the sparsity distribution S [T, n], found by depth-first
+// search.  Components are numbered in the order in which a scan over the rows
+// 0, 1, ... discovers them; row_comp / col_comp give each node's component, -1
+// for a node without any edge.  Returns the number of components L.
+// ---------------------------------------------------------------------------
+int orc_components_dfs(int T, int n, const uint8_t* S, int32_t* row_comp, int32_t* col_comp) {
+    for (int r = 0; r < T; ++r) row_comp[r] = -1;
+    for (int c = 0; c < n; ++c) col_comp[c] = -1;
+    int L = 0;
+    std::vector<int> stack;                       // node ids: rows 0..T-1, columns T..T+n-1
+    for (int start = 0; start < T; ++start) {
+        if (row_comp[start] >= 0) continue;
+        bool has_edge = false;
+        for (int c = 0; c < n && !has_edge; ++c) has_edge = S[(size_t)start * n + c] != 0;
+        if (!has_edge) continue;
+        row_comp[start] = L;
+        stack.assign(1, start);
+        while (!stack.empty()) {
+            const int node = stack.back();
+            stack.pop_back();
+            if (node < T) {
+                for (int c = 0; c < n; ++c)
+                    if (S[(size_t)node * n + c] != 0 && col_comp[c] < 0) {
+                        col_comp[c] = L;
+                        stack.push_back(T + c);
+                    }
+            } else {
+                const int c = node - T;
+                for (int r = 0; r < T; ++r)
+                    if (S[(size_t)r * n + c] != 0 && row_comp[r] < 0) {
+                        row_comp[r] = L;
+                        stack.push_back(r);
+                    }
+            }
+        }
+        ++L;
+    }
+    return L;
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 2 (SOMM) in general.  Y is [K, Dy]; compact column c stands for
+// column I[c] of Y; S is the sparsity distribution of the compact result [T, n].
+// For every component: I_x, I_y (line 3), IndexRows / IndexCols (lines 4-5),
+// Pi_MatMul with that component's own triple (line 6), and Merge (line 8) puts
+// the result block at (I_x, I_y); every other entry of the result is zero in
+// both shares, and rows / columns outside all components are neither masked nor
+// sent (their message rows stay zero).  The per-component triples arrive
+// stacked: A [T, K] holds in row r the mask row of r's component, B [K, n] in
+// column c that of c's component, C [T, n] the blocks c^t = a^t b^t at (I_x, I_y)
+// (whatever else C holds is ignored).
+// cost[0] = rows and columns masked (Theorem 1's communication count, in rows /
+// columns), cost[1] = dot products evaluated, sum_t |I_x||I_y|.
+// Returns L.
+// ---------------------------------------------------------------------------
+int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uint8_t* S,
+                        const u64* X0, const u64* X1, const u64* Y0, const u64* Y1,
+                        const u64* A0, const u64* A1, const u64* B0, const u64* B1,
+                        const u64* C0, const u64* C1,
+                        u64* E0, u64* E1, u64* F0, u64* F1, u64* R0, u64* R1,
+                        int32_t* row_comp, int32_t* col_comp, long long* cost) {
+    const int L = orc_components_dfs(T, n, S, row_comp, col_comp);            // line 1
+    const u64* Xs[2] = {X0, X1};
+    const u64* Ys[2] = {Y0, Y1};
+    const u64* As[2] = {A0, A1};
+    const u64* Bs[2] = {B0, B1};
+    const u64* Cs[2] = {C0, C1};
+    u64* Es[2] = {E0, E1};
+    u64* Fs[2] = {F0, F1};
+    u64* Rs[2] = {R0, R1};
+    for (int i = 0; i < 2; ++i) {
+        for (size_t t = 0; t < (size_t)T * K; ++t) Es[i][t] = 0;
+        for (size_t t = 0; t < (size_t)K * n; ++t) Fs[i][t] = 0;
+        for (size_t t = 0; t < (size_t)T * n; ++t) Rs[i][t] = 0;
+    }
+    cost[0] = cost[1] = 0;
+    std::vector<int> Ix, Iy;
+    for (int t = 0; t < L; ++t) {
+        Ix.clear();
+        Iy.clear();
+        for (int r = 0; r < T; ++r) if (row_comp[r] == t) Ix.push_back(r);    // line 3
+        for (int c = 0; c < n; ++c) if (col_comp[c] == t) Iy.push_back(c);
+        const int tx = (int)Ix.size(), ty = (int)Iy.size();
+        cost[0] += tx + ty;
+        cost[1] += (long long)tx * ty;
+        std::vector<u64> xt[2], yt[2], at[2], bt[2], ct[2], et[2], ft[2], rt[2];
+        for (int i = 0; i < 2; ++i) {
+            xt[i].resize((size_t)tx * K); at[i].resize((size_t)tx * K); et[i].resize((size_t)tx * K);
+            yt[i].resize((size_t)K * ty); bt[i].resize((size_t)K * ty); ft[i].resize((size_t)K * ty);
+            ct[i].resize((size_t)tx * ty); rt[i].resize((size_t)tx * ty);
+            for (int a = 0; a < tx; ++a)                                     // line 4: IndexRows
+                for (int k = 0; k < K; ++k) {
+                    xt[i][(size_t)a * K + k] = Xs[i][(size_t)Ix[a] * K + k];
+                    at[i][(size_t)a * K + k] = As[i][(size_t)Ix[a] * K + k];
+                }
+            for (int k = 0; k < K; ++k)                                      // line 5: IndexCols
+                for (int b = 0; b < ty; ++b) {
+                    yt[i][(size_t)k * ty + b] = Ys[i][(size_t)k * Dy + I[Iy[b]]];
+                    bt[i][(size_t)k * ty + b] = Bs[i][(size_t)k * n + Iy[b]];
+                }
+            for (int a = 0; a < tx; ++a)
+                for (int b = 0; b < ty; ++b) ct[i][(size_t)a * ty + b] = Cs[i][(size_t)Ix[a] * n + Iy[b]];
+        }
+        orc_pi_matmul(tx, K, ty, xt[0].data(), xt[1].data(), yt[0].data(), yt[1].data(),             // line 6
+                      at[0].data(), at[1].data(), bt[0].data(), bt[1].data(), ct[0].data(), ct[1].data(),
+                      et[0].data(), et[1].data(), ft[0].data(), ft[1].data(), rt[0].data(), rt[1].data());
+        for (int i = 0; i < 2; ++i) {                                        // line 8: Merge
+            for (int a = 0; a < tx; ++a)
+                for (int k = 0; k < K; ++k) Es[i][(size_t)Ix[a] * K + k] = et[i][(size_t)a * K + k];
+            for (int k = 0; k < K; ++k)
+                for (int b = 0; b < ty; ++b) Fs[i][(size_t)k * n + Iy[b]] = ft[i][(size_t)k * ty + b];
+            for (int a = 0; a < tx; ++a)
+                for (int b = 0; b < ty; ++b) Rs[i][(size_t)Ix[a] * n + Iy[b]] = rt[i][(size_t)a * ty + b];
+        }
+    }
+    return L;
 }
 
 // ---------------------------------------------------------------------------

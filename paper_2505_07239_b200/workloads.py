@@ -298,6 +298,40 @@ def token_block_masks(seed: int, stream: str, tokens: int, n_blocks: int, p_toke
     return m
 
 
+def bipartite_components(S: np.ndarray):
+    """Connected components of the bipartite graph rows x columns with the non-zeros of S as edges, by a library
+    routine (scipy).  Returns (row_label, col_label) with -1 for nodes without an edge; labels are arbitrary."""
+    from scipy.sparse import coo_matrix
+    from scipy.sparse.csgraph import connected_components
+
+    T, n = S.shape
+    r, c = np.nonzero(S)
+    adj = coo_matrix((np.ones(r.size, np.int8), (r, T + c)), shape=(T + n, T + n))
+    _, lab = connected_components(adj, directed=False)
+    row, col = lab[:T].astype(np.int64), lab[T:].astype(np.int64)
+    row[~(S != 0).any(axis=1)] = -1
+    col[~(S != 0).any(axis=0)] = -1
+    return row, col
+
+
+def dealer_triple_components(seed: int, stream: str, S: np.ndarray, inner: int) -> dict:
+    """Stacked per-component triples of a SOMM product with result distribution S [rows, cols]: A [rows, inner] and
+    B [inner, cols] uniform (row r / column c carry the mask of their component's triple), C = A B on the component
+    blocks.  The C shares are uniformly random OFF the blocks: whoever uses them has to ignore those words."""
+    rows, cols = S.shape
+    A = random_u64(seed, stream + "/A", rows * inner).reshape(rows, inner)
+    B = random_u64(seed, stream + "/B", inner * cols).reshape(inner, cols)
+    A0, A1 = split_shares(A, seed, stream + "/A")
+    B0, B1 = split_shares(B, seed, stream + "/B")
+    rl, cl = bipartite_components(S)
+    same = (rl[:, None] == cl[None, :]) & (rl[:, None] >= 0)
+    C = np.where(same, ring_matmul(A, B), U64(0))
+    C0, C1 = split_shares(C, seed, stream + "/C")
+    junk = random_u64(seed, stream + "/C/junk", rows * cols).reshape(rows, cols)
+    C0 = np.where(same, C0, junk)
+    return {"A": (A, A0, A1), "B": (B, B0, B1), "C": (C, C0, C1), "same_component": same}
+
+
 def dealer_triple_rowsets(seed: int, stream: str, S: np.ndarray, cols: int) -> dict:
     """Triple of a SIMM product whose left operand has the sparsity distribution S [rows, inner]: A' and B' uniform,
     C' = (S * A') B' (only the entries of A' on the support take part), each split into two uniform shares.  The A'
