@@ -122,6 +122,8 @@ typedef struct {
        count per phase since profiling was switched on, from CUDA events on the stream */
     double phase_ms[COMET_NUM_PHASES];
     int64_t phase_launches[COMET_NUM_PHASES];
+    int32_t n_components;    /* connected components under the current token mask (0 without one) */
+    int32_t reserved;
 } comet_stats_t;
 
 /* Create a context: validates the configuration, selects the device, and
@@ -166,15 +168,33 @@ int comet_set_mask(comet_ctx* ctx, const uint8_t* block_mask, int location, int3
  * nothing. */
 int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
 
-/* Protocol 3 (SIMM) in general, lines 1-5: the sparsity distribution of the hidden
- * state may differ from token to token.  `token_mask` is [tokens, n_active_blocks]
+/* Protocols 2 and 3 in general: the sparsity distribution may differ from token to
+ * token.  One call sets it for both projections.
+ *
+ * Up-projection, Protocol 2: the connected components of the bipartite graph
+ * (tokens) x (active blocks) are found on the GPU (minimum-label propagation
+ * instead of the paper's depth-first search; the partition is the same), each
+ * token row and each weight column is opened once (rows / blocks without any
+ * edge not at all: their message words are zero), and comet_ffn_up leaves in
+ * COMET_Z_UP the result blocks of the components, with every entry whose token
+ * and block lie in different components zero in both shares (Merge).  The
+ * per-component triples are passed stacked: row r of COMET_A_UP is the mask row
+ * of r's component, row c of COMET_B_UP that of c's, COMET_C_UP holds a^t b^t
+ * on the blocks (its other words are ignored).  The products are evaluated as
+ * ONE dense product over [tokens, g*n] and masked afterwards: communication is
+ * Theorem 1's minimum, the dot-product count is not when there are several
+ * components.
+ *
+ * Down-projection, Protocol 3, lines 1-5: the sparsity distribution of the hidden
+ * state.  `token_mask` is [tokens, n_active_blocks]
  * bytes, row-major; byte (t, b) non-zero means that the neurons of the b-th ACTIVE
  * block (in the ascending order of comet_get_index) are non-zeros of token t, so
  * R_j = {t : token_mask[t, block(j)] != 0}.  It refines the block mask of
  * comet_set_mask (which must precede it and should be the union of the token
  * masks) and applies to the comet_ffn_down calls that follow, until the next
  * comet_set_mask or until it is cleared with token_mask = NULL, tokens = 0,
- * n_active_blocks = 0.  Under a token mask comet_ffn_down opens only the
+ * n_active_blocks = 0; comet_ffn_up and comet_ffn_down must then be called with
+ * the same `tokens`.  Under a token mask comet_ffn_down opens only the
  * non-zero entries (E'_i is zero elsewhere: those words are not part of the
  * message) and ignores whatever COMET_H and COMET_A_DN hold off the support;
  * the dealer's C' is sum_j a_j b_j^T scattered to the rows R_j, i.e.
@@ -186,6 +206,13 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * (tokens out of range, n_active_blocks not the current count), INVALID_ARG. */
 int comet_set_token_mask(comet_ctx* ctx, const uint8_t* token_mask, int location, int32_t tokens,
                          int32_t n_active_blocks, int64_t* masked_out);
+
+/* The partition found by comet_set_token_mask: row_label[t] (tokens entries) and
+ * blk_label[b] (one per active block) hold the smallest token index of the node's
+ * component, -1 for a node without an edge; *n_components_out the number of
+ * components.  Errors: STATE (no token mask), INVALID_ARG. */
+int comet_get_components(comet_ctx* ctx, int32_t* row_label, int32_t* blk_label, int location,
+                         int32_t* n_components_out);
 
 /* Protocol 3 (SIMM) with R_j = all tokens for every active column j, so that
  * Merge&Sum of the per-column products is one matmul with inner size n:

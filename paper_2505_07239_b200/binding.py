@@ -30,7 +30,7 @@ EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
-    "comet_beaver_mul", "comet_set_token_mask",
+    "comet_beaver_mul", "comet_set_token_mask", "comet_get_components",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -47,7 +47,8 @@ class CometStats(ctypes.Structure):
     _fields_ = [("message_bytes", ctypes.c_int64), ("ring_macs", ctypes.c_int64), ("n_active", ctypes.c_int32),
                 ("n_active_blocks", ctypes.c_int32), ("tokens", ctypes.c_int32), ("matmul_path", ctypes.c_int32),
                 ("kernel_launches", ctypes.c_int64), ("phase_ms", ctypes.c_double * 5),
-                ("phase_launches", ctypes.c_int64 * 5)]
+                ("phase_launches", ctypes.c_int64 * 5), ("n_components", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
 class CometError(RuntimeError):
@@ -73,6 +74,7 @@ def _load():
     lib.comet_load_shares.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64, i64]
     lib.comet_set_mask.argtypes = [vp, vp, ctypes.c_int, i32, ctypes.POINTER(i32)]
     lib.comet_set_token_mask.argtypes = [vp, vp, ctypes.c_int, i32, i32, ctypes.POINTER(i64)]
+    lib.comet_get_components.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.POINTER(i32)]
     lib.comet_ffn_up.argtypes = [vp, i32]
     lib.comet_ffn_down.argtypes = [vp, i32]
     lib.comet_truncate.argtypes = [vp, ctypes.c_int]
@@ -181,6 +183,16 @@ class Comet:
         self._check(_lib.comet_set_token_mask(self._h, ptr, loc, mask.shape[0], mask.shape[1], ctypes.byref(masked)),
                     "comet_set_token_mask")
         return masked.value
+
+    def get_components(self, tokens: int, n_active_blocks: int):
+        """(row_label [tokens], blk_label [n_active_blocks], number of components) under the current token mask."""
+        rl = torch.empty(tokens, dtype=torch.int32, device=self.device)
+        bl = torch.empty(n_active_blocks, dtype=torch.int32, device=self.device)
+        cnt = ctypes.c_int32(0)
+        self._check(_lib.comet_get_components(self._h, rl.data_ptr(), bl.data_ptr(), DEVICE, ctypes.byref(cnt)),
+                    "comet_get_components")
+        self.synchronize()
+        return rl.cpu().numpy(), bl.cpu().numpy(), cnt.value
 
     def ffn_up(self, tokens: int):
         self._check(_lib.comet_ffn_up(self._h, tokens), "comet_ffn_up")

@@ -47,8 +47,11 @@ struct comet_ctx {
     bool tmask_set;
     int32_t tmask_tokens;
     int64_t tmask_masked;         // non-zero entries of the hidden state under the token mask (neurons, not blocks)
-    long long* h_masked;          // pinned and mapped: the count reported by count_mask_kernel
+    long long* h_masked;          // pinned and mapped: [0] count_mask_kernel's count, [1..3] token_components_kernel's report
     long long* h_masked_dev;
+    int32_t* d_row_label;         // component label per token row / per active block under the token mask
+    int32_t* d_blk_label;
+    int32_t n_components, live_rows, live_blocks;
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
     int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
@@ -212,6 +215,8 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
     a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
     a.tmask_ld = c->n_active_blocks;
+    a.row_label = (!pr.down && c->tmask_set) ? c->d_row_label : nullptr;
+    a.blk_label = (!pr.down && c->tmask_set) ? c->d_blk_label : nullptr;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
@@ -316,6 +321,21 @@ int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA,
     comet::combine_simt_kernel<<<grid, comet::simt::THREADS, 0, c->stream>>>(a);
     c->stats.kernel_launches += 1;
     c->stats.matmul_path = COMET_PATH_SIMT;
+    COMET_CUDA(c, cudaGetLastError());
+    return COMET_OK;
+}
+
+// Protocol 2 line 8 under a token mask: entries of the compact result outside the component blocks become zero.
+int somm_merge(comet_ctx* c, int tokens) {
+    if (!c->tmask_set) return COMET_OK;
+    const int cols = c->groups * c->n_active;
+    const int64_t pairs = (int64_t)tokens * cols / 2;
+    if (pairs == 0) return COMET_OK;
+    comet::PartyOut Z;
+    for (int p = 0; p < 2; ++p) Z.p[p] = c->buf[p][COMET_Z_UP];
+    comet::somm_merge_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
+        Z, pairs, cols, c->n_active, c->cfg.block, c->d_row_label, c->d_blk_label);
+    c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
 }
@@ -426,7 +446,9 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_tmask, (size_t)nb * (size_t)c->cap_T) == cudaSuccess;
-    ok = ok && cudaHostAlloc((void**)&c->h_masked, sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_masked, 4 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_row_label, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_blk_label, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaHostGetDevicePointer((void**)&c->h_masked_dev, c->h_masked, 0) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_ids, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_count, 2 * sizeof(int32_t)) == cudaSuccess;   // {count, error flag}
@@ -463,6 +485,8 @@ void comet_destroy(comet_ctx* c) {
     if (c->d_mask) cudaFree(c->d_mask);
     if (c->d_tmask) cudaFree(c->d_tmask);
     if (c->h_masked) cudaFreeHost(c->h_masked);
+    if (c->d_row_label) cudaFree(c->d_row_label);
+    if (c->d_blk_label) cudaFree(c->d_blk_label);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
     if (c->h_count) cudaFreeHost(c->h_count);
@@ -565,10 +589,17 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     const size_t bytes = (size_t)tokens * (size_t)n_active_blocks;
     COMET_CUDA(c, cudaMemcpyAsync(c->d_tmask, token_mask, bytes, copy_kind(location, true), c->stream));
     comet::count_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, (long long)bytes, c->h_masked_dev);
-    c->stats.kernel_launches += 1;
+    // Protocol 2 line 1: the connected components the up-projection is partitioned into
+    comet::token_components_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, tokens, n_active_blocks, c->d_row_label,
+                                                             c->d_blk_label, c->h_masked_dev + 1);
+    c->stats.kernel_launches += 2;
     COMET_CUDA(c, cudaGetLastError());
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
-    c->tmask_masked = (int64_t)*c->h_masked * c->cfg.block;
+    c->tmask_masked = (int64_t)c->h_masked[0] * c->cfg.block;
+    c->n_components = (int32_t)c->h_masked[1];
+    c->live_rows = (int32_t)c->h_masked[2];
+    c->live_blocks = (int32_t)c->h_masked[3];
+    c->stats.n_components = c->n_components;
     c->tmask_tokens = tokens;
     c->tmask_set = true;
     if (masked_out) *masked_out = c->tmask_masked;
@@ -586,8 +617,12 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
         if (c->groups == 2 && !c->loaded[p][COMET_WG]) return COMET_ERR_STATE;
     }
     const int d = c->cfg.d_model, n = c->n_active, g = c->groups, bs = c->cfg.block;
+    if (c->tmask_set && c->tmask_tokens != tokens) return COMET_ERR_SHAPE;   // the token mask was given for another T
     c->stats.tokens = tokens;
-    c->stats.message_bytes = 2ll * 8 * ((int64_t)tokens * d + (int64_t)d * g * n);
+    // under a token mask only the rows and columns of the connected components are opened (Theorem 1)
+    c->stats.message_bytes = c->tmask_set
+        ? 2ll * 8 * ((int64_t)c->live_rows * d + (int64_t)d * g * c->live_blocks * bs)
+        : 2ll * 8 * ((int64_t)tokens * d + (int64_t)d * g * n);
     c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)d * g * n;
     c->up_tokens = tokens;
     c->up_done = true;
@@ -623,7 +658,9 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
             c->dn_right_ready = true;
             c->dn_right_few = limb_few(dn);
         }
-        return limb_combine(c, up);
+        rc = limb_combine(c, up);
+        if (rc != COMET_OK) return rc;
+        return somm_merge(c, tokens);
     }
 
     comet::PartyPtrs X, A, W0, W1, B;
@@ -640,16 +677,18 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
     const int64_t pairs = (int64_t)tokens * d / 2;
     {
         PhaseTimer timer(c, COMET_PHASE_OPEN, 2);
-        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(X, A, E, pairs, nullptr,
-                                                                                              0, d, bs);
+        comet::open_activation_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
+            X, A, E, pairs, nullptr, 0, d, bs, c->tmask_set ? c->d_row_label : nullptr);
         int rows_grid = g * n < c->sm_count * 8 ? g * n : c->sm_count * 8;
-        comet::open_weight_rows_kernel<<<dim3(rows_grid, 2), 256, 0, c->stream>>>(W0, W1, B, F, c->d_ids, n, g, bs,
-                                                                                   d);
+        comet::open_weight_rows_kernel<<<dim3(rows_grid, 2), 256, 0, c->stream>>>(
+            W0, W1, B, F, c->d_ids, n, g, bs, d, c->tmask_set ? c->d_blk_label : nullptr);
     }
     c->stats.kernel_launches += 2;
     COMET_CUDA(c, cudaGetLastError());
-    return launch_combine(c, tokens, g * n, d, COMET_E_UP, COMET_F_UP, COMET_A_UP, COMET_B_UP, COMET_C_UP,
-                          COMET_Z_UP);
+    const int rc = launch_combine(c, tokens, g * n, d, COMET_E_UP, COMET_F_UP, COMET_A_UP, COMET_B_UP, COMET_C_UP,
+                                  COMET_Z_UP);
+    if (rc != COMET_OK) return rc;
+    return somm_merge(c, tokens);
 }
 
 int comet_ffn_down(comet_ctx* c, int32_t tokens) {
@@ -772,6 +811,19 @@ int comet_get_index(comet_ctx* c, int32_t* out, int location, int32_t capacity, 
         COMET_CUDA(c, cudaMemcpyAsync(out, c->d_ids, (size_t)c->n_active_blocks * sizeof(int32_t),
                                       copy_kind(location, false), c->stream));
     *n_active_blocks_out = c->n_active_blocks;
+    return COMET_OK;
+}
+
+int comet_get_components(comet_ctx* c, int32_t* row_label, int32_t* blk_label, int location,
+                         int32_t* n_components_out) {
+    if (!c || !row_label || !blk_label || !n_components_out) return COMET_ERR_INVALID_ARG;
+    if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (!c->mask_set || !c->tmask_set) return COMET_ERR_STATE;
+    COMET_CUDA(c, cudaMemcpyAsync(row_label, c->d_row_label, (size_t)c->tmask_tokens * sizeof(int32_t),
+                                  copy_kind(location, false), c->stream));
+    COMET_CUDA(c, cudaMemcpyAsync(blk_label, c->d_blk_label, (size_t)c->n_active_blocks * sizeof(int32_t),
+                                  copy_kind(location, false), c->stream));
+    *n_components_out = c->n_components;
     return COMET_OK;
 }
 

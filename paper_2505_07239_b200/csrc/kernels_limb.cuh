@@ -128,6 +128,10 @@ struct LimbOpenArgs {
     // null.  Where it is zero the entry of X is no non-zero: it is not opened and E_i is zero there.
     const uint8_t* tmask;
     int tmask_ld;
+    // Protocol 2 over connected components: component label per row of X and per active block (-1 = in no
+    // component), or null.  A row / column outside every component is not opened: its message words are zero.
+    const int32_t* row_label;
+    const int32_t* blk_label;
 };
 
 __global__ void __launch_bounds__(256)
@@ -147,6 +151,10 @@ limb_open_kernel(LimbOpenArgs a) {
                     e[t] = make_ulonglong2(0ull, 0ull);
                     continue;
                 }
+            }
+            if (a.row_label && a.row_label[(unsigned)(2 * t) / (unsigned)a.K] < 0) {
+                e[t] = make_ulonglong2(0ull, 0ull);
+                continue;
             }
             const ulonglong2 xv = __ldg(x + t), av = __ldg(m + t);
             e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
@@ -171,18 +179,21 @@ limb_open_kernel(LimbOpenArgs a) {
             u64 b0 = 0, b1 = 0;
             if (row < a.rows && k < a.K) {
                 const u64* wsrc;
+                bool dead = false;
                 if (a.down) {
                     wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
                 } else {
                     const int grp = row / a.n, j = row - grp * a.n;
                     const int neuron = a.ids[j / a.bs] * a.bs + (j % a.bs);
+                    dead = a.blk_label && a.blk_label[j / a.bs] < 0;
                     wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0]) : (party ? a.W1[1] : a.W1[0])) +
                            (size_t)neuron * a.ldw + k;
                 }
                 const size_t o = (size_t)row * a.K + k;
                 const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2*>(wsrc));
                 const ulonglong2 b = __ldg(reinterpret_cast<const ulonglong2*>(Bi + o));
-                *reinterpret_cast<ulonglong2*>(Fi + o) = make_ulonglong2(w.x - b.x, w.y - b.y);
+                *reinterpret_cast<ulonglong2*>(Fi + o) = dead ? make_ulonglong2(0ull, 0ull)
+                                                              : make_ulonglong2(w.x - b.x, w.y - b.y);
                 b0 = b.x;
                 b1 = b.y;
             }

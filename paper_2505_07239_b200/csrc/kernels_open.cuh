@@ -72,7 +72,7 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
 // sets) an entry whose mask byte is zero is no non-zero of X: it is not opened and E_i is zero there.
 __global__ void __launch_bounds__(256)
 open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, const uint8_t* __restrict__ tmask,
-                       int tmask_ld, int K, int bs) {
+                       int tmask_ld, int K, int bs, const int32_t* __restrict__ row_label = nullptr) {
     const int party = blockIdx.y;
     const ulonglong2* __restrict__ x = reinterpret_cast<const ulonglong2*>((party ? X.p[1] : X.p[0]));
     const ulonglong2* __restrict__ a = reinterpret_cast<const ulonglong2*>((party ? A.p[1] : A.p[0]));
@@ -86,8 +86,97 @@ open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, cons
                 continue;
             }
         }
+        if (row_label && row_label[(unsigned)(2 * t) / (unsigned)K] < 0) {   // a row outside every component is not opened
+            e[t] = make_ulonglong2(0ull, 0ull);
+            continue;
+        }
         const ulonglong2 xv = __ldg(x + t), av = __ldg(a + t);
         e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Protocol 2 line 1 on the GPU: connected components of the bipartite graph
+// (token rows) x (active blocks) whose edges are the non-zero bytes of the
+// per-token mask S [T, nab].  The paper uses depth-first search; here one CTA
+// propagates minimum labels back and forth (block <- min over its tokens,
+// token <- min over its blocks) until nothing changes, at most T + nab + 1
+// rounds.  Every node of a component ends up with the component's smallest
+// token index as its label; nodes without an edge get -1.
+// report[0] = number of components, [1] = tokens with an edge, [2] = blocks with
+// an edge (mapped host memory).
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+token_components_kernel(const uint8_t* __restrict__ S, int T, int nab, int32_t* row_label, int32_t* blk_label,
+                        long long* report) {
+    __shared__ int changed;
+    __shared__ int counts[3];
+    const int tid = threadIdx.x;
+    const int INF = 0x7fffffff;
+    for (int r = tid; r < T; r += 1024) {
+        bool edge = false;
+        for (int b = 0; b < nab && !edge; ++b) edge = S[(size_t)r * nab + b] != 0;
+        row_label[r] = edge ? r : INF;
+    }
+    for (int b = tid; b < nab; b += 1024) blk_label[b] = INF;
+    if (tid == 0) counts[0] = counts[1] = counts[2] = 0;
+    __syncthreads();
+    for (int round = 0; round <= T + nab; ++round) {
+        if (tid == 0) changed = 0;
+        __syncthreads();
+        for (int b = tid; b < nab; b += 1024) {
+            int best = blk_label[b];
+            for (int r = 0; r < T; ++r)
+                if (S[(size_t)r * nab + b] != 0) best = min(best, row_label[r]);
+            if (best < blk_label[b]) { blk_label[b] = best; changed = 1; }
+        }
+        __syncthreads();
+        for (int r = tid; r < T; r += 1024) {
+            int best = row_label[r];
+            if (best != INF) {
+                for (int b = 0; b < nab; ++b)
+                    if (S[(size_t)r * nab + b] != 0) best = min(best, blk_label[b]);
+                if (best < row_label[r]) { row_label[r] = best; changed = 1; }
+            }
+        }
+        __syncthreads();
+        if (!changed) break;
+        __syncthreads();
+    }
+    for (int r = tid; r < T; r += 1024) {
+        const int l = row_label[r];
+        if (l == INF) row_label[r] = -1;
+        else {
+            atomicAdd(&counts[1], 1);
+            if (l == r) atomicAdd(&counts[0], 1);
+        }
+    }
+    for (int b = tid; b < nab; b += 1024) {
+        if (blk_label[b] == INF) blk_label[b] = -1;
+        else atomicAdd(&counts[2], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        report[0] = counts[0];
+        report[1] = counts[1];
+        report[2] = counts[2];
+        __threadfence_system();
+    }
+}
+
+// Protocol 2 line 8 (Merge) on the compact result [T, cols]: an entry whose token and block are not in the same
+// component is no part of any result block and is zero in both shares.  Compact column c belongs to active block
+// (c mod n) / bs.  `pairs` = 16-byte word pairs per party.
+__global__ void __launch_bounds__(256)
+somm_merge_kernel(PartyOut Z, int64_t pairs, int cols, int n, int bs, const int32_t* __restrict__ row_label,
+                  const int32_t* __restrict__ blk_label) {
+    const int party = blockIdx.y;
+    ulonglong2* __restrict__ z = reinterpret_cast<ulonglong2*>((party ? Z.p[1] : Z.p[0]));
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < pairs; t += stride) {
+        const unsigned word = (unsigned)(2 * t), row = word / (unsigned)cols, col = word - row * (unsigned)cols;
+        const int rl = row_label[row];
+        if (rl < 0 || rl != blk_label[(col % (unsigned)n) / (unsigned)bs]) z[t] = make_ulonglong2(0ull, 0ull);
     }
 }
 
@@ -120,12 +209,17 @@ count_mask_kernel(const uint8_t* __restrict__ mask, long long count, long long* 
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs B, PartyOut F, const int32_t* __restrict__ ids,
-                        int n, int groups, int bs, int d) {
+                        int n, int groups, int bs, int d, const int32_t* __restrict__ blk_label = nullptr) {
     const int party = blockIdx.y;
     const int pairs = d >> 1;
     for (int c = blockIdx.x; c < groups * n; c += gridDim.x) {
         const int grp = c / n, j = c - grp * n;
         const int neuron = ids[j / bs] * bs + (j % bs);
+        if (blk_label && blk_label[j / bs] < 0) {        // a column outside every component is not opened
+            ulonglong2* f0 = reinterpret_cast<ulonglong2*>((party ? F.p[1] : F.p[0]) + (size_t)c * d);
+            for (int t = threadIdx.x; t < pairs; t += blockDim.x) f0[t] = make_ulonglong2(0ull, 0ull);
+            continue;
+        }
         const u64* W = (grp == 0 ? (party ? Wg0.p[1] : Wg0.p[0]) : (party ? Wg1.p[1] : Wg1.p[0]));
         const ulonglong2* __restrict__ w = reinterpret_cast<const ulonglong2*>(W + (size_t)neuron * d);
         const ulonglong2* __restrict__ b = reinterpret_cast<const ulonglong2*>((party ? B.p[1] : B.p[0]) + (size_t)c * d);
