@@ -287,6 +287,9 @@ def main():
     ap.add_argument("--sparsity", type=float, default=None)
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "limb"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--token-masks", type=float, default=0.0, metavar="P",
+                    help="give every token its own Bernoulli(P) mask over the active blocks (Protocols 2 and 3 in "
+                         "general: connected components, per-column row sets); set_token_mask is timed with set_mask")
     ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle"],
                     help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage")
     ap.add_argument("--shuffle-rows", type=int, default=0, help="--op shuffle: rows instead of the workload's tokens")
@@ -337,7 +340,13 @@ def main():
         host = lib_tensors(inp)
         pinned = [{k: torch.from_numpy(v.view(np.int64)).pin_memory() for k, v in hp.items()} for hp in host]
         devt = [{k: v.to(dev) for k, v in hp.items()} for hp in pinned]
-        sets.append({"n": inp["n"], "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
+        tm = None
+        if args.token_masks > 0:
+            tm = torch.from_numpy(wl.token_block_masks(seed, f"bench/tm/{s}", T, int(inp["mask"].sum()),
+                                                       args.token_masks))
+        sets.append({"n": inp["n"], "tm_host": tm.pin_memory() if tm is not None else None,
+                     "tm_dev": tm.to(dev) if tm is not None else None,
+                     "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
                      "mask_dev": torch.from_numpy(inp["mask"]).to(dev), "pinned": pinned, "dev": devt})
     torch.cuda.synchronize(dev)
     n = sets[0]["n"]
@@ -360,6 +369,8 @@ def main():
             e = [ev() for _ in range(6)]
             e[0].record(stream)
             ctx.set_mask(st["mask_dev"])
+            if st["tm_dev"] is not None:
+                ctx.set_token_mask(st["tm_dev"])
             e[1].record(stream)
             for p in (0, 1):
                 for tid in UP_IDS:
@@ -385,6 +396,8 @@ def main():
             e0, e1 = ev(), ev()
             e0.record(stream)
             ctx.set_mask(st["mask_host"].numpy())
+            if st["tm_host"] is not None:
+                ctx.set_token_mask(st["tm_host"].numpy())
             for p in (0, 1):
                 for tid in UP_IDS:
                     ctx.load_shares(p, tid, st["pinned"][p][tid])
@@ -494,6 +507,8 @@ def main():
             "config": {"workload": workload_name(cfg, sparsity), "matmul_path": used_path,
                        "l2": "512 MiB buffer written between steps, and 4 rotating input sets with different masks",
                        "timed": "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream",
+                       "token_masks": (f"per-token Bernoulli({args.token_masks}) masks over the active blocks, "
+                                       f"{stats.n_components} component(s)" if args.token_masks > 0 else "none"),
                        "parallelism": f"independent FFN per GPU x{world}"},
             "gpu_launches": int(launches),
             "clocks": clocks,
