@@ -411,6 +411,30 @@ __device__ __forceinline__ bool limb_wait(uint32_t bar, uint32_t parity, volatil
     return limb_wait_slow(bar, parity, abort_flag);
 }
 
+// The epilogue warps' wait for a finished segment lasts tens of microseconds and involves 256 threads: one lane
+// per warp polls, sleeping between polls so that the warp leaves the issue slots to whoever shares the SM (a
+// co-resident memory-side CTA), and then every lane acquires the completed phase with one (succeeding) poll.
+__device__ __noinline__ bool limb_wait_sleeping(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (;;) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limb::WAIT_CYCLES) {
+            *abort_flag = 1;
+            return false;
+        }
+        __nanosleep(400);
+    }
+}
+
+__device__ __forceinline__ bool limb_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0) ok = limb_wait_sleeping(bar, parity, abort_flag);
+    ok = __shfl_sync(0xffffffffu, ok, 0);      // also reconverges the warp for the aligned TMEM loads
+    if (ok) ok = limb_wait(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
+
 // One contiguous piece of a CTA's share of the (party, tile, k-block) space: a run of k-blocks of one tile.
 struct LimbSegment {
     int party, tm, tn;
@@ -597,38 +621,37 @@ combine_limb_kernel(LimbArgs a) {
         for (long long u = u_begin; u < u_end && ok;) {
             const LimbSegment sg = limb_segment(a, u, u_end);
             u += sg.count;
-            ok = limb_wait(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
-            ok = __all_sync(0xffffffffu, ok);          // also reconverges the warp for the aligned TMEM loads
+            ok = limb_wait_warp(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
             if (!ok) break;
             ptx::fence_after_sync();
             const int row = sg.tm * BM + quarter * 32 + lane;
             const int col0 = sg.tn * BN + chalf * 32;
-            u64 z[32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t d[PLANES][8];
-#pragma unroll
-                for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + c * 8, d[s]);
-                ptx::tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    u64 v = (u64)d[0][j];
-#pragma unroll
-                    for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
-                    z[c * 8 + j] = v;
-                }
-            }
-            // the accumulators are in registers: hand TMEM back before the reduction traffic starts
-            ptx::fence_before_sync();
-            ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
             u64* zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0;
 #pragma unroll
-            for (int h = 0; h < 32 / OUT_COLS; ++h) {
-                ptx::bulk_wait_group_read0();          // the previous reduction has read this thread's staging row
+            for (int h = 0; h < 32 / OUT_COLS; ++h) {          // this thread's 32 columns, OUT_COLS at a time
+                ptx::bulk_wait_group_read0();                  // the previous reduction has read this thread's staging row
 #pragma unroll
-                for (int j = 0; j < OUT_COLS; j += 2)
-                    *reinterpret_cast<ulonglong2*>(my_row + j * 8) =
-                        make_ulonglong2(z[h * OUT_COLS + j], z[h * OUT_COLS + j + 1]);
+                for (int c = 0; c < OUT_COLS / 8; ++c) {
+                    uint32_t d[PLANES][8];
+#pragma unroll
+                    for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + h * OUT_COLS + c * 8, d[s]);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 8; j += 2) {
+                        u64 v0 = (u64)d[0][j], v1 = (u64)d[0][j + 1];
+#pragma unroll
+                        for (int s = 1; s < PLANES; ++s) {
+                            v0 += (u64)d[s][j] << (8 * s);
+                            v1 += (u64)d[s][j + 1] << (8 * s);
+                        }
+                        *reinterpret_cast<ulonglong2*>(my_row + (c * 8 + j) * 8) = make_ulonglong2(v0, v1);
+                    }
+                }
+                if (h == 32 / OUT_COLS - 1) {
+                    // every accumulator has been read: hand TMEM back before the reduction traffic of this round
+                    ptx::fence_before_sync();
+                    ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
+                }
                 int cols = a.N - col0 - h * OUT_COLS;
                 if (cols > OUT_COLS) cols = OUT_COLS;
                 if (row < a.M && cols > 0) {
@@ -811,8 +834,7 @@ combine_limb_few_kernel(LimbArgs a) {
         for (long long u = u_begin; u < u_end && ok;) {
             const LimbSegment sg = limb_segment(a, u, u_end);
             u += sg.count;
-            ok = limb_wait(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = limb_wait_warp(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
             if (!ok) break;
             ptx::fence_after_sync();
             u64 z[16];
