@@ -38,8 +38,8 @@ L2_FLUSH_BYTES = 512 << 20
 # up- and the down-projection launch).  Valid only for the kernel source it was taken on: keyed by its SHA-256.
 COMBINE_LIMB_TRAFFIC = {
     "workload": ("opt1.3b", 0.9),
-    "kernel_sha256": "bde0e5c18ff3d9f03566223900c7a4b121d6c7b98a99ee579388baee226720f5",
-    "bytes_per_launch": 116595456,
+    "kernel_sha256": "203d0add673df528a2987a47adec406f405f4e075aa592bf039e7e19f6b52c78",
+    "bytes_per_launch": 118532096,
 }
 
 
