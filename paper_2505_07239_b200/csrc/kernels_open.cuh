@@ -23,11 +23,13 @@ struct PartyOut {
 // ranks each active block inside its warp, a shuffle scan over the 32 warp
 // totals gives each warp's base, and a running base carries across chunks.
 // `count` points at two words {count, error flag}; both are also written to
-// `host_report` (mapped host memory) so that the host needs no copy.
+// `host_report` (mapped host memory) so that the host needs no copy, followed
+// by `ticket` in host_report[2]: the host may watch that word instead of
+// waiting for the stream.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids, int32_t* __restrict__ count,
-                    int32_t* __restrict__ host_report) {
+                    int32_t* __restrict__ host_report, int32_t ticket) {
     __shared__ int warp_excl[32];
     __shared__ int chunk_total;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -60,6 +62,8 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
         // {count, error flag raised by an earlier kernel's bounded wait} for the host, in mapped pinned memory
         host_report[0] = running;
         host_report[1] = count[1];
+        __threadfence_system();
+        *reinterpret_cast<volatile int32_t*>(host_report + 2) = ticket;
         __threadfence_system();
     }
 }
