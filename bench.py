@@ -321,7 +321,7 @@ def main():
     path = {"auto": cb.PATH_AUTO, "simt": cb.PATH_SIMT, "limb": cb.PATH_LIMB}[args.path]
     stream = torch.cuda.Stream(device=dev)
     n_cap = cfg.n_active_blocks(sparsity) * cfg.block
-    ctx = cb.Comet(T, d, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.gated, local, n_cap, path, stream)
+    ctx = cb.Comet(T, d, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.groups - 1, local, n_cap, path, stream)
     W = wl.model_shares(cfg, seed, plain=False)
     with torch.cuda.stream(stream):
         for p in (0, 1):

@@ -13,10 +13,11 @@
  *     their masks B and the messages F) are stored OUTPUT-FEATURE-MAJOR, i.e.
  *     as the transpose of the paper's matrix: W1 and WG are [d_ff, d_model],
  *     W2 is [d_model, d_ff], B_UP is [g*n, d_model], B_DN is [d_model, n].
- *     (n = active neurons, g = 2 for a gated FFN, else 1.)
+ *     (n = active neurons, g = 1 + `gated` = matrices stacked in the up-projection.)
  *   - Compact column c of the up-projection stands for neuron I[c mod n], I the
  *     ascending list of neurons in active blocks; for g = 2 columns [0,n) are
- *     the gate projection and [n,2n) the up projection.
+ *     the gate projection (WG) and [n,2n) the up projection (W1); for g = 3 columns
+ *     [2n,3n) belong to W3.
  *   - Parties are 0 and 1 (the paper's P_1, P_2); party 1 carries the public
  *     product term of Eq. 1.
  *   - Every call returns COMET_OK or a negative error code; nothing traps or
@@ -84,7 +85,8 @@ enum {
     COMET_E_DN = 14,  /* out: message H_i - A'_i         [T, n]                 */
     COMET_F_DN = 15,  /* out: message W2_i[I, :] - B'_i  [d_model, n]           */
     COMET_Y = 16,     /* out: down-projection share      [T, d_model]           */
-    COMET_NUM_TENSORS = 17
+    COMET_W3 = 17,    /* in : third weight matrix (gated = 2 only) [d_ff, d_model] */
+    COMET_NUM_TENSORS = 18
 };
 
 typedef struct {
@@ -93,7 +95,11 @@ typedef struct {
     int32_t d_ff;         /* multiple of `block`                                        */
     int32_t block;        /* neurons per mask block, multiple of 16                     */
     int32_t frac_bits;    /* fixed-point fractional bits f, 1..31                       */
-    int32_t gated;        /* 0: Y = act(X W1) W2;  1: Y = (act(X WG) * (X W1)) W2       */
+    int32_t gated;        /* weight matrices of the up-projection that share the mask, minus one:
+                             0: W1 alone, Y = act(X W1) W2;  1: [WG || W1], a gated FFN;
+                             2: [WG || W1 || W3], e.g. the query, key and value projections of an
+                             attention layer under a head mask (block = head size, d_ff = heads *
+                             head size, W2 = the output projection): X is still opened once      */
     int32_t device;       /* CUDA device ordinal                                        */
     int32_t max_active;   /* capacity in active neurons, 0 = d_ff                       */
     int32_t matmul_path;  /* COMET_PATH_*                                               */

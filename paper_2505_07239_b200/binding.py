@@ -23,8 +23,8 @@ DEVICE, HOST = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_LIMB = 0, 1, 2
 
 (X, W1, WG, W2, A_UP, B_UP, C_UP, H, A_DN, B_DN, C_DN,
- E_UP, F_UP, Z_UP, E_DN, F_DN, Y) = range(17)
-NUM_TENSORS = 17
+ E_UP, F_UP, Z_UP, E_DN, F_DN, Y, W3) = range(18)
+NUM_TENSORS = 18
 
 EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
@@ -123,7 +123,7 @@ class Comet:
         self._h = ctypes.c_void_p()
         sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
         self._check(_lib.comet_init(ctypes.byref(self.cfg), sp, ctypes.byref(self._h)), "comet_init")
-        self.groups = 2 if gated else 1
+        self.groups = int(gated) + 1
         self.n_active = 0
 
     # ------------------------------------------------------------------ plumbing

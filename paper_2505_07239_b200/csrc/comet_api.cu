@@ -24,7 +24,7 @@ using comet::u64;
 struct comet_ctx {
     comet_config cfg;
     cudaStream_t stream;
-    int groups;                   // 1 or 2
+    int groups;                   // 1, 2 or 3 weight matrices stacked in the up-projection
     int64_t cap_T, cap_n;         // capacities
     int sm_count;
     u64* buf[2][COMET_NUM_TENSORS];
@@ -114,14 +114,14 @@ struct PhaseTimer {
     }
 };
 
-inline int is_input(int id) { return id >= COMET_X && id <= COMET_C_DN; }
+inline int is_input(int id) { return (id >= COMET_X && id <= COMET_C_DN) || id == COMET_W3; }
 
 // current shape of a tensor as stored; rows = cols = 0 when not defined yet
 void tensor_shape(const comet_ctx* c, int id, int64_t T, int64_t* rows, int64_t* cols) {
     const int64_t d = c->cfg.d_model, D = c->cfg.d_ff, n = c->n_active, gn = (int64_t)c->groups * n;
     switch (id) {
         case COMET_X: case COMET_A_UP: case COMET_E_UP: case COMET_C_DN: case COMET_Y: *rows = T; *cols = d; break;
-        case COMET_W1: case COMET_WG: *rows = D; *cols = d; break;
+        case COMET_W1: case COMET_WG: case COMET_W3: *rows = D; *cols = d; break;
         case COMET_W2: *rows = d; *cols = D; break;
         case COMET_B_UP: case COMET_F_UP: *rows = gn; *cols = d; break;
         case COMET_C_UP: case COMET_Z_UP: *rows = T; *cols = gn; break;
@@ -136,7 +136,8 @@ int64_t tensor_capacity(const comet_ctx* c, int id) {
     switch (id) {
         case COMET_X: case COMET_A_UP: case COMET_E_UP: case COMET_C_DN: case COMET_Y: return T * d;
         case COMET_W1: return D * d;
-        case COMET_WG: return c->groups == 2 ? D * d : 0;
+        case COMET_WG: return c->groups >= 2 ? D * d : 0;
+        case COMET_W3: return c->groups == 3 ? D * d : 0;
         case COMET_W2: return d * D;
         case COMET_B_UP: case COMET_F_UP: return gn * d;
         case COMET_C_UP: case COMET_Z_UP: return T * gn;
@@ -199,8 +200,9 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
         a.X[p] = c->buf[p][pr.idX];
         a.A[p] = c->buf[p][pr.idA];
         a.E[p] = c->buf[p][pr.idE];
-        a.W0[p] = pr.down ? c->buf[p][COMET_W2] : (c->groups == 2 ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1]);
+        a.W0[p] = pr.down ? c->buf[p][COMET_W2] : (c->groups >= 2 ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1]);
         a.W1[p] = c->buf[p][COMET_W1];
+        a.W2g[p] = c->buf[p][COMET_W3];
         a.B[p] = c->buf[p][pr.idB];
         a.F[p] = c->buf[p][pr.idF];
         a.Bpl[p] = planes[p][0];
@@ -367,7 +369,7 @@ int comet_last_cuda_error(comet_ctx* ctx) { return ctx ? ctx->last_cuda_error : 
 int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     if (!cfg || !out) return COMET_ERR_INVALID_ARG;
     *out = nullptr;
-    if (cfg->gated != 0 && cfg->gated != 1) return COMET_ERR_INVALID_ARG;
+    if (cfg->gated < 0 || cfg->gated > 2) return COMET_ERR_INVALID_ARG;
     if (cfg->matmul_path < COMET_PATH_AUTO || cfg->matmul_path > COMET_PATH_LIMB) return COMET_ERR_INVALID_ARG;
     if (cfg->device < 0) return COMET_ERR_INVALID_ARG;
     if (cfg->max_tokens < 1 || cfg->d_model < 16 || cfg->d_ff < 16 || cfg->block < 16) return COMET_ERR_SHAPE;
@@ -393,7 +395,7 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     }
     c->cfg = *cfg;
     c->stream = (cudaStream_t)cuda_stream;
-    c->groups = cfg->gated ? 2 : 1;
+    c->groups = cfg->gated + 1;
     c->cap_T = cfg->max_tokens;
     c->cap_n = cfg->max_active ? cfg->max_active : cfg->d_ff;
     if (cudaSetDevice(cfg->device) != cudaSuccess ||
@@ -510,7 +512,8 @@ int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* pt
     if (!c || (party != 0 && party != 1) || !is_input(tensor_id)) return COMET_ERR_INVALID_ARG;
     if (!ptr && rows * cols != 0) return COMET_ERR_INVALID_ARG;      // an empty tensor may come with a null pointer
     if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
-    if (tensor_id == COMET_WG && c->groups != 2) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_WG && c->groups < 2) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_W3 && c->groups != 3) return COMET_ERR_INVALID_ARG;
     const bool needs_mask = tensor_id == COMET_B_UP || tensor_id == COMET_C_UP || tensor_id == COMET_H ||
                             tensor_id == COMET_A_DN || tensor_id == COMET_B_DN;
     if (needs_mask && !c->mask_set) return COMET_ERR_STATE;
@@ -631,7 +634,8 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
     for (int p = 0; p < 2; ++p) {
         for (int id : need)
             if (!c->loaded[p][id]) return COMET_ERR_STATE;
-        if (c->groups == 2 && !c->loaded[p][COMET_WG]) return COMET_ERR_STATE;
+        if (c->groups >= 2 && !c->loaded[p][COMET_WG]) return COMET_ERR_STATE;
+        if (c->groups == 3 && !c->loaded[p][COMET_W3]) return COMET_ERR_STATE;
     }
     const int d = c->cfg.d_model, n = c->n_active, g = c->groups, bs = c->cfg.block;
     if (c->tmask_set && c->tmask_tokens != tokens) return COMET_ERR_SHAPE;   // the token mask was given for another T
@@ -680,13 +684,14 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
         return somm_merge(c, tokens);
     }
 
-    comet::PartyPtrs X, A, W0, W1, B;
+    comet::PartyPtrs X, A, W0, W1, W3, B;
     comet::PartyOut E, F;
     for (int p = 0; p < 2; ++p) {
         X.p[p] = c->buf[p][COMET_X];
         A.p[p] = c->buf[p][COMET_A_UP];
         E.p[p] = c->buf[p][COMET_E_UP];
-        W0.p[p] = (g == 2) ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1];
+        W0.p[p] = (g >= 2) ? c->buf[p][COMET_WG] : c->buf[p][COMET_W1];
+        W3.p[p] = c->buf[p][COMET_W3];
         W1.p[p] = c->buf[p][COMET_W1];
         B.p[p] = c->buf[p][COMET_B_UP];
         F.p[p] = c->buf[p][COMET_F_UP];
@@ -698,7 +703,7 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
             X, A, E, pairs, nullptr, 0, d, bs, c->tmask_set ? c->d_row_label : nullptr);
         int rows_grid = g * n < c->sm_count * 8 ? g * n : c->sm_count * 8;
         comet::open_weight_rows_kernel<<<dim3(rows_grid, 2), 256, 0, c->stream>>>(
-            W0, W1, B, F, c->d_ids, n, g, bs, d, c->tmask_set ? c->d_blk_label : nullptr);
+            W0, W1, W3, B, F, c->d_ids, n, g, bs, d, c->tmask_set ? c->d_blk_label : nullptr);
     }
     c->stats.kernel_launches += 2;
     COMET_CUDA(c, cudaGetLastError());
@@ -800,7 +805,8 @@ int comet_get(comet_ctx* c, int party, int tensor_id, uint64_t* out, int locatio
     if (!c || !out || (party != 0 && party != 1) || tensor_id < 0 || tensor_id >= COMET_NUM_TENSORS)
         return COMET_ERR_INVALID_ARG;
     if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
-    if (tensor_id == COMET_WG && c->groups != 2) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_WG && c->groups < 2) return COMET_ERR_INVALID_ARG;
+    if (tensor_id == COMET_W3 && c->groups != 3) return COMET_ERR_INVALID_ARG;
     int64_t T = c->tokens;
     if (tensor_id == COMET_E_UP || tensor_id == COMET_Z_UP) T = c->up_tokens;
     if (tensor_id == COMET_E_DN || tensor_id == COMET_Y) T = c->down_tokens;

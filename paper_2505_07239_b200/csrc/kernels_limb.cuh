@@ -115,6 +115,7 @@ struct LimbOpenArgs {
     int left_blocks;
     const u64* W0[2];        // weights of group 0 (gate when gated, else the only matrix)
     const u64* W1[2];        // weights of group 1 (up-projection of a gated FFN)
+    const u64* W2g[2];       // weights of group 2 (third stacked matrix, e.g. the value projection)
     const u64* B[2];
     u64* F[2];
     uint8_t* Bpl[2];
@@ -186,7 +187,8 @@ limb_open_kernel(LimbOpenArgs a) {
                     const int grp = row / a.n, j = row - grp * a.n;
                     const int neuron = a.ids[j / a.bs] * a.bs + (j % a.bs);
                     dead = a.blk_label && a.blk_label[j / a.bs] < 0;
-                    wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0]) : (party ? a.W1[1] : a.W1[0])) +
+                    wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0])
+                                     : grp == 1 ? (party ? a.W1[1] : a.W1[0]) : (party ? a.W2g[1] : a.W2g[0])) +
                            (size_t)neuron * a.ldw + k;
                 }
                 const size_t o = (size_t)row * a.K + k;

@@ -207,12 +207,12 @@ count_mask_kernel(const uint8_t* __restrict__ mask, long long count, long long* 
 // K3 (up): F_i[c, :] = W_i[neuron(c), :] - B_i[c, :].  The paper's IndexCols
 // (Protocol 2 line 5) followed by [e]_i = [y]_i - [b]_i; with weights stored
 // output-feature-major the column gather is a gather of whole rows of d words.
-// Compact row c in [0, g*n): group = c / n selects the weight matrix (gate
-// first when gated), j = c mod n, neuron = ids[j / bs] * bs + j mod bs.
+// Compact row c in [0, g*n): group = c / n selects the weight matrix (WG, W1,
+// W3 in that order when there are several), j = c mod n, neuron = ids[j / bs] * bs + j mod bs.
 // One CTA per compact row (grid-strided); threads sweep the row 16 bytes each.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs B, PartyOut F, const int32_t* __restrict__ ids,
+open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs Wg2, PartyPtrs B, PartyOut F, const int32_t* __restrict__ ids,
                         int n, int groups, int bs, int d, const int32_t* __restrict__ blk_label = nullptr) {
     const int party = blockIdx.y;
     const int pairs = d >> 1;
@@ -224,7 +224,8 @@ open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs B, PartyOut F, c
             for (int t = threadIdx.x; t < pairs; t += blockDim.x) f0[t] = make_ulonglong2(0ull, 0ull);
             continue;
         }
-        const u64* W = (grp == 0 ? (party ? Wg0.p[1] : Wg0.p[0]) : (party ? Wg1.p[1] : Wg1.p[0]));
+        const u64* W = (grp == 0 ? (party ? Wg0.p[1] : Wg0.p[0])
+                                 : grp == 1 ? (party ? Wg1.p[1] : Wg1.p[0]) : (party ? Wg2.p[1] : Wg2.p[0]));
         const ulonglong2* __restrict__ w = reinterpret_cast<const ulonglong2*>(W + (size_t)neuron * d);
         const ulonglong2* __restrict__ b = reinterpret_cast<const ulonglong2*>((party ? B.p[1] : B.p[0]) + (size_t)c * d);
         ulonglong2* __restrict__ f = reinterpret_cast<ulonglong2*>((party ? F.p[1] : F.p[0]) + (size_t)c * d);

@@ -108,6 +108,7 @@ class FFNConfig:
     x_dist: str               # "uniform" | "normal"
     w_dist: str               # "uniform" | "normal0.02"
     steps: int = 1            # decode: number of single-token steps, fresh mask each
+    stacked: int = 0          # weight matrices stacked in the up-projection; 0 = 2 if gated else 1
 
     @property
     def n_blocks(self) -> int:
@@ -115,7 +116,7 @@ class FFNConfig:
 
     @property
     def groups(self) -> int:
-        return 2 if self.gated else 1
+        return self.stacked if self.stacked else (2 if self.gated else 1)
 
     def n_active_blocks(self, sparsity: Optional[float] = None) -> int:
         p = self.active_fraction if sparsity is None else 1.0 - sparsity
@@ -212,8 +213,10 @@ def model_shares(cfg: FFNConfig, seed: int, plain: bool = True) -> dict:
     """
     out = {}
     names = [("W1", (cfg.d_model, cfg.d_ff)), ("W2", (cfg.d_ff, cfg.d_model))]
-    if cfg.gated:
+    if cfg.groups >= 2:
         names.insert(1, ("WG", (cfg.d_model, cfg.d_ff)))
+    if cfg.groups == 3:
+        names.append(("W3", (cfg.d_model, cfg.d_ff)))
     for name, shape in names:
         if plain:
             ring = encode(_draw(cfg.w_dist, seed, f"{cfg.name}/{name}", shape), cfg.frac_bits)

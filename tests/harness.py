@@ -24,20 +24,25 @@ def _mismatch(name, got, want, report):
 
 
 def make_context(cfg, tokens, matmul_path=cb.PATH_AUTO, max_active=0):
-    return cb.Comet(tokens, cfg.d_model, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.gated, 0, max_active, matmul_path)
+    return cb.Comet(tokens, cfg.d_model, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.groups - 1, 0, max_active, matmul_path)
 
 
 def load_weights(ctx, cfg, W):
     for party in (0, 1):
         ctx.load_shares(party, cb.W1, cb.to_device(wl.lib_layout(W["W1"][1 + party])))
         ctx.load_shares(party, cb.W2, cb.to_device(wl.lib_layout(W["W2"][1 + party])))
-        if cfg.gated:
+        if cfg.groups >= 2:
             ctx.load_shares(party, cb.WG, cb.to_device(wl.lib_layout(W["WG"][1 + party])))
+        if cfg.groups == 3:
+            ctx.load_shares(party, cb.W3, cb.to_device(wl.lib_layout(W["W3"][1 + party])))
 
 
 def oracle_up_operand(cfg, W, party_slot):
-    """The paper-shaped right operand of the up product: W1, or [WG || W1] when gated."""
-    if cfg.gated:
+    """The paper-shaped right operand of the up product: W1, [WG || W1] when gated, [WG || W1 || W3] for three
+    stacked matrices."""
+    if cfg.groups == 3:
+        return np.concatenate([W["WG"][party_slot], W["W1"][party_slot], W["W3"][party_slot]], axis=1)
+    if cfg.groups == 2:
         return np.concatenate([W["WG"][party_slot], W["W1"][party_slot]], axis=1)
     return W["W1"][party_slot]
 

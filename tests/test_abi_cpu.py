@@ -44,7 +44,7 @@ def test_init_validates_before_any_cuda_call(cb):
     good = dict(max_tokens=16, d_model=256, d_ff=1024, block=32, frac_bits=12, gated=0, device=0, max_active=0,
                 matmul_path=0)
     bad = [
-        (dict(good, gated=2), -1), (dict(good, matmul_path=7), -1), (dict(good, device=-1), -1),
+        (dict(good, gated=3), -1), (dict(good, gated=-1), -1), (dict(good, matmul_path=7), -1), (dict(good, device=-1), -1),
         (dict(good, max_tokens=0), -2), (dict(good, d_model=250), -2), (dict(good, d_ff=1000), -2),
         (dict(good, block=8), -2), (dict(good, block=24), -2), (dict(good, frac_bits=0), -2),
         (dict(good, frac_bits=32), -2), (dict(good, max_active=48), -2), (dict(good, max_active=2048), -2),
