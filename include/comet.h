@@ -297,6 +297,25 @@ int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* in
                              int32_t* bad_index_flag);
 
 /* ---------------------------------------------------------------------------
+ * KV-cache manager, Section 6: which cache entries to compute together with the
+ * current token.  Host logic only (HOST pointers, no GPU work): the result is a
+ * per-token mask over heads, exactly what comet_set_token_mask takes for the
+ * sparse QKV product, so that every token and every head takes part once
+ * (Section 6.1, merging).
+ *   present [tokens, heads]  non-zero = the (token, head) key/value is cached
+ *   active  [heads]          non-zero = head activated for the current token
+ *   x, w                     token vector size and size of one head's weight
+ *                            matrix, in words (OPT-6.7B: 4096 and 4096*128)
+ * request [tokens, heads] (out) gets 1 for every absent entry of an activated
+ * head and of every prefetched head; prefetch [heads] (out) gets 1 for the heads
+ * that are not activated but are worth refilling now by the rule of Section 6.2,
+ * L2 > w/x + max(0, L2 - L1), L2 the head's absent entries and L1 the number of
+ * tokens the merged refill of the activated heads sends anyway.  *l1_out (may be
+ * NULL) receives L1.  Errors: INVALID_ARG (null pointer), SHAPE (sizes < 1). */
+int comet_kv_plan(const uint8_t* present, const uint8_t* active, int32_t tokens, int32_t heads, int64_t x, int64_t w,
+                  uint8_t* request, uint8_t* prefetch, int32_t* l1_out);
+
+/* ---------------------------------------------------------------------------
  * Element-wise Beaver product, Section 2.1 "Multiplication", Eq. 1 applied to
  * every element (in a gated FFN: ReLU(gate) times up), for both parties:
  *     D[i] = X[i] - A[i],  E[i] = Y[i] - B[i]            (the two messages), then

@@ -30,7 +30,7 @@ EXPORTS = (
     "comet_init", "comet_destroy", "comet_load_shares", "comet_set_mask", "comet_ffn_up", "comet_ffn_down",
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
-    "comet_beaver_mul", "comet_set_token_mask", "comet_get_components",
+    "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -89,6 +89,7 @@ def _load():
     lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
     lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
     lib.comet_invert_permutation.argtypes = [vp, vp, vp, i64, vp]
+    lib.comet_kv_plan.argtypes = [vp, vp, i32, i32, i64, i64, vp, vp, ctypes.POINTER(i32)]
     lib.comet_beaver_mul.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, pair, i64]
     return lib
 
@@ -326,3 +327,19 @@ def beaver_mul(X, Y, A, B, C, stream: Optional[torch.cuda.Stream] = None):
     if code != OK:
         raise CometError(code, "comet_beaver_mul")
     return D, E, Z
+
+
+def kv_plan(present: np.ndarray, active: np.ndarray, x: int, w: int):
+    """KV-cache manager's request planning (comet_kv_plan, host logic): returns (request [tokens, heads] uint8,
+    prefetch [heads] uint8, L1).  `request` is the per-token head mask of the merged refill + prefetch batch."""
+    present = np.ascontiguousarray(present, dtype=np.uint8)
+    active = np.ascontiguousarray(active, dtype=np.uint8)
+    tokens, heads = present.shape
+    request = np.empty((tokens, heads), np.uint8)
+    prefetch = np.empty(heads, np.uint8)
+    l1 = ctypes.c_int32(0)
+    code = _lib.comet_kv_plan(present.ctypes.data, active.ctypes.data, tokens, heads, x, w, request.ctypes.data,
+                              prefetch.ctypes.data, ctypes.byref(l1))
+    if code != OK:
+        raise CometError(code, "comet_kv_plan")
+    return request, prefetch, l1.value

@@ -1071,3 +1071,38 @@ extern "C" int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], c
     }
     return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------
+// KV-cache manager (Section 6): request merging and the prefetch rule.  Host logic.
+// ---------------------------------------------------------------------------
+extern "C" int comet_kv_plan(const uint8_t* present, const uint8_t* active, int32_t tokens, int32_t heads, int64_t x,
+                             int64_t w, uint8_t* request, uint8_t* prefetch, int32_t* l1_out) {
+    if (!present || !active || !request || !prefetch) return COMET_ERR_INVALID_ARG;
+    if (tokens < 1 || heads < 1 || x < 1 || w < 1) return COMET_ERR_SHAPE;
+    std::vector<int64_t> missing(heads, 0);
+    int32_t l1 = 0;
+    for (int32_t t = 0; t < tokens; ++t) {
+        bool in_batch = false;
+        for (int32_t h = 0; h < heads; ++h) {
+            const bool miss = present[(size_t)t * heads + h] == 0;
+            missing[h] += miss;
+            const bool want = miss && active[h] != 0;
+            request[(size_t)t * heads + h] = want ? 1 : 0;
+            in_batch = in_batch || want;
+        }
+        l1 += in_batch;
+    }
+    for (int32_t h = 0; h < heads; ++h) {
+        prefetch[h] = 0;
+        if (active[h] != 0) continue;
+        const int64_t l2 = missing[h], beyond = l2 > l1 ? l2 - l1 : 0;
+        // saved 2*L2*x against spent 2*(w + x*max(0, L2 - L1)), in integers: L2 > w/x + max(0, L2 - L1)
+        if (l2 * x > w + x * beyond) {
+            prefetch[h] = 1;
+            for (int32_t t = 0; t < tokens; ++t)
+                if (present[(size_t)t * heads + h] == 0) request[(size_t)t * heads + h] = 1;
+        }
+    }
+    if (l1_out) *l1_out = l1;
+    return COMET_OK;
+}
