@@ -296,6 +296,13 @@ int comet_shuffle(void* cuda_stream, const uint64_t* const X[2], const int32_t* 
 int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* inverse, int64_t rows,
                              int32_t* bad_index_flag);
 
+/* Section 2.1 "Addition": a secret-shared bias is added locally, each party adding its
+ * own share: Z[i][r, :] += bias[i] for every row r, in place, for both parties.
+ * DEVICE pointers on the current device, Z[i] of rows*cols words, bias[i] of cols
+ * words, at the same fixed-point scale.  One kernel on `cuda_stream`; stateless.
+ * Errors: INVALID_ARG (null pointer), SHAPE (rows or cols < 1), CUDA. */
+int comet_add_bias(void* cuda_stream, uint64_t* const Z[2], const uint64_t* const bias[2], int64_t rows, int64_t cols);
+
 /* ---------------------------------------------------------------------------
  * KV-cache manager, Section 6: which cache entries to compute together with the
  * current token.  Host logic only (HOST pointers, no GPU work): the result is a

@@ -307,3 +307,13 @@ def beaver_mul(x, y, a, b, c):
     outs = [np.empty(shape, U64) for _ in range(6)]
     lib().orc_beaver_mul(ctypes.c_size_t(arrs[0].size), *[_p(v) for v in arrs], *[_p(o) for o in outs])
     return {"D": (outs[0], outs[1]), "E": (outs[2], outs[3]), "Z": (outs[4], outs[5])}
+
+
+def add_bias(Zi, bias_i):
+    """One party's local addition of its bias share [N] to every row of its share [T, N]."""
+    Zi, bias_i = _u64(Zi), _u64(bias_i)
+    T, N = Zi.shape
+    assert bias_i.shape == (N,)
+    out = np.empty_like(Zi)
+    lib().orc_add_bias(ctypes.c_int(T), ctypes.c_int(N), _p(Zi), _p(bias_i), _p(out))
+    return out

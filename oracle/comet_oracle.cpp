@@ -502,4 +502,14 @@ void orc_beaver_mul(size_t count, const u64* x0, const u64* x1, const u64* y0, c
     }
 }
 
+// ---------------------------------------------------------------------------
+// Section 2.1, "Addition": adding a secret-shared vector is local, each party
+// adds its own share.  Here a shared bias [N] is added to every row of a shared
+// matrix [T, N] (both at the same fixed-point scale).
+// ---------------------------------------------------------------------------
+void orc_add_bias(int T, int N, const u64* Zi, const u64* bias_i, u64* out) {
+    for (int r = 0; r < T; ++r)
+        for (int c = 0; c < N; ++c) out[(size_t)r * N + c] = Zi[(size_t)r * N + c] + bias_i[c];
+}
+
 }  // extern "C"

@@ -31,6 +31,7 @@ EXPORTS = (
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
     "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
+    "comet_add_bias",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -89,6 +90,7 @@ def _load():
     lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
     lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
     lib.comet_invert_permutation.argtypes = [vp, vp, vp, i64, vp]
+    lib.comet_add_bias.argtypes = [vp, pair, pair, i64, i64]
     lib.comet_kv_plan.argtypes = [vp, vp, i32, i32, i64, i64, vp, vp, ctypes.POINTER(i32)]
     lib.comet_beaver_mul.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, pair, i64]
     return lib
@@ -343,3 +345,14 @@ def kv_plan(present: np.ndarray, active: np.ndarray, x: int, w: int):
     if code != OK:
         raise CometError(code, "comet_kv_plan")
     return request, prefetch, l1.value
+
+
+def add_bias(Z, bias, stream: Optional[torch.cuda.Stream] = None):
+    """Z[i][r, :] += bias[i] in place for both parties (comet_add_bias)."""
+    rows, cols = Z[0].shape
+    for t in bias:
+        assert t.element_size() == 8 and tuple(t.shape) == (cols,)
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    code = _lib.comet_add_bias(sp, _pair(Z, (rows, cols)), _pair(bias), rows, cols)
+    if code != OK:
+        raise CometError(code, "comet_add_bias")

@@ -1106,3 +1106,18 @@ extern "C" int comet_kv_plan(const uint8_t* present, const uint8_t* active, int3
     if (l1_out) *l1_out = l1;
     return COMET_OK;
 }
+
+extern "C" int comet_add_bias(void* cuda_stream, uint64_t* const Z[2], const uint64_t* const bias[2], int64_t rows,
+                              int64_t cols) {
+    if (!Z || !bias || !Z[0] || !Z[1] || !bias[0] || !bias[1]) return COMET_ERR_INVALID_ARG;
+    if (rows < 1 || cols < 1 || cols > 0x7fffffffll) return COMET_ERR_SHAPE;
+    comet::BiasArgs g;
+    for (int p = 0; p < 2; ++p) {
+        g.z[p] = reinterpret_cast<u64*>(Z[p]);
+        g.bias[p] = reinterpret_cast<const u64*>(bias[p]);
+    }
+    g.rows = rows;
+    g.cols = (int)cols;
+    comet::add_bias_kernel<<<dim3(shuffle_grid(rows * cols), 2), 256, 0, (cudaStream_t)cuda_stream>>>(g);
+    return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
+}

@@ -68,4 +68,22 @@ beaver_mul_combine_kernel(MulArgs g) {
         z[t] = mul_combine(__ldg(c + t), d0[t], d1[t], e0[t], e1[t], __ldg(a + t), __ldg(b + t), party);
 }
 
+// Section 2.1 "Addition": a shared bias [cols] added to every row of a shared matrix, in place; purely local.
+struct BiasArgs {
+    u64* z[2];
+    const u64* bias[2];
+    long long rows;
+    int cols;
+};
+
+__global__ void __launch_bounds__(256)
+add_bias_kernel(BiasArgs g) {
+    const int party = blockIdx.y;
+    u64* __restrict__ z = party ? g.z[1] : g.z[0];
+    const u64* __restrict__ b = party ? g.bias[1] : g.bias[0];
+    const long long total = g.rows * g.cols, stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride)
+        z[t] += __ldg(b + (int)(t % g.cols));
+}
+
 }  // namespace comet

@@ -77,3 +77,74 @@ def test_beaver_mul_argument_errors():
     assert lib.comet_beaver_mul(None, ok, ok, ok, null, ok, ok, ok, ok, 4) == -1
     assert lib.comet_beaver_mul(None, ok, ok, ok, ok, ok, ok, ok, ok, 0) == -2
     torch.cuda.synchronize()
+
+
+def test_gated_ffn_chain_with_bias_only_the_comparison_is_ideal():
+    """Whole gated FFN on shares with everything but the comparison done by the library: up-projection [gate || up],
+    bias, truncation, ReLU(gate) by the ideal functionality, the element-wise Beaver product, truncation, and the
+    down-projection.  Bit-exact against the oracle chain, and close to the float64 FFN."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    cfg = wl.FFNConfig("gated-chain", 40, 128, 512, 64, 16, True, 0.5, "uniform", "normal", "normal0.02")
+    seed, T, d, f, bs = 606, cfg.tokens, cfg.d_model, cfg.frac_bits, cfg.block
+    W = wl.model_shares(cfg, seed)
+    Xr, X0, X1 = wl.activation_shares(cfg, seed)
+    mask = wl.block_mask(cfg, seed)
+    I1, Ig = oracle.index_set(mask, bs, 1), oracle.index_set(mask, bs, 2)
+    n = I1.size
+    bias_plain = wl.encode(wl.random_normal(seed, "bias", 2 * n, 0.1), 2 * f)        # at the product's scale 2f
+    bias = wl.split_shares(bias_plain, seed, "bias")
+
+    ctx = hz.make_context(cfg, T, cb.PATH_LIMB)
+    hz.load_weights(ctx, cfg, W)
+    for p, Xs in ((0, X0), (1, X1)):
+        ctx.load_shares(p, cb.X, cb.to_device(Xs))
+    assert ctx.set_mask(mask) == n
+    tri = wl.dealer_triple(seed, "up", T, d, 2 * n)
+    hz.load_triple_up(ctx, tri)
+    ctx.ffn_up(T)
+    ref = oracle.somm((X0, X1), (hz.oracle_up_operand(cfg, W, 1), hz.oracle_up_operand(cfg, W, 2)), Ig,
+                      tri["A"][1:], tri["B"][1:], tri["C"][1:])
+    # bias and truncation: library on its own copies of Z (stateless calls), oracle beside it
+    Zdev = [_dev(ctx.get(p, cb.Z_UP, (T, 2 * n))) for p in (0, 1)]
+    cb.add_bias(Zdev, [_dev(b) for b in bias])
+    torch.cuda.synchronize()
+    Zb_ref = [oracle.add_bias(ref["Z"][p], bias[p]) for p in (0, 1)]
+    for p in (0, 1):
+        assert np.array_equal(_host(Zdev[p]), Zb_ref[p])
+    Hpre = [oracle.truncate(p, Zb_ref[p], f) for p in (0, 1)]
+    gate = (Hpre[0][:, :n] + Hpre[1][:, :n]).view(np.int64)
+    relu = np.maximum(gate, 0).view(np.uint64)                                       # the only ideal step
+    rs = wl.split_shares(relu, seed, "relu")
+    us = (np.ascontiguousarray(Hpre[0][:, n:]), np.ascontiguousarray(Hpre[1][:, n:]))
+    tm = wl.dealer_triple_elementwise(seed, "mul", (T, n))
+    _, _, Zm = cb.beaver_mul([_dev(v) for v in rs], [_dev(v) for v in us], [_dev(v) for v in tm["a"][1:]],
+                             [_dev(v) for v in tm["b"][1:]], [_dev(v) for v in tm["c"][1:]])
+    torch.cuda.synchronize()
+    mref = oracle.beaver_mul(rs, us, tm["a"][1:], tm["b"][1:], tm["c"][1:])
+    H = []
+    for p in (0, 1):
+        assert np.array_equal(_host(Zm[p]), mref["Z"][p])
+        H.append(oracle.truncate(p, mref["Z"][p], f))
+    for p in (0, 1):
+        ctx.load_shares(p, cb.H, cb.to_device(H[p]))
+    trd = wl.dealer_triple(seed, "down", T, n, d)
+    hz.load_triple_down(ctx, trd)
+    ctx.ffn_down(T)
+    ctx.truncate(cb.Y)
+    refd = oracle.simm((H[0], H[1]), W["W2"][1:], I1, trd["A"][1:], trd["B"][1:], trd["C"][1:])
+    O = []
+    for p in (0, 1):
+        O.append(ctx.get(p, cb.Y, (T, d)))
+        assert np.array_equal(O[p], oracle.truncate(p, refd["Z"][p], f))
+    ctx.close()
+    # against the float64 gated FFN with the same bias (bias decoded at scale 2f)
+    x = wl.decode(Xr, f)
+    g64 = x @ wl.decode(W["WG"][0], f)[:, I1] + wl.decode(bias_plain[:n], 2 * f)
+    u64 = x @ wl.decode(W["W1"][0], f)[:, I1] + wl.decode(bias_plain[n:], 2 * f)
+    want = (np.maximum(g64, 0.0) * u64) @ wl.decode(W["W2"][0], f)[I1, :]
+    got = wl.decode(O[0] + O[1], f)
+    assert np.abs(got - want).max() < 2.0 ** -10

@@ -77,3 +77,13 @@ def test_planted_mistakes_are_caught():
     assert not np.array_equal(same["Z"][0] + same["Z"][1], want)
     both = oracle.beaver_mul(xs, ys, t["a"][1:], t["b"][1:], (t["c"][1], t["c"][1]))   # not a sharing of c
     assert not np.array_equal(both["Z"][0] + both["Z"][1], want)
+
+
+def test_bias_addition_is_local_and_reconstructs():
+    seed, T, N = 8, 5, 7
+    z = wl.random_u64(seed, "z", T * N).reshape(T, N)
+    b = wl.random_u64(seed, "b", N)
+    zs, bs = wl.split_shares(z, seed, "z"), wl.split_shares(b, seed, "b")
+    out = [oracle.add_bias(zs[i], bs[i]) for i in (0, 1)]
+    assert np.array_equal(out[0] + out[1], z + b[None, :])        # Section 2.1: z = x + y share by share
+    assert np.array_equal(out[0], zs[0] + bs[0][None, :])
