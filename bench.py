@@ -35,10 +35,10 @@ L2_FLUSH_BYTES = 512 << 20
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the tensor-core combine kernel on the
 # default workload, from the ncu capture summarised in profiles/combine_limb__opt1.3b_s90.md (average of the
-# up- and the down-projection launch).  Valid only for the kernel source it was taken on: keyed by its SHA-256.
+# up- and the down-projection launch).  Valid only for the kernel source it was taken on: keyed by the SHA-256 of the kernel's part of kernels_limb.cuh.
 COMBINE_LIMB_TRAFFIC = {
     "workload": ("opt1.3b", 0.9),
-    "kernel_sha256": "203d0add673df528a2987a47adec406f405f4e075aa592bf039e7e19f6b52c78",
+    "kernel_sha256": "f6fc21e7dbfc2e6caffd71774bd4a40d907e7c300ea5cca4d46c2bdd0a96c87f",
     "bytes_per_launch": 118532096,
 }
 
@@ -51,9 +51,12 @@ def combine_traffic(workload, sparsity, used_path):
         return None
     src = os.path.join(ROOT, "paper_2505_07239_b200", "csrc", "kernels_limb.cuh")
     try:
-        with open(src, "rb") as fh:
-            digest = hashlib.sha256(fh.read()).hexdigest()
-    except OSError:
+        with open(src) as fh:
+            text = fh.read()
+        # the kernel proper: from its argument block to the banner of the next kernel in the file
+        text = text[text.index("struct LimbArgs {"):text.index("// Few tokens (M <= 32")]
+        digest = hashlib.sha256(text.encode()).hexdigest()
+    except (OSError, ValueError):
         return None
     return COMBINE_LIMB_TRAFFIC["bytes_per_launch"] if digest == COMBINE_LIMB_TRAFFIC["kernel_sha256"] else None
 
@@ -290,6 +293,10 @@ def main():
     ap.add_argument("--token-masks", type=float, default=0.0, metavar="P",
                     help="give every token its own Bernoulli(P) mask over the active blocks (Protocols 2 and 3 in "
                          "general: connected components, per-column row sets); set_token_mask is timed with set_mask")
+    ap.add_argument("--in-flight", type=int, default=4, metavar="C",
+                    help="independent FFN problems in flight (contexts, one stream each, inputs bound in place); the "
+                         "headline throughput is measured that way when C > 1, the one-problem-at-a-time figures are "
+                         "reported beside it; 1 = only the latter")
     ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle"],
                     help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage")
     ap.add_argument("--shuffle-rows", type=int, default=0, help="--op shuffle: rows instead of the workload's tokens")
@@ -330,7 +337,6 @@ def main():
             if cfg.gated:
                 ctx.load_shares(p, cb.WG, cb.to_device(wl.lib_layout(W["WG"][1 + p]), dev))
     ctx.synchronize()
-    del W
 
     # rotating input sets: a fresh mask (so different weight rows), X, triples and H each
     R = 4
@@ -445,6 +451,71 @@ def main():
     stats = ctx.stats()
     ctx.set_profiling(False)
 
+    # ---- several independent problems in flight (throughput mode): C contexts with their own weights, stream and
+    #      two input sets each, inputs bound in place (no copies), steps issued round-robin; the region is timed
+    #      as a whole on the device.  No flush here: consecutive uses of a context see different masks and inputs,
+    #      and the contexts together hold far more than the L2.
+    piped = None
+    if args.in_flight > 1:
+        C = args.in_flight
+        tstream = torch.cuda.Stream(device=dev)
+        pctx, psets = [], []
+        for k in range(C):
+            sk = torch.cuda.Stream(device=dev)
+            cx = cb.Comet(T, d, cfg.d_ff, cfg.block, cfg.frac_bits, cfg.groups - 1, local, n_cap, path, sk)
+            with torch.cuda.stream(sk):
+                for p in (0, 1):
+                    cx.load_shares(p, cb.W1, cb.to_device(wl.lib_layout(W["W1"][1 + p]), dev))
+                    cx.load_shares(p, cb.W2, cb.to_device(wl.lib_layout(W["W2"][1 + p]), dev))
+                    if cfg.gated:
+                        cx.load_shares(p, cb.WG, cb.to_device(wl.lib_layout(W["WG"][1 + p]), dev))
+            cx.synchronize()
+            mine = []
+            for j in range(2):
+                inp = make_inputs(cfg, seed, sparsity, 100 + 2 * k + j, T)
+                devt = [{kk: torch.from_numpy(v.view(np.int64)).to(dev) for kk, v in hp.items()} for hp in lib_tensors(inp)]
+                mine.append({"mask_dev": torch.from_numpy(inp["mask"]).to(dev), "dev": devt})
+            pctx.append((cx, sk))
+            psets.append(mine)
+
+        def piped_step(s):
+            cx, sk = pctx[s % C]
+            st = psets[s % C][(s // C) % 2]
+            with torch.cuda.stream(sk):
+                cx.set_mask(st["mask_dev"])
+                for p in (0, 1):
+                    for tid in UP_IDS:
+                        cx.bind_shares(p, tid, st["dev"][p][tid])
+                cx.ffn_up(T)
+                cx.truncate(cb.Z_UP)
+                for p in (0, 1):
+                    cx.bind_shares(p, cb.H, st["dev"][p][cb.H])
+                cx.ffn_down(T)
+                cx.truncate(cb.Y)
+
+        for s in range(max(2 * C, args.warmup)):
+            piped_step(s)
+        barrier()
+        launched0 = sum(cx.stats().kernel_launches for cx, _ in pctx)
+        p0, p1 = ev(), ev()
+        p0.record(tstream)
+        for s in range(args.steps):
+            piped_step(s)
+        for cx, sk in pctx:
+            done = torch.cuda.Event()
+            done.record(sk)
+            tstream.wait_event(done)
+        p1.record(tstream)
+        barrier()
+        (piped_ms,) = ranks.max_over_ranks([p0.elapsed_time(p1)], dev)
+        piped = {"in_flight": C, "ms_per_step": piped_ms / args.steps,
+                 "launches": int(sum(cx.stats().kernel_launches for cx, _ in pctx) - launched0),
+                 "value": ranks.whole_job_throughput(macs, world, args.steps, piped_ms), "unit": UNIT,
+                 "note": "C independent problems on C streams, inputs bound in place, whole region timed on the device"}
+        for cx, _ in pctx:
+            cx.close()
+    del W
+
     # ---- end-to-end timing (host buffers)
     for s in range(3):
         e2e_step(s)
@@ -458,8 +529,14 @@ def main():
     total_ms, e2e_ms = ranks.max_over_ranks([total_ms, e2e_ms], dev)
 
     if rank == 0:
-        ms_per_step = total_ms / args.steps
-        value = ranks.whole_job_throughput(macs, world, args.steps, total_ms)
+        single = {"ms_per_step": total_ms / args.steps,
+                  "value": ranks.whole_job_throughput(macs, world, args.steps, total_ms), "unit": UNIT,
+                  "note": "one problem at a time on one stream; sum over set_mask, ffn_up + truncate, ffn_down + "
+                          "truncate of CUDA-event pairs; 512 MiB written between steps to flush L2"}
+        if piped is not None:
+            ms_per_step, value = piped["ms_per_step"], piped["value"]
+        else:
+            ms_per_step, value = single["ms_per_step"], single["value"]
         phase = {name: {"ms_per_step": stats.phase_ms[k] / prof_steps, "launches_per_step":
                         stats.phase_launches[k] / prof_steps} for k, name in enumerate(cb.PHASE_NAMES)}
         comb_launch_ms = stats.phase_ms[3] / max(1, stats.phase_launches[3])
@@ -505,12 +582,18 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {"workload": workload_name(cfg, sparsity), "matmul_path": used_path,
-                       "l2": "512 MiB buffer written between steps, and 4 rotating input sets with different masks",
-                       "timed": "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream",
+                       "in_flight": args.in_flight,
+                       "l2": (f"{args.in_flight} contexts x 2 input sets with different masks rotate (inputs, gathered "
+                              "weight rows and intermediates of consecutive steps far exceed the L2); no flush"
+                              if piped is not None else
+                              "512 MiB buffer written between steps, and 4 rotating input sets with different masks"),
+                       "timed": ("every step = set_mask + bind inputs + ffn_up + truncate + ffn_down + truncate; the whole "
+                                 "region of K steps between two CUDA events" if piped is not None else
+                                 "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream"),
                        "token_masks": (f"per-token Bernoulli({args.token_masks}) masks over the active blocks, "
                                        f"{stats.n_components} component(s)" if args.token_masks > 0 else "none"),
                        "parallelism": f"independent FFN per GPU x{world}"},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(piped["launches"] if piped is not None else launches),
             "clocks": clocks,
             "e2e": {"value": ranks.whole_job_throughput(macs, world, args.steps, e2e_ms), "unit": UNIT,
                     "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
@@ -518,6 +601,7 @@ def main():
             "path_roofline": {"algorithmic_bytes": ffn_bytes(cfg, T, n), "algorithmic_macs": macs,
                               "hbm_gbs": hbm, "hbm_source": src, "roofline_ms": t_roof * 1e3,
                               "frac": t_roof * 1e3 / ms_per_step},
+            "single_problem": single,
             "phases": phase,
             "phases_note": f"separate pass of {prof_steps} steps with the per-phase event timers on",
             "wall_ms_per_step_incl_untimed": wall / args.steps * 1e3,

@@ -26,7 +26,9 @@
  *   - Pointers passed in belong to the caller.  `location` says where they
  *     point: COMET_DEVICE (memory of the context's GPU) or COMET_HOST (pinned or
  *     pageable host memory).  The library copies what it is given into memory
- *     it allocated at comet_init; nothing of the caller's is kept.
+ *     it allocated at comet_init; nothing of the caller's is kept (the one
+ *     exception is comet_bind_shares, which reads the caller's device memory in
+ *     place).
  *   - All work is enqueued on the CUDA stream given to comet_init.  Calls are
  *     asynchronous with respect to the host except comet_set_mask (it returns
  *     the public count n), comet_get/comet_load_shares with host pointers to
@@ -154,6 +156,17 @@ void comet_destroy(comet_ctx* ctx);
  * call. */
 int comet_load_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* ptr, int location,
                       int64_t rows, int64_t cols);
+
+/* As comet_load_shares, but nothing is copied: the library reads party `party`'s
+ * share of `tensor_id` in place from `dev_ptr` (device memory of the context's GPU,
+ * 16-byte aligned, rows*cols words) whenever a later call needs it.  The caller
+ * keeps the memory valid and unchanged until the last call that uses the tensor
+ * has completed on the stream (for a triple: the ffn call; for weights: as long as
+ * they stay bound).  A later comet_load_shares or comet_bind_shares of the same
+ * tensor replaces the binding; comet_set_mask drops the bindings of the triples
+ * and of H like their loaded state.  Same shape rules and errors as
+ * comet_load_shares, plus INVALID_ARG for an unaligned pointer. */
+int comet_bind_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* dev_ptr, int64_t rows, int64_t cols);
 
 /* Protocol 2 line 3 and Protocol 3 lines 1-5 under a block mask shared by all
  * tokens: turn the plaintext sparsity distribution (one byte per block, non-zero

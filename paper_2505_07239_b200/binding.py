@@ -31,7 +31,7 @@ EXPORTS = (
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
     "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
-    "comet_add_bias",
+    "comet_add_bias", "comet_bind_shares",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -73,6 +73,7 @@ def _load():
     lib.comet_destroy.argtypes = [vp]
     lib.comet_destroy.restype = None
     lib.comet_load_shares.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, i64, i64]
+    lib.comet_bind_shares.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, i64, i64]
     lib.comet_set_mask.argtypes = [vp, vp, ctypes.c_int, i32, ctypes.POINTER(i32)]
     lib.comet_set_token_mask.argtypes = [vp, vp, ctypes.c_int, i32, i32, ctypes.POINTER(i64)]
     lib.comet_get_components.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.POINTER(i32)]
@@ -156,6 +157,13 @@ class Comet:
         ptr, loc, _ = _ptr_loc(t)
         rows, cols = t.shape
         self._check(_lib.comet_load_shares(self._h, party, tensor_id, ptr, loc, rows, cols), "comet_load_shares")
+
+    def bind_shares(self, party: int, tensor_id: int, t):
+        """Use a CUDA tensor of 8-byte words in place (no copy); the caller keeps it alive and unchanged."""
+        ptr, loc, _ = _ptr_loc(t)
+        assert loc == DEVICE
+        rows, cols = t.shape
+        self._check(_lib.comet_bind_shares(self._h, party, tensor_id, ptr, rows, cols), "comet_bind_shares")
 
     def set_mask(self, mask) -> int:
         if isinstance(mask, np.ndarray):

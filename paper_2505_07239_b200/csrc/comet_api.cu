@@ -27,7 +27,8 @@ struct comet_ctx {
     int groups;                   // 1, 2 or 3 weight matrices stacked in the up-projection
     int64_t cap_T, cap_n;         // capacities
     int sm_count;
-    u64* buf[2][COMET_NUM_TENSORS];
+    u64* buf[2][COMET_NUM_TENSORS];   // where each tensor is read / written: the library's own buffer, or a bound one
+    u64* own[2][COMET_NUM_TENSORS];   // the library's own buffers (allocated in comet_init, freed in comet_destroy)
     int64_t cap_words[COMET_NUM_TENSORS];
     bool loaded[2][COMET_NUM_TENSORS];
     // limb path: blocked limb planes per party (left: E and V_i; right: B_i and F), and the device error flag
@@ -411,7 +412,10 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
         c->cap_words[id] = tensor_capacity(c, id);
         for (int p = 0; p < 2 && ok; ++p)
             if (c->cap_words[id] > 0)
-                ok = cudaMalloc((void**)&c->buf[p][id], (size_t)c->cap_words[id] * sizeof(u64)) == cudaSuccess;
+            {
+                ok = cudaMalloc((void**)&c->own[p][id], (size_t)c->cap_words[id] * sizeof(u64)) == cudaSuccess;
+                c->buf[p][id] = c->own[p][id];
+            }
     }
     c->path = cfg->matmul_path == COMET_PATH_AUTO ? COMET_PATH_LIMB : cfg->matmul_path;
     if (c->path == COMET_PATH_LIMB) {
@@ -477,7 +481,7 @@ void comet_destroy(comet_ctx* c) {
     cudaStreamSynchronize(c->stream);
     for (int id = 0; id < COMET_NUM_TENSORS; ++id)
         for (int p = 0; p < 2; ++p)
-            if (c->buf[p][id]) cudaFree(c->buf[p][id]);
+            if (c->own[p][id]) cudaFree(c->own[p][id]);
     if (c->side) cudaStreamSynchronize(c->side);
     for (int p = 0; p < 2; ++p)
         for (int w = 0; w < 2; ++w) {
@@ -507,11 +511,13 @@ void comet_destroy(comet_ctx* c) {
     delete c;
 }
 
-int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* ptr, int location, int64_t rows,
-                      int64_t cols) {
+// Shared by comet_load_shares (copy) and comet_bind_shares (use in place).
+static int set_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* ptr, int location, int64_t rows,
+                      int64_t cols, bool bind) {
     if (!c || (party != 0 && party != 1) || !is_input(tensor_id)) return COMET_ERR_INVALID_ARG;
     if (!ptr && rows * cols != 0) return COMET_ERR_INVALID_ARG;      // an empty tensor may come with a null pointer
     if (location != COMET_DEVICE && location != COMET_HOST) return COMET_ERR_INVALID_ARG;
+    if (bind && (location != COMET_DEVICE || (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0)) return COMET_ERR_INVALID_ARG;
     if (tensor_id == COMET_WG && c->groups < 2) return COMET_ERR_INVALID_ARG;
     if (tensor_id == COMET_W3 && c->groups != 3) return COMET_ERR_INVALID_ARG;
     const bool needs_mask = tensor_id == COMET_B_UP || tensor_id == COMET_C_UP || tensor_id == COMET_H ||
@@ -529,12 +535,26 @@ int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* pt
         if (rc != COMET_OK) return rc;
         c->dn_right_ready = false;
     }
-    if (rows * cols > 0)
-        COMET_CUDA(c, cudaMemcpyAsync(c->buf[party][tensor_id], ptr, (size_t)(rows * cols) * sizeof(u64),
-                                      copy_kind(location, true), c->stream));
+    if (bind && rows * cols > 0) {
+        c->buf[party][tensor_id] = const_cast<u64*>(reinterpret_cast<const u64*>(ptr));   // only ever read
+    } else {
+        c->buf[party][tensor_id] = c->own[party][tensor_id];
+        if (rows * cols > 0)
+            COMET_CUDA(c, cudaMemcpyAsync(c->buf[party][tensor_id], ptr, (size_t)(rows * cols) * sizeof(u64),
+                                          copy_kind(location, true), c->stream));
+    }
     c->loaded[party][tensor_id] = true;
     if (token_rows) c->tokens = (int32_t)rows;
     return COMET_OK;
+}
+
+int comet_load_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* ptr, int location, int64_t rows,
+                      int64_t cols) {
+    return set_shares(c, party, tensor_id, ptr, location, rows, cols, false);
+}
+
+int comet_bind_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* dev_ptr, int64_t rows, int64_t cols) {
+    return set_shares(c, party, tensor_id, dev_ptr, COMET_DEVICE, rows, cols, true);
 }
 
 int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_t n_blocks, int32_t* n_active_out) {
@@ -585,7 +605,10 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     c->tmask_set = false;             // a token mask refines one block mask
     c->up_done = c->down_done = false;
     for (int p = 0; p < 2; ++p)
-        for (int id = COMET_A_UP; id <= COMET_C_DN; ++id) c->loaded[p][id] = false;
+        for (int id = COMET_A_UP; id <= COMET_C_DN; ++id) {
+            c->loaded[p][id] = false;
+            c->buf[p][id] = c->own[p][id];          // a binding ends with the mask it was made under
+        }
     c->stats.n_active = c->n_active;
     c->stats.n_active_blocks = blocks;
     *n_active_out = c->n_active;

@@ -220,3 +220,53 @@ def test_errors_are_status_codes(hz):
     # the context is still usable afterwards
     ctx.close()
     hz.run_and_compare_full(cfg, seed=14, float_report=False)
+
+
+def test_bound_inputs_give_the_same_bits_as_copied_ones(hz):
+    """comet_bind_shares: inputs read in place from the caller's device memory."""
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["opt125m"]
+    T, d, seed = cfg.tokens, cfg.d_model, 15
+    W = wl.model_shares(cfg, seed, plain=False)
+    mask = wl.block_mask(cfg, seed)
+    _, X0, X1 = wl.activation_shares(cfg, seed)
+    outs = []
+    for bind in (False, True):
+        ctx = hz.make_context(cfg, T)
+        keep = []                                     # bound tensors stay alive until the context is closed
+
+        def put(p, tid, arr):
+            t = cb.to_device(arr)
+            if bind:
+                keep.append(t)
+                ctx.bind_shares(p, tid, t)
+            else:
+                ctx.load_shares(p, tid, t)
+
+        for p in (0, 1):
+            put(p, cb.W1, wl.lib_layout(W["W1"][1 + p]))
+            put(p, cb.W2, wl.lib_layout(W["W2"][1 + p]))
+            put(p, cb.X, (X0, X1)[p])
+        n = ctx.set_mask(mask)
+        tri = wl.dealer_triple(seed, "u", T, d, n, valid=False)
+        trd = wl.dealer_triple(seed, "d", T, n, d, valid=False)
+        _, H0, H1 = wl.hidden_shares(cfg, seed, n)
+        for p in (0, 1):
+            put(p, cb.A_UP, tri["A"][1 + p]); put(p, cb.B_UP, wl.lib_layout(tri["B"][1 + p])); put(p, cb.C_UP, tri["C"][1 + p])
+            put(p, cb.A_DN, trd["A"][1 + p]); put(p, cb.B_DN, wl.lib_layout(trd["B"][1 + p])); put(p, cb.C_DN, trd["C"][1 + p])
+            put(p, cb.H, (H0, H1)[p])
+        ctx.ffn_up(T)
+        ctx.truncate(cb.Z_UP)
+        ctx.ffn_down(T)
+        ctx.truncate(cb.Y)
+        outs.append([ctx.get(p, t, s) for p in (0, 1) for t, s in ((cb.Z_UP, (T, n)), (cb.Y, (T, d)), (cb.E_DN, (T, n)))])
+        if bind:
+            # an unaligned pointer is refused, and a new mask ends the bindings of the triples
+            t = torch.zeros(T * d + 1, dtype=torch.int64, device="cuda")
+            assert cb.library().comet_bind_shares(ctx._h, 0, cb.X, t.data_ptr() + 8, T, d) == -1
+            ctx.set_mask(mask)
+            assert cb.library().comet_ffn_up(ctx._h, T) == -3
+        ctx.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
