@@ -533,7 +533,11 @@ def main():
                   "value": ranks.whole_job_throughput(macs, world, args.steps, total_ms), "unit": UNIT,
                   "note": "one problem at a time on one stream; sum over set_mask, ffn_up + truncate, ffn_down + "
                           "truncate of CUDA-event pairs; 512 MiB written between steps to flush L2"}
-        if piped is not None:
+        # Two issue policies are measured in this run; the headline is the faster one (large dense problems gain
+        # nothing from sharing the GPU, small sparse ones hide their memory-side kernels under another problem's
+        # tensor-core kernel), and both are reported.
+        use_piped = piped is not None and piped["value"] > single["value"]
+        if use_piped:
             ms_per_step, value = piped["ms_per_step"], piped["value"]
         else:
             ms_per_step, value = single["ms_per_step"], single["value"]
@@ -582,18 +586,18 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {"workload": workload_name(cfg, sparsity), "matmul_path": used_path,
-                       "in_flight": args.in_flight,
+                       "in_flight": args.in_flight if use_piped else 1,
                        "l2": (f"{args.in_flight} contexts x 2 input sets with different masks rotate (inputs, gathered "
                               "weight rows and intermediates of consecutive steps far exceed the L2); no flush"
-                              if piped is not None else
+                              if use_piped else
                               "512 MiB buffer written between steps, and 4 rotating input sets with different masks"),
                        "timed": ("every step = set_mask + bind inputs + ffn_up + truncate + ffn_down + truncate; the whole "
-                                 "region of K steps between two CUDA events" if piped is not None else
+                                 "region of K steps between two CUDA events" if use_piped else
                                  "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream"),
                        "token_masks": (f"per-token Bernoulli({args.token_masks}) masks over the active blocks, "
                                        f"{stats.n_components} component(s)" if args.token_masks > 0 else "none"),
                        "parallelism": f"independent FFN per GPU x{world}"},
-            "gpu_launches": int(piped["launches"] if piped is not None else launches),
+            "gpu_launches": int(piped["launches"] if use_piped else launches),
             "clocks": clocks,
             "e2e": {"value": ranks.whole_job_throughput(macs, world, args.steps, e2e_ms), "unit": UNIT,
                     "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
@@ -602,6 +606,7 @@ def main():
                               "hbm_gbs": hbm, "hbm_source": src, "roofline_ms": t_roof * 1e3,
                               "frac": t_roof * 1e3 / ms_per_step},
             "single_problem": single,
+            "problems_in_flight": piped,
             "phases": phase,
             "phases_note": f"separate pass of {prof_steps} steps with the per-phase event timers on",
             "wall_ms_per_step_incl_untimed": wall / args.steps * 1e3,
