@@ -168,7 +168,7 @@ int comet_load_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* 
  * comet_load_shares, plus INVALID_ARG for an unaligned pointer. */
 int comet_bind_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* dev_ptr, int64_t rows, int64_t cols);
 
-/* Protocol 2 line 3 and Protocol 3 lines 1-5 under a block mask shared by all
+/* The index-set steps of Protocol 2 and Protocol 3 under a block mask shared by all
  * tokens: turn the plaintext sparsity distribution (one byte per block, non-zero
  * = active) into the ascending list of active blocks, i.e. the index set I.
  * `n_blocks` must equal d_ff / block.  Returns the number of active NEURONS in
@@ -204,7 +204,7 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * Theorem 1's minimum, the dot-product count is not when there are several
  * components.
  *
- * Down-projection, Protocol 3, lines 1-5: the sparsity distribution of the hidden
+ * Down-projection, Protocol 3 (its row sets R_j): the sparsity distribution of the hidden
  * state.  `token_mask` is [tokens, n_active_blocks]
  * bytes, row-major; byte (t, b) non-zero means that the neurons of the b-th ACTIVE
  * block (in the ascending order of comet_get_index) are non-zeros of token t, so

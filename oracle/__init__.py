@@ -174,7 +174,7 @@ def simm(X, Y, I, A, B, C):
 
 
 def components_dfs(S):
-    """Connected components of the bipartite graph of S [T, n] (Protocol 2 line 1).
+    """Connected components of the bipartite graph of S [T, n] (the first step of Protocol 2).
     Returns (row_comp [T], col_comp [n], L); -1 marks a node without an edge."""
     S = np.ascontiguousarray(S, dtype=np.uint8)
     T, n = S.shape

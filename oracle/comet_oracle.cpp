@@ -45,8 +45,8 @@ void orc_reconstruct(const u64* s0, const u64* s1, u64* out, size_t count) {
 }
 
 // ---------------------------------------------------------------------------
-// Index sets.  Protocol 2 line 3 (I_y of the single connected component) and
-// Protocol 3 lines 1-5 (the nonzero columns j) for a sparsity distribution
+// Index sets.  Protocol 2's I_y of the single connected component and
+// Protocol 3's nonzero columns j, for a sparsity distribution
 // that is one block mask shared by all tokens: neuron j is active iff
 // block_mask[j / bs] != 0.  With `groups` = 2 (gated FFN, Y = [W_gate || W_up]
 // of width 2*D) the set is I followed by D + I.  Ascending order.
@@ -61,19 +61,19 @@ int orc_index_set(const uint8_t* block_mask, int nb, int bs, int groups, int32_t
     return count;
 }
 
-// Protocol 2 line 5: IndexCols(Y, I_y).  Y is [K, D]; out is [K, n].
+// Protocol 2: IndexCols(Y, I_y).  Y is [K, D]; out is [K, n].
 void orc_index_cols(const u64* Y, int K, int D, const int32_t* I, int n, u64* out) {
     for (int k = 0; k < K; ++k)
         for (int c = 0; c < n; ++c) out[(size_t)k * n + c] = Y[(size_t)k * D + I[c]];
 }
 
-// Protocol 3 line 9: IndexRow(Y, j) for every j in I.  Y is [D, N]; out is [n, N].
+// Protocol 3: IndexRow(Y, j) for every j in I.  Y is [D, N]; out is [n, N].
 void orc_index_rows(const u64* Y, int N, const int32_t* I, int n, u64* out) {
     for (int r = 0; r < n; ++r)
         for (int c = 0; c < N; ++c) out[(size_t)r * N + c] = Y[(size_t)I[r] * N + c];
 }
 
-// Protocol 2 line 8, Merge: compact columns back to a dense [T, D] layout,
+// Protocol 2, Merge: compact columns back to a dense [T, D] layout,
 // zero (in this share) at every inactive position.
 void orc_merge_cols(const u64* R, int T, int n, const int32_t* I, int D, u64* Z) {
     for (size_t t = 0; t < (size_t)T * D; ++t) Z[t] = 0;
@@ -167,14 +167,14 @@ void orc_somm(int T, int K, int Dy, const int32_t* I, int n,
               const u64* C0, const u64* C1,
               u64* E0, u64* E1, u64* F0, u64* F1, u64* R0, u64* R1) {
     std::vector<u64> Yt0((size_t)K * n), Yt1((size_t)K * n);
-    orc_index_cols(Y0, K, Dy, I, n, Yt0.data());          // line 5
+    orc_index_cols(Y0, K, Dy, I, n, Yt0.data());          // IndexCols
     orc_index_cols(Y1, K, Dy, I, n, Yt1.data());
-    orc_pi_matmul(T, K, n, X0, X1, Yt0.data(), Yt1.data(), // line 6
+    orc_pi_matmul(T, K, n, X0, X1, Yt0.data(), Yt1.data(), // Pi_MatMul
                   A0, A1, B0, B1, C0, C1, E0, E1, F0, F1, R0, R1);
 }
 
 // ---------------------------------------------------------------------------
-// Protocol 2 line 1: the connected components {G_t} of the bipartite graph whose
+// Protocol 2, first step: the connected components {G_t} of the bipartite graph whose
 // nodes are the T rows of X and the n (compact) columns of Y and whose edges are
 // the non-zeros of the sparsity distribution S [T, n], found by depth-first
 // search.  Components are numbered in the order in which a scan over the rows
@@ -219,8 +219,8 @@ int orc_components_dfs(int T, int n, const uint8_t* S, int32_t* row_comp, int32_
 // ---------------------------------------------------------------------------
 // Protocol 2 (SOMM) in general.  Y is [K, Dy]; compact column c stands for
 // column I[c] of Y; S is the sparsity distribution of the compact result [T, n].
-// For every component: I_x, I_y (line 3), IndexRows / IndexCols (lines 4-5),
-// Pi_MatMul with that component's own triple (line 6), and Merge (line 8) puts
+// For every component: the index sets I_x, I_y, IndexRows / IndexCols,
+// Pi_MatMul with that component's own triple, and Merge puts
 // the result block at (I_x, I_y); every other entry of the result is zero in
 // both shares, and rows / columns outside all components are neither masked nor
 // sent (their message rows stay zero).  The per-component triples arrive
@@ -237,7 +237,7 @@ int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uin
                         const u64* C0, const u64* C1,
                         u64* E0, u64* E1, u64* F0, u64* F1, u64* R0, u64* R1,
                         int32_t* row_comp, int32_t* col_comp, long long* cost) {
-    const int L = orc_components_dfs(T, n, S, row_comp, col_comp);            // line 1
+    const int L = orc_components_dfs(T, n, S, row_comp, col_comp);            // the components
     const u64* Xs[2] = {X0, X1};
     const u64* Ys[2] = {Y0, Y1};
     const u64* As[2] = {A0, A1};
@@ -256,7 +256,7 @@ int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uin
     for (int t = 0; t < L; ++t) {
         Ix.clear();
         Iy.clear();
-        for (int r = 0; r < T; ++r) if (row_comp[r] == t) Ix.push_back(r);    // line 3
+        for (int r = 0; r < T; ++r) if (row_comp[r] == t) Ix.push_back(r);    // I_x, I_y
         for (int c = 0; c < n; ++c) if (col_comp[c] == t) Iy.push_back(c);
         const int tx = (int)Ix.size(), ty = (int)Iy.size();
         cost[0] += tx + ty;
@@ -266,12 +266,12 @@ int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uin
             xt[i].resize((size_t)tx * K); at[i].resize((size_t)tx * K); et[i].resize((size_t)tx * K);
             yt[i].resize((size_t)K * ty); bt[i].resize((size_t)K * ty); ft[i].resize((size_t)K * ty);
             ct[i].resize((size_t)tx * ty); rt[i].resize((size_t)tx * ty);
-            for (int a = 0; a < tx; ++a)                                     // line 4: IndexRows
+            for (int a = 0; a < tx; ++a)                                     // IndexRows
                 for (int k = 0; k < K; ++k) {
                     xt[i][(size_t)a * K + k] = Xs[i][(size_t)Ix[a] * K + k];
                     at[i][(size_t)a * K + k] = As[i][(size_t)Ix[a] * K + k];
                 }
-            for (int k = 0; k < K; ++k)                                      // line 5: IndexCols
+            for (int k = 0; k < K; ++k)                                      // IndexCols
                 for (int b = 0; b < ty; ++b) {
                     yt[i][(size_t)k * ty + b] = Ys[i][(size_t)k * Dy + I[Iy[b]]];
                     bt[i][(size_t)k * ty + b] = Bs[i][(size_t)k * n + Iy[b]];
@@ -279,10 +279,10 @@ int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uin
             for (int a = 0; a < tx; ++a)
                 for (int b = 0; b < ty; ++b) ct[i][(size_t)a * ty + b] = Cs[i][(size_t)Ix[a] * n + Iy[b]];
         }
-        orc_pi_matmul(tx, K, ty, xt[0].data(), xt[1].data(), yt[0].data(), yt[1].data(),             // line 6
+        orc_pi_matmul(tx, K, ty, xt[0].data(), xt[1].data(), yt[0].data(), yt[1].data(),             // Pi_MatMul
                       at[0].data(), at[1].data(), bt[0].data(), bt[1].data(), ct[0].data(), ct[1].data(),
                       et[0].data(), et[1].data(), ft[0].data(), ft[1].data(), rt[0].data(), rt[1].data());
-        for (int i = 0; i < 2; ++i) {                                        // line 8: Merge
+        for (int i = 0; i < 2; ++i) {                                        // Merge
             for (int a = 0; a < tx; ++a)
                 for (int k = 0; k < K; ++k) Es[i][(size_t)Ix[a] * K + k] = et[i][(size_t)a * K + k];
             for (int k = 0; k < K; ++k)
@@ -300,7 +300,7 @@ int orc_somm_components(int T, int K, int Dy, const int32_t* I, int n, const uin
 // column (token-shared mask).  Each column's Pi_MatMul is the outer product of
 // a T-vector with row I[c] of Y [D, N]; it uses column c of A' [T,n] and row c
 // of B' [n,N] as its (a_j, b_j), and the dealer's C' [T,N] is the sum over j
-// of the per-column c_j = a_j b_j^T, added once in Merge&Sum (line 12).
+// of the per-column c_j = a_j b_j^T, added once in Merge&Sum.
 // Outputs: messages E_i [T,n], F_i [n,N]; result Z_i [T,N].
 // ---------------------------------------------------------------------------
 void orc_simm(int T, int n, int N, const int32_t* I,
@@ -319,17 +319,17 @@ void orc_simm(int T, int n, int N, const int32_t* I,
     for (int i = 0; i < 2; ++i)
         for (size_t t = 0; t < (size_t)T * N; ++t) Zs[i][t] = Cs[i][t];
     std::vector<u64> e(T), f(N);
-    for (int c = 0; c < n; ++c) {                    // lines 6-11, one column j = I[c]
+    for (int c = 0; c < n; ++c) {                    // the protocol's loop body, one column j = I[c]
         int j = I[c];
         for (int i = 0; i < 2; ++i) {
-            for (int r = 0; r < T; ++r)              // lines 7-8 + masking of x''
+            for (int r = 0; r < T; ++r)              // IndexCol, IndexRows + masking of x''
                 Es[i][(size_t)r * n + c] = Xs[i][(size_t)r * n + c] - As[i][(size_t)r * n + c];
-            for (int q = 0; q < N; ++q)              // line 9 + masking of y
+            for (int q = 0; q < N; ++q)              // IndexRow + masking of y
                 Fs[i][(size_t)c * N + q] = Ys[i][(size_t)j * N + q] - Bs[i][(size_t)c * N + q];
         }
         for (int r = 0; r < T; ++r) e[r] = E0[(size_t)r * n + c] + E1[(size_t)r * n + c];
         for (int q = 0; q < N; ++q) f[q] = F0[(size_t)c * N + q] + F1[(size_t)c * N + q];
-        for (int i = 0; i < 2; ++i)                  // line 10 (Eq. 1 without c_j) + line 12 sum
+        for (int i = 0; i < 2; ++i)                  // Pi_MatMul (Eq. 1 without c_j) + the sum of Merge&Sum
             for (int r = 0; r < T; ++r) {
                 u64 a = As[i][(size_t)r * n + c];
                 for (int q = 0; q < N; ++q) {
@@ -343,7 +343,7 @@ void orc_simm(int T, int n, int N, const int32_t* I,
 // ---------------------------------------------------------------------------
 // Protocol 3 (SIMM) with a sparsity distribution S of X that differs from row
 // to row: S is [T, n] over the compact columns (non-zero byte = X[r, c] is a
-// non-zero), so R_j of compact column c is {r : S[r, c] != 0} (lines 1-5).
+// non-zero), so R_j of compact column c is {r : S[r, c] != 0} (the protocol's first loop).
 // A column with empty R_j is not a "nonzero column": nothing of it is masked,
 // sent or multiplied, and its message rows stay zero.  For the others, only the
 // entries of x'' = X[R_j, j] are masked and sent (E is zero off the support),
@@ -376,20 +376,20 @@ long long orc_simm_rowsets(int T, int n, int N, const int32_t* I, const uint8_t*
     for (int c = 0; c < n; ++c) {
         R.clear();
         for (int r = 0; r < T; ++r)
-            if (S[(size_t)r * n + c] != 0) R.push_back(r);         // line 3: R_j
+            if (S[(size_t)r * n + c] != 0) R.push_back(r);         // R_j
         if (R.empty()) continue;                                    // not a nonzero column
         const int j = I[c];
         masked += (long long)R.size();
         e.assign(R.size(), 0);
         for (int i = 0; i < 2; ++i) {
-            for (size_t k = 0; k < R.size(); ++k)                   // lines 7-8 + masking of x''
+            for (size_t k = 0; k < R.size(); ++k)                   // IndexCol, IndexRows + masking of x''
                 Es[i][(size_t)R[k] * n + c] = Xs[i][(size_t)R[k] * n + c] - As[i][(size_t)R[k] * n + c];
-            for (int q = 0; q < N; ++q)                             // line 9 + masking of y
+            for (int q = 0; q < N; ++q)                             // IndexRow + masking of y
                 Fs[i][(size_t)c * N + q] = Ys[i][(size_t)j * N + q] - Bs[i][(size_t)c * N + q];
         }
         for (size_t k = 0; k < R.size(); ++k) e[k] = E0[(size_t)R[k] * n + c] + E1[(size_t)R[k] * n + c];
         for (int q = 0; q < N; ++q) f[q] = F0[(size_t)c * N + q] + F1[(size_t)c * N + q];
-        for (int i = 0; i < 2; ++i)                                 // line 10 and the sum of line 12
+        for (int i = 0; i < 2; ++i)                                 // Pi_MatMul and the sum of Merge&Sum
             for (size_t k = 0; k < R.size(); ++k) {
                 const u64 a = As[i][(size_t)R[k] * n + c];
                 for (int q = 0; q < N; ++q) {

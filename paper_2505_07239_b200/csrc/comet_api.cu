@@ -331,7 +331,7 @@ int launch_combine(comet_ctx* c, int M, int N, int K, int idE, int idF, int idA,
     return COMET_OK;
 }
 
-// Protocol 2 line 8 under a token mask: entries of the compact result outside the component blocks become zero.
+// The Merge step of Protocol 2 under a token mask: entries of the compact result outside the component blocks become zero.
 int somm_merge(comet_ctx* c, int tokens) {
     if (!c->tmask_set) return COMET_OK;
     const int cols = c->groups * c->n_active;
@@ -632,7 +632,7 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     const size_t bytes = (size_t)tokens * (size_t)n_active_blocks;
     COMET_CUDA(c, cudaMemcpyAsync(c->d_tmask, token_mask, bytes, copy_kind(location, true), c->stream));
     comet::count_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, (long long)bytes, c->h_masked_dev);
-    // Protocol 2 line 1: the connected components the up-projection is partitioned into
+    // Protocol 2, first step: the connected components the up-projection is partitioned into
     comet::token_components_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, tokens, n_active_blocks, c->d_row_label,
                                                              c->d_blk_label, c->h_masked_dev + 1);
     c->stats.kernel_launches += 2;

@@ -99,7 +99,7 @@ __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows,
 }
 
 // ---------------------------------------------------------------------------
-// Before the exchange (Section 2.1 "Multiplication"; Protocol 2 line 5, Protocol 3 line 9), one launch:
+// Before the exchange (Section 2.1 "Multiplication"; IndexCols of Protocol 2, IndexRow of Protocol 3), one launch:
 //   left  blocks: E_i = X_i - A_i, elementwise;
 //   right tiles : F_i = gather(W_i) - B_i written as the message, and the blocked limb planes of the party's
 //                 own B_i (it is in registers anyway, so it is not read a second time later).

@@ -18,7 +18,7 @@ struct PartyOut {
 
 // ---------------------------------------------------------------------------
 // K1: block mask -> ascending list of active block ids and their count.
-// Protocol 2 line 3 / Protocol 3 lines 1-5 for a token-shared block mask.
+// The index-set steps of Protocol 2 (I_x, I_y) and Protocol 3 (the non-zero columns) for a token-shared block mask.
 // One CTA of 1024 threads walks the mask 1024 blocks at a time: a warp ballot
 // ranks each active block inside its warp, a shuffle scan over the 32 warp
 // totals gives each warp's base, and a running base carries across chunks.
@@ -100,7 +100,7 @@ open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, cons
 }
 
 // ---------------------------------------------------------------------------
-// Protocol 2 line 1 on the GPU: connected components of the bipartite graph
+// The first step of Protocol 2 on the GPU: connected components of the bipartite graph
 // (token rows) x (active blocks) whose edges are the non-zero bytes of the
 // per-token mask S [T, nab].  The paper uses depth-first search; here one CTA
 // propagates minimum labels back and forth (block <- min over its tokens,
@@ -168,7 +168,7 @@ token_components_kernel(const uint8_t* __restrict__ S, int T, int nab, int32_t* 
     }
 }
 
-// Protocol 2 line 8 (Merge) on the compact result [T, cols]: an entry whose token and block are not in the same
+// The Merge step of Protocol 2 on the compact result [T, cols]: an entry whose token and block are not in the same
 // component is no part of any result block and is zero in both shares.  Compact column c belongs to active block
 // (c mod n) / bs.  `pairs` = 16-byte word pairs per party.
 __global__ void __launch_bounds__(256)
@@ -205,7 +205,7 @@ count_mask_kernel(const uint8_t* __restrict__ mask, long long count, long long* 
 
 // ---------------------------------------------------------------------------
 // K3 (up): F_i[c, :] = W_i[neuron(c), :] - B_i[c, :].  The paper's IndexCols
-// (Protocol 2 line 5) followed by [e]_i = [y]_i - [b]_i; with weights stored
+// (Protocol 2) followed by [e]_i = [y]_i - [b]_i; with weights stored
 // output-feature-major the column gather is a gather of whole rows of d words.
 // Compact row c in [0, g*n): group = c / n selects the weight matrix (WG, W1,
 // W3 in that order when there are several), j = c mod n, neuron = ids[j / bs] * bs + j mod bs.
@@ -238,7 +238,7 @@ open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs Wg2, PartyPtrs B
 
 // ---------------------------------------------------------------------------
 // K3 (down): F'_i[q, c] = W2_i[q, neuron(c)] - B'_i[q, c].  The paper's
-// IndexRow (Protocol 3 line 9) on the stored transpose [d, D] is a gather of
+// IndexRow (Protocol 3) on the stored transpose [d, D] is a gather of
 // bs-word strips (256 or 512 contiguous bytes) out of every row q.
 // Flat index over (q, c/2); consecutive threads walk consecutive pairs of a row.
 // ---------------------------------------------------------------------------
