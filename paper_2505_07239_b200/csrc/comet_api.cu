@@ -59,6 +59,7 @@ struct comet_ctx {
     int32_t* d_count;             // {count, error flag of the bounded waits}
     int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
     int32_t* h_count_dev;         // device-side address of h_count
+    int top_priority;             // the device's highest stream / launch priority (numerically lowest)
     int32_t ticket;               // sequence number of the last compaction launch (echoed in h_count[2])
     bool mask_set;
     int32_t n_active, n_active_blocks;
@@ -290,8 +291,22 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
         PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
-        if (few) comet::combine_limb_few_kernel<<<grid, lf::THREADS, lf::SMEM_BYTES, c->stream>>>(a);
-        else comet::combine_limb_kernel<<<grid, lb::THREADS, lb::SMEM_BYTES, c->stream>>>(a);
+        // The persistent kernel needs a slot on every SM.  With the device's highest scheduling priority its CTAs
+        // get the slots that free up before the memory-side CTAs of other contexts queued beside it do, so the
+        // tensor cores do not wait behind work that could as well run under them.
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof(lc));
+        lc.gridDim = dim3(grid);
+        lc.blockDim = dim3(few ? lf::THREADS : lb::THREADS);
+        lc.dynamicSmemBytes = few ? lf::SMEM_BYTES : lb::SMEM_BYTES;
+        lc.stream = c->stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributePriority;
+        attr.val.priority = c->top_priority;
+        lc.attrs = &attr;
+        lc.numAttrs = 1;
+        if (few) COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_few_kernel, a));
+        else COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_kernel, a));
     }
     c->stats.kernel_launches += 1;
     c->stats.matmul_path = COMET_PATH_LIMB;
@@ -406,6 +421,11 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
         delete c->free_events;
         delete c;
         return COMET_ERR_CUDA;
+    }
+    {
+        int least = 0, greatest = 0;
+        if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) cudaGetLastError();
+        c->top_priority = greatest;
     }
     bool ok = true;
     for (int id = 0; id < COMET_NUM_TENSORS && ok; ++id) {
