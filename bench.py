@@ -93,6 +93,14 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def warm(self, step, limit_s: float = 3.0):
+        """Keep the device under the timed load (untimed calls of `step`) until the first sample has
+        arrived, so that a timed region shorter than the tool's start-up still has samples inside it."""
+        t0, s = time.perf_counter(), 0
+        while self.proc is not None and not self.lines and time.perf_counter() - t0 < limit_s:
+            step(s)
+            s += 1
+
     def _pump(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
@@ -432,11 +440,13 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        sampler.warm(lambda s: device_step(s, False))
+    barrier()
     wall0 = time.perf_counter()
     events = [device_step(args.warmup + s, True) for s in range(args.steps)]
     barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop() if rank == 0 else None
+    clocks_single = sampler.stop() if rank == 0 else None
     launches = ctx.stats().kernel_launches - launches0
     step_ms = [e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) + e[4].elapsed_time(e[5]) for e in events]
     total_ms = float(sum(step_ms))
@@ -497,6 +507,11 @@ def main():
             piped_step(s)
         barrier()
         launched0 = sum(cx.stats().kernel_launches for cx, _ in pctx)
+        sampler2 = ClockSampler(local)
+        if rank == 0:
+            sampler2.start()
+            sampler2.warm(piped_step)
+        barrier()
         p0, p1 = ev(), ev()
         p0.record(tstream)
         for s in range(args.steps):
@@ -507,6 +522,7 @@ def main():
             tstream.wait_event(done)
         p1.record(tstream)
         barrier()
+        clocks_piped = sampler2.stop() if rank == 0 else None
         (piped_ms,) = ranks.max_over_ranks([p0.elapsed_time(p1)], dev)
         piped = {"in_flight": C, "ms_per_step": piped_ms / args.steps,
                  "launches": int(sum(cx.stats().kernel_launches for cx, _ in pctx) - launched0),
@@ -598,7 +614,7 @@ def main():
                                        f"{stats.n_components} component(s)" if args.token_masks > 0 else "none"),
                        "parallelism": f"independent FFN per GPU x{world}"},
             "gpu_launches": int(piped["launches"] if use_piped else launches),
-            "clocks": clocks,
+            "clocks": clocks_piped if use_piped else clocks_single,
             "e2e": {"value": ranks.whole_job_throughput(macs, world, args.steps, e2e_ms), "unit": UNIT,
                     "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "roofline": roof,
