@@ -309,6 +309,19 @@ def beaver_mul(x, y, a, b, c):
     return {"D": (outs[0], outs[1]), "E": (outs[2], outs[3]), "Z": (outs[4], outs[5])}
 
 
+def truncate_pair(z, r, rp, frac_bits: int):
+    """Truncation with a dealer's pair (r, r' = floor(r / 2^f)) for both parties: z, r, rp are pairs of
+    equally shaped uint64 arrays.  Returns dict with the messages M = z - r (pair) and the result OUT (pair)."""
+    arrs = _pairs(z, r, rp)
+    shape = arrs[0].shape
+    for v in arrs:
+        assert v.shape == shape
+    outs = [np.empty(shape, U64) for _ in range(4)]
+    lib().orc_truncate_pair(ctypes.c_size_t(arrs[0].size), ctypes.c_int(frac_bits), *[_p(v) for v in arrs],
+                            *[_p(o) for o in outs])
+    return {"M": (outs[0], outs[1]), "OUT": (outs[2], outs[3])}
+
+
 def add_bias(Zi, bias_i):
     """One party's local addition of its bias share [N] to every row of its share [T, N]."""
     Zi, bias_i = _u64(Zi), _u64(bias_i)

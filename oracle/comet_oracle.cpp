@@ -28,6 +28,11 @@
 // example, by z_1 + z_2 = pi(x) against numpy indexing, by the operator
 // identities rho_1 o tau_2 = rho_2 o tau_1 = pi, by exhaustive permutations of
 // three elements and by unshuffle(shuffle(x)) = x.
+// Truncation with a dealer's pair (not a protocol of the paper; built from its
+// Reconstruction and Addition, Section 2.1): pinned by the closed forms r = 0 and
+// "low f bits of z and r all zero", by the {-1,0}-ulp invariant against Python
+// big integers, by [out]_0 = [r']_0 (the public term goes to the party with
+// factor i), and by hand-computed words.  Parity unpinned by the paper itself.
 
 #include <cstddef>
 #include <cstdint>
@@ -510,6 +515,32 @@ void orc_beaver_mul(size_t count, const u64* x0, const u64* x1, const u64* y0, c
 void orc_add_bias(int T, int N, const u64* Zi, const u64* bias_i, u64* out) {
     for (int r = 0; r < T; ++r)
         for (int c = 0; c < N; ++c) out[(size_t)r * N + c] = Zi[(size_t)r * N + c] + bias_i[c];
+}
+
+// ---------------------------------------------------------------------------
+// Truncation by f bits with a dealer's pair.  The paper has no truncation
+// protocol; this one is put together from two of its primitives (Section 2.1):
+// the dealer shares a uniform word r and r' = floor(r / 2^f) (r read as a signed
+// 64-bit integer); "Reconstruction" opens m = z - r from the messages
+// [m]_i = [z]_i - [r]_i; "Addition" with the public value c = floor(m / 2^f)
+// (m read as signed) gives [out]_i = [r']_i + i*c.
+// out_0 + out_1 = floor(m/2^f) + floor(r/2^f), which is floor(z/2^f) or one less
+// unless m + r leaves the signed range (probability about |z| / 2^64).
+// ---------------------------------------------------------------------------
+void orc_truncate_pair(size_t count, int f, const u64* z0, const u64* z1, const u64* r0, const u64* r1,
+                       const u64* rp0, const u64* rp1, u64* m0, u64* m1, u64* out0, u64* out1) {
+    for (size_t t = 0; t < count; ++t) {
+        m0[t] = z0[t] - r0[t];
+        m1[t] = z1[t] - r1[t];
+    }
+    for (size_t t = 0; t < count; ++t) {
+        const u64 m = m0[t] + m1[t];                        // reconstruction
+        // floor division of the signed reading by 2^f, written without relying on >> of a negative value
+        const bool neg = (m >> 63) != 0;
+        const u64 c = neg ? ~((~m) >> f) : (m >> f);
+        out0[t] = rp0[t];                                   // i = 0: no public term
+        out1[t] = rp1[t] + c;                               // i = 1 adds the public value
+    }
 }
 
 }  // extern "C"

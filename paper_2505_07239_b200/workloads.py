@@ -361,6 +361,15 @@ def dealer_triple_elementwise(seed: int, stream: str, shape) -> dict:
             "c": (c, *split_shares(c, seed, stream + "/c"))}
 
 
+def dealer_truncation_pair(seed: int, stream: str, shape, frac_bits: int) -> dict:
+    """The dealer's pair for one truncation by `frac_bits`: r uniform in the ring and r' = floor(r / 2^f) with r
+    read as a signed 64-bit integer, each split into two uniform shares.  Returns {"r": (r, r0, r1), "rp": ...}."""
+    count = int(np.prod(shape))
+    r = random_u64(seed, stream + "/r", count).reshape(shape)
+    rp = (r.view(np.int64) >> np.int64(frac_bits)).view(np.uint64)
+    return {"r": (r, *split_shares(r, seed, stream + "/r")), "rp": (rp, *split_shares(rp, seed, stream + "/rp"))}
+
+
 def random_permutation(seed: int, stream: str, count: int) -> np.ndarray:
     """Seeded uniform permutation of range(count) (rank of random keys), int32."""
     keys = random_u64(seed, stream, count)
