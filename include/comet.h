@@ -316,6 +316,22 @@ int comet_invert_permutation(void* cuda_stream, const int32_t* perm, int32_t* in
  * Errors: INVALID_ARG (null pointer), SHAPE (rows or cols < 1), CUDA. */
 int comet_add_bias(void* cuda_stream, uint64_t* const Z[2], const uint64_t* const bias[2], int64_t rows, int64_t cols);
 
+/* Truncation by frac_bits with a dealer's pair, for both parties, in place.  The
+ * paper has no truncation protocol; this one consists of two of its primitives
+ * (Section 2.1): the dealer shares a uniform word r and r' = floor(r / 2^f), r
+ * read as a signed 64-bit integer; "Reconstruction" opens m = z - r from the
+ * messages M[i] = Z[i] - R[i]; "Addition" of the public value floor(m / 2^f), m
+ * read as signed, to the shares of r' gives Z[i] <- RP[i] + i * floor(m / 2^f).
+ * Z[0] + Z[1] afterwards is floor(z / 2^f) or one less, unless m + r leaves the
+ * signed 64-bit range (probability about |z| / 2^64).  The alternative to
+ * comet_truncate, which needs no dealer material and no message.
+ * Stateless; DEVICE pointers on the current device to `count` words each, owned
+ * by the caller; R, RP are only read, Z is replaced, M is overwritten and must not
+ * overlap the others.  Two kernels on `cuda_stream`; the call does not wait.
+ * Errors: INVALID_ARG (null pointer), SHAPE (count < 1, frac_bits outside [1, 31]), CUDA. */
+int comet_truncate_pair(void* cuda_stream, uint64_t* const Z[2], const uint64_t* const R[2],
+                        const uint64_t* const RP[2], uint64_t* const M[2], int64_t count, int32_t frac_bits);
+
 /* ---------------------------------------------------------------------------
  * KV-cache manager, Section 6: which cache entries to compute together with the
  * current token.  Host logic only (HOST pointers, no GPU work): the result is a

@@ -31,7 +31,7 @@ EXPORTS = (
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
     "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
-    "comet_add_bias", "comet_bind_shares",
+    "comet_add_bias", "comet_bind_shares", "comet_truncate_pair",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -92,6 +92,7 @@ def _load():
     lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
     lib.comet_invert_permutation.argtypes = [vp, vp, vp, i64, vp]
     lib.comet_add_bias.argtypes = [vp, pair, pair, i64, i64]
+    lib.comet_truncate_pair.argtypes = [vp, pair, pair, pair, pair, i64, i32]
     lib.comet_kv_plan.argtypes = [vp, vp, i32, i32, i64, i64, vp, vp, ctypes.POINTER(i32)]
     lib.comet_beaver_mul.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, pair, i64]
     return lib
@@ -337,6 +338,21 @@ def beaver_mul(X, Y, A, B, C, stream: Optional[torch.cuda.Stream] = None):
     if code != OK:
         raise CometError(code, "comet_beaver_mul")
     return D, E, Z
+
+
+def truncate_pair(Z, R, RP, frac_bits: int, stream: Optional[torch.cuda.Stream] = None):
+    """Truncation with a dealer's pair (comet_truncate_pair), both parties: Z is replaced by shares of
+    floor(z / 2^frac_bits) (or one less).  Z, R, RP are pairs of equally shaped CUDA tensors of 8-byte words.
+    Returns the messages M = Z - R (a pair)."""
+    shape = Z[0].shape
+    for t in (*Z, *R, *RP):
+        assert t.element_size() == 8 and t.shape == shape
+    M = [torch.empty_like(Z[0]) for _ in (0, 1)]
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    code = _lib.comet_truncate_pair(sp, _pair(Z), _pair(R), _pair(RP), _pair(M), Z[0].numel(), frac_bits)
+    if code != OK:
+        raise CometError(code, "comet_truncate_pair")
+    return M
 
 
 def kv_plan(present: np.ndarray, active: np.ndarray, x: int, w: int):

@@ -1116,6 +1116,38 @@ extern "C" int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], c
 }
 
 // ---------------------------------------------------------------------------
+// Truncation with a dealer's pair: Section 2.1's Reconstruction and Addition.
+// ---------------------------------------------------------------------------
+extern "C" int comet_truncate_pair(void* cuda_stream, uint64_t* const Z[2], const uint64_t* const R[2],
+                                   const uint64_t* const RP[2], uint64_t* const M[2], int64_t count,
+                                   int32_t frac_bits) {
+    if (!Z || !R || !RP || !M) return COMET_ERR_INVALID_ARG;
+    for (int p = 0; p < 2; ++p)
+        if (!Z[p] || !R[p] || !RP[p] || !M[p]) return COMET_ERR_INVALID_ARG;
+    if (count < 1) return COMET_ERR_SHAPE;
+    if (frac_bits < 1 || frac_bits > 31) return COMET_ERR_SHAPE;
+    comet::TruncPairArgs g;
+    bool vec = (count % 2) == 0;
+    for (int p = 0; p < 2; ++p) {
+        g.z[p] = reinterpret_cast<u64*>(Z[p]); g.m[p] = reinterpret_cast<u64*>(M[p]);
+        g.r[p] = reinterpret_cast<const u64*>(R[p]); g.rp[p] = reinterpret_cast<const u64*>(RP[p]);
+        vec = vec && aligned16(Z[p]) && aligned16(R[p]) && aligned16(RP[p]) && aligned16(M[p]);
+    }
+    g.pieces = vec ? count / 2 : count;
+    g.f = frac_bits;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const dim3 grid(shuffle_grid(g.pieces), 2);
+    if (vec) {
+        comet::trunc_pair_open_kernel<ulonglong2><<<grid, 256, 0, stream>>>(g);
+        comet::trunc_pair_combine_kernel<ulonglong2><<<grid, 256, 0, stream>>>(g);      // after the exchange
+    } else {
+        comet::trunc_pair_open_kernel<u64><<<grid, 256, 0, stream>>>(g);
+        comet::trunc_pair_combine_kernel<u64><<<grid, 256, 0, stream>>>(g);
+    }
+    return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
 // KV-cache manager (Section 6): request merging and the prefetch rule.  Host logic.
 // ---------------------------------------------------------------------------
 extern "C" int comet_kv_plan(const uint8_t* present, const uint8_t* active, int32_t tokens, int32_t heads, int64_t x,

@@ -68,6 +68,52 @@ beaver_mul_combine_kernel(MulArgs g) {
         z[t] = mul_combine(__ldg(c + t), d0[t], d1[t], e0[t], e1[t], __ldg(a + t), __ldg(b + t), party);
 }
 
+// Truncation by f bits with a dealer's pair (r, r' = floor(r / 2^f), r read as signed).  Not a protocol of the
+// paper; it is Section 2.1's "Reconstruction" of m = z - r followed by its "Addition" of the public value
+// floor(m / 2^f):
+//   open   : [m]_i = [z]_i - [r]_i                                      (before the exchange)
+//   combine: m = [m]_0 + [m]_1,  [z]_i <- [r']_i + i * (m >> f, arithmetic)  (after it)
+struct TruncPairArgs {
+    u64* z[2];                   // in: shares at scale 2f; out: shares at scale f
+    const u64* r[2]; const u64* rp[2];
+    u64* m[2];                   // the messages
+    long long pieces;
+    int f;
+};
+
+__device__ __forceinline__ u64 trunc_floor(u64 m, int f) { return (u64)((long long)m >> f); }
+__device__ __forceinline__ u64 trunc_pair_out(u64 rp, u64 m0, u64 m1, int f, int party) {
+    return party ? rp + trunc_floor(m0 + m1, f) : rp;
+}
+__device__ __forceinline__ ulonglong2 trunc_pair_out(ulonglong2 rp, ulonglong2 m0, ulonglong2 m1, int f, int party) {
+    return make_ulonglong2(trunc_pair_out(rp.x, m0.x, m1.x, f, party), trunc_pair_out(rp.y, m0.y, m1.y, f, party));
+}
+
+template <typename PIECE>
+__global__ void __launch_bounds__(256)
+trunc_pair_open_kernel(TruncPairArgs g) {
+    const int party = blockIdx.y;
+    const PIECE* __restrict__ z = reinterpret_cast<const PIECE*>(party ? g.z[1] : g.z[0]);
+    const PIECE* __restrict__ r = reinterpret_cast<const PIECE*>(party ? g.r[1] : g.r[0]);
+    PIECE* __restrict__ m = reinterpret_cast<PIECE*>(party ? g.m[1] : g.m[0]);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < g.pieces; t += stride)
+        m[t] = mul_sub(z[t], __ldg(r + t));
+}
+
+template <typename PIECE>
+__global__ void __launch_bounds__(256)
+trunc_pair_combine_kernel(TruncPairArgs g) {
+    const int party = blockIdx.y;
+    const PIECE* __restrict__ m0 = reinterpret_cast<const PIECE*>(g.m[0]);
+    const PIECE* __restrict__ m1 = reinterpret_cast<const PIECE*>(g.m[1]);
+    const PIECE* __restrict__ rp = reinterpret_cast<const PIECE*>(party ? g.rp[1] : g.rp[0]);
+    PIECE* __restrict__ z = reinterpret_cast<PIECE*>(party ? g.z[1] : g.z[0]);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < g.pieces; t += stride)
+        z[t] = trunc_pair_out(__ldg(rp + t), m0[t], m1[t], g.f, party);
+}
+
 // Section 2.1 "Addition": a shared bias [cols] added to every row of a shared matrix, in place; purely local.
 struct BiasArgs {
     u64* z[2];
