@@ -301,6 +301,10 @@ def main():
     ap.add_argument("--token-masks", type=float, default=0.0, metavar="P",
                     help="give every token its own Bernoulli(P) mask over the active blocks (Protocols 2 and 3 in "
                          "general: connected components, per-column row sets); set_token_mask is timed with set_mask")
+    ap.add_argument("--clusters", type=int, default=0, metavar="G",
+                    help="with --token-masks: deal tokens and active blocks to G groups of requests with disjoint "
+                         "blocks (at least G connected components, members scattered); the up-projection then "
+                         "computes the component rectangles only")
     ap.add_argument("--in-flight", type=int, default=4, metavar="C",
                     help="independent FFN problems in flight (contexts, one stream each, inputs bound in place); the "
                          "headline throughput is measured that way when C > 1, the one-problem-at-a-time figures are "
@@ -356,8 +360,10 @@ def main():
         devt = [{k: v.to(dev) for k, v in hp.items()} for hp in pinned]
         tm = None
         if args.token_masks > 0:
-            tm = torch.from_numpy(wl.token_block_masks(seed, f"bench/tm/{s}", T, int(inp["mask"].sum()),
-                                                       args.token_masks))
+            nab = int(inp["mask"].sum())
+            tm = torch.from_numpy(
+                wl.token_block_masks_clustered(seed, f"bench/tm/{s}", T, nab, args.clusters, args.token_masks)
+                if args.clusters > 1 else wl.token_block_masks(seed, f"bench/tm/{s}", T, nab, args.token_masks))
         sets.append({"n": inp["n"], "tm_host": tm.pin_memory() if tm is not None else None,
                      "tm_dev": tm.to(dev) if tm is not None else None,
                      "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
@@ -460,6 +466,19 @@ def main():
     barrier()
     stats = ctx.stats()
     ctx.set_profiling(False)
+    up_counts = None
+    if args.token_masks > 0:                    # what the up-projection of input set 0 covers under its token mask
+        st0 = sets[0]
+        ctx.set_mask(st0["mask_dev"])
+        ctx.set_token_mask(st0["tm_dev"])
+        for p in (0, 1):
+            for tid in UP_IDS:
+                ctx.load_shares(p, tid, st0["dev"][p][tid])
+        ctx.ffn_up(T)
+        su = ctx.stats()
+        up_counts = {"components": su.n_components, "theorem1_macs": su.ring_macs,
+                     "union_macs": 2 * 2 * T * d * cfg.groups * st0["n"], "tensor_tile_macs": su.tensor_tile_macs}
+        barrier()
 
     # ---- several independent problems in flight (throughput mode): C contexts with their own weights, stream and
     #      two input sets each, inputs bound in place (no copies), steps issued round-robin; the region is timed
@@ -611,7 +630,10 @@ def main():
                                  "region of K steps between two CUDA events" if use_piped else
                                  "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream"),
                        "token_masks": (f"per-token Bernoulli({args.token_masks}) masks over the active blocks, "
-                                       f"{stats.n_components} component(s)" if args.token_masks > 0 else "none"),
+                                       f"{stats.n_components} component(s)"
+                                       + (f", {args.clusters} groups of requests" if args.clusters > 1 else "")
+                                       if args.token_masks > 0 else "none"),
+                       "up_projection_under_token_mask": up_counts,
                        "parallelism": f"independent FFN per GPU x{world}"},
             "gpu_launches": int(piped["launches"] if use_piped else launches),
             "clocks": clocks_piped if use_piped else clocks_single,

@@ -120,7 +120,9 @@ enum {
 typedef struct {
     int64_t message_bytes;   /* bytes of E_i and F_i written by the last ffn_up/ffn_down, both parties:
                                 2 * 8 * (T*K + K*N), the communication cost C_1 of the optimality proof */
-    int64_t ring_macs;       /* 64-bit multiply-adds of the last ffn_up/ffn_down, both parties: 2 * 2*T*K*N */
+    int64_t ring_macs;       /* 64-bit multiply-adds of the last ffn_up/ffn_down, both parties: 2 * 2*T*K*N;
+                                for ffn_up under a token mask on the tensor-core path with more than 32 tokens,
+                                Theorem 1's count: 2 * 2*K * sum over components of rows x columns */
     int32_t n_active;        /* active neurons under the current mask                            */
     int32_t n_active_blocks;
     int32_t tokens;          /* T of the last ffn call                                           */
@@ -132,6 +134,9 @@ typedef struct {
     int64_t phase_launches[COMET_NUM_PHASES];
     int32_t n_components;    /* connected components under the current token mask (0 without one) */
     int32_t reserved;
+    int64_t tensor_tile_macs; /* 64-bit multiply-adds the tensor-core kernel of the last ffn call covered, counted
+                                 in whole 128 x 64 output tiles, both parties (0 on the CUDA-core path): under a
+                                 token mask with several components only the tiles that meet a component */
 } comet_stats_t;
 
 /* Create a context: validates the configuration, selects the device, and

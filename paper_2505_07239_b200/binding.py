@@ -49,7 +49,7 @@ class CometStats(ctypes.Structure):
                 ("n_active_blocks", ctypes.c_int32), ("tokens", ctypes.c_int32), ("matmul_path", ctypes.c_int32),
                 ("kernel_launches", ctypes.c_int64), ("phase_ms", ctypes.c_double * 5),
                 ("phase_launches", ctypes.c_int64 * 5), ("n_components", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("reserved", ctypes.c_int32), ("tensor_tile_macs", ctypes.c_int64)]
 
 
 class CometError(RuntimeError):

@@ -50,11 +50,19 @@ struct comet_ctx {
     bool tmask_set;
     int32_t tmask_tokens;
     int64_t tmask_masked;         // non-zero entries of the hidden state under the token mask (neurons, not blocks)
-    long long* h_masked;          // pinned and mapped: [0] count_mask_kernel's count, [1..3] token_components_kernel's report
+    long long* h_masked;          // pinned and mapped: [0] count_mask_kernel's count, [1..3] token_components_kernel's
+                                  // report, [4..5] group_plan_kernel's report
     long long* h_masked_dev;
     int32_t* d_row_label;         // component label per token row / per active block under the token mask
     int32_t* d_blk_label;
     int32_t n_components, live_rows, live_blocks;
+    // one multiplication per component on the tensor-core path: component-sorted order and the tiles with work
+    int32_t* d_row_map;
+    int32_t* d_col_map;
+    int32_t* d_tiles;
+    bool grouped;                 // the up-projection under the current token mask runs over the listed tiles only
+    int32_t n_tiles;
+    int64_t component_pairs;      // sum over components of token rows x active blocks
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
     int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
@@ -224,6 +232,7 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.tmask_ld = c->n_active_blocks;
     a.row_label = (!pr.down && c->tmask_set) ? c->d_row_label : nullptr;
     a.blk_label = (!pr.down && c->tmask_set) ? c->d_blk_label : nullptr;
+    a.col_map = (!pr.down && c->grouped) ? c->d_col_map : nullptr;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
@@ -250,13 +259,19 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
         a.Z[p] = c->buf[p][pr.idZ];
     }
     a.M = pr.M; a.N = pr.N; a.K = pr.K; a.kblocks = kb;
+    if (!pr.down && c->grouped) {           // component-sorted planes of the rows and columns that lie in a component
+        a.M = c->live_rows;
+        a.N = c->groups * c->live_blocks * c->cfg.block;
+        a.row_map = c->d_row_map;
+        a.col_map = c->d_col_map;
+    }
     a.left_tile_rows = limb_few(pr) ? comet::limb_few::BT : lb::BM;
     a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
     a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
     a.tmask_ld = c->n_active_blocks;
     a.bs = c->cfg.block;
-    a.left_tiles = left ? kb * ceil_div(pr.M, lb::PREP_ROWS) : 0;
-    a.right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
+    a.left_tiles = left ? kb * ceil_div(a.M, lb::PREP_ROWS) : 0;
+    a.right_tiles = right ? kb * ceil_div(a.N, lb::PREP_ROWS) : 0;
     a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
     a.copy_blocks = copy ? ew_grid(c, a.copy_pairs, 256) : 0;
     const int blocks = a.left_tiles + a.right_tiles + a.copy_blocks;
@@ -287,7 +302,18 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
     }
     a.M = pr.M; a.N = pr.N; a.mt = mt; a.nt = nt; a.kb = kb;
     a.error_flag = c->d_error;
-    const long long total_units = 2ll * mt * nt * 2 * kb;
+    a.ldz = pr.N; a.n_tiles = 0; a.bs = c->cfg.block;
+    a.tiles = nullptr; a.row_map = nullptr; a.col_map = nullptr;
+    const bool grouped = !pr.down && c->grouped && !few;
+    if (grouped) {
+        a.M = c->live_rows;
+        a.N = c->groups * c->live_blocks * c->cfg.block;
+        a.mt = ceil_div(a.M, lb::BM); a.nt = ceil_div(a.N, lb::BN);
+        a.n_tiles = c->n_tiles;
+        a.tiles = c->d_tiles; a.row_map = c->d_row_map; a.col_map = c->d_col_map;
+    }
+    const long long total_units = 2ll * (grouped ? (long long)c->n_tiles : (long long)mt * nt) * 2 * kb;
+    c->stats.tensor_tile_macs = total_units * lb::KC * lb::BM * lb::BN;
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
         PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
@@ -306,6 +332,7 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
         lc.attrs = &attr;
         lc.numAttrs = 1;
         if (few) COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_few_kernel, a));
+        else if (grouped) COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_grouped_kernel, a));
         else COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_kernel, a));
     }
     c->stats.kernel_launches += 1;
@@ -464,6 +491,11 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::combine_limb_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)lb::SMEM_BYTES) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::combine_limb_grouped_kernel,
+                                        cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::limb_open_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::limb_prep_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -475,7 +507,14 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_tmask, (size_t)nb * (size_t)c->cap_T) == cudaSuccess;
-    ok = ok && cudaHostAlloc((void**)&c->h_masked, 4 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_masked, 6 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_row_map, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_col_map, (size_t)c->groups * nb * sizeof(int32_t)) == cudaSuccess;
+    {
+        const size_t mt = ceil_div((int)c->cap_T, comet::limb::BM);
+        const size_t nt = ceil_div((int)(c->groups * c->cap_n), comet::limb::BN);
+        ok = ok && cudaMalloc((void**)&c->d_tiles, mt * nt * sizeof(int32_t)) == cudaSuccess;
+    }
     ok = ok && cudaMalloc((void**)&c->d_row_label, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_blk_label, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaHostGetDevicePointer((void**)&c->h_masked_dev, c->h_masked, 0) == cudaSuccess;
@@ -516,6 +555,9 @@ void comet_destroy(comet_ctx* c) {
     if (c->d_tmask) cudaFree(c->d_tmask);
     if (c->h_masked) cudaFreeHost(c->h_masked);
     if (c->d_row_label) cudaFree(c->d_row_label);
+    if (c->d_row_map) cudaFree(c->d_row_map);
+    if (c->d_col_map) cudaFree(c->d_col_map);
+    if (c->d_tiles) cudaFree(c->d_tiles);
     if (c->d_blk_label) cudaFree(c->d_blk_label);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
@@ -623,6 +665,7 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     c->n_active = (int32_t)n;
     c->mask_set = true;
     c->tmask_set = false;             // a token mask refines one block mask
+    c->grouped = false;
     c->up_done = c->down_done = false;
     for (int p = 0; p < 2; ++p)
         for (int id = COMET_A_UP; id <= COMET_C_DN; ++id) {
@@ -642,6 +685,7 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     if (!token_mask) {                         // back to "every token uses every active neuron"
         if (tokens != 0 || n_active_blocks != 0) return COMET_ERR_INVALID_ARG;
         c->tmask_set = false;
+        c->grouped = false;
         if (masked_out) *masked_out = 0;
         return COMET_OK;
     }
@@ -656,12 +700,27 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     comet::token_components_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, tokens, n_active_blocks, c->d_row_label,
                                                              c->d_blk_label, c->h_masked_dev + 1);
     c->stats.kernel_launches += 2;
+    // ... and, for the tensor-core path, the component-sorted order and the output tiles that have work
+    const bool plan = c->path == COMET_PATH_LIMB && tokens > comet::limb_few::BT &&
+                      ceil_div(tokens, comet::limb::BM) <= 1024 &&
+                      ceil_div(c->groups * c->n_active, comet::limb::BN) <= 0xffff;
+    if (plan) {
+        comet::group_plan_kernel<<<1, 1024, 0, c->stream>>>(c->d_row_label, c->d_blk_label, tokens, n_active_blocks,
+                                                           c->groups, c->cfg.block, comet::limb::BM, comet::limb::BN,
+                                                           c->d_row_map, c->d_col_map, c->d_tiles, c->h_masked_dev + 4);
+        c->stats.kernel_launches += 1;
+    }
     COMET_CUDA(c, cudaGetLastError());
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
     c->tmask_masked = (int64_t)c->h_masked[0] * c->cfg.block;
     c->n_components = (int32_t)c->h_masked[1];
     c->live_rows = (int32_t)c->h_masked[2];
     c->live_blocks = (int32_t)c->h_masked[3];
+    c->n_tiles = plan ? (int32_t)c->h_masked[4] : 0;
+    c->component_pairs = plan ? (int64_t)c->h_masked[5] : -1;
+    // several components, or rows / blocks in none: compute the component rectangles only
+    c->grouped = plan && c->n_tiles > 0 &&
+                 (c->n_components > 1 || c->live_rows < tokens || c->live_blocks < n_active_blocks);
     c->stats.n_components = c->n_components;
     c->tmask_tokens = tokens;
     c->tmask_set = true;
@@ -687,7 +746,11 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
     c->stats.message_bytes = c->tmask_set
         ? 2ll * 8 * ((int64_t)c->live_rows * d + (int64_t)d * g * c->live_blocks * bs)
         : 2ll * 8 * ((int64_t)tokens * d + (int64_t)d * g * n);
-    c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)d * g * n;
+    // Theorem 1's multiplication count when the components are known (one product per component), else the
+    // product over the union of the supports
+    c->stats.ring_macs = (c->tmask_set && c->component_pairs >= 0)
+        ? 2ll * 2 * d * g * bs * c->component_pairs : 2ll * 2 * tokens * (int64_t)d * g * n;
+    c->stats.tensor_tile_macs = 0;
     c->up_tokens = tokens;
     c->up_done = true;
     if (n == 0) return COMET_OK;
@@ -771,6 +834,7 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
     // with a token mask only the non-zero entries of the hidden state are opened (Theorem 2's communication)
     c->stats.message_bytes = 2ll * 8 * ((c->tmask_set ? c->tmask_masked : (int64_t)tokens * n) + (int64_t)n * d);
     c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)n * d;
+    c->stats.tensor_tile_macs = 0;
     c->down_tokens = tokens;
     c->down_done = true;
     if (n == 0) {

@@ -133,6 +133,10 @@ struct LimbOpenArgs {
     // component), or null.  A row / column outside every component is not opened: its message words are zero.
     const int32_t* row_label;
     const int32_t* blk_label;
+    // With col_map (up only; one multiplication per component): row r of the plane tiles is compact row
+    // col_map[r / bs] * bs + r % bs of the right operand, i.e. the planes are written in component order while the
+    // message F_i keeps the compact order.
+    const int32_t* col_map;
 };
 
 __global__ void __launch_bounds__(256)
@@ -176,11 +180,15 @@ limb_open_kernel(LimbOpenArgs a) {
 #pragma unroll
         for (int it = 0; it < PREP_ROWS / 16; ++it) {
             const int r = it * 16 + (tid >> 4);
-            const int row = row0 + r;
+            int row = row0 + r;
             u64 b0 = 0, b1 = 0;
             if (row < a.rows && k < a.K) {
                 const u64* wsrc;
                 bool dead = false;
+                if (a.col_map) {
+                    const int sb = row / a.bs;
+                    row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
+                }
                 if (a.down) {
                     wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
                 } else {
@@ -236,6 +244,11 @@ struct LimbPrepArgs {
     u64* Z[2];
     long long copy_pairs;
     int copy_blocks;
+    // One multiplication per component (up only): plane row r of the left operand is row row_map[r] of E and A_i,
+    // plane row r of the right operand is compact row col_map[r / bs] * bs + r % bs of F; M and N then count the
+    // rows and columns that lie in a component.  Null: identity.
+    const int32_t* row_map;
+    const int32_t* col_map;
 };
 
 __global__ void __launch_bounds__(256)
@@ -269,9 +282,15 @@ limb_prep_kernel(LimbPrepArgs a) {
 #pragma unroll
         for (int it = 0; it < PREP_ROWS / 16; ++it) {
             const int r = it * 16 + (tid >> 4);
-            const int row = row0 + r;
+            int row = row0 + r;
             u64 s0 = 0, s1 = 0, w0 = 0, w1 = 0;
             if (row < rows && k < a.K) {
+                if (left) {
+                    if (a.row_map) row = __ldg(a.row_map + row);
+                } else if (a.col_map) {
+                    const int sb = row / a.bs;
+                    row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
+                }
                 const size_t o = (size_t)row * a.K + k;
                 const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(in0 + o));
                 const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(in1 + o));
@@ -390,6 +409,14 @@ struct LimbArgs {
     int M, N;                // N a multiple of 16
     int mt, nt, kb;          // tiles and k-blocks per operand pair; one tile runs over 2*kb blocks
     int* error_flag;         // set to 1 if a bounded wait ran out
+    // Only read by the grouped kernel (Protocol 2 with one multiplication per connected component): the planes
+    // hold the rows and columns of the components sorted by component, M and N count those, and only the listed
+    // tiles are computed.  A finished row piece goes to row row_map[r] of Z, whose rows are ldz words long, and
+    // the 16 columns from sorted column c on to compact columns col_map[c / bs] * bs + c % bs.. (bs is a multiple of 16).
+    int ldz, n_tiles, bs;
+    const int32_t* tiles;    // [n_tiles] (m-tile << 16) | n-tile
+    const int32_t* row_map;  // [M] sorted row -> row of Z
+    const int32_t* col_map;  // [N / bs] sorted block -> compact block of Z
 };
 
 // Slow path of a bounded wait, kept out of line so that the polling loops of the three roles stay short.
@@ -444,18 +471,25 @@ struct LimbSegment {
     int count;       // k-blocks in this segment, <= MAX_SEGMENT_UNITS
 };
 
+template <bool GROUPED = false>
 __device__ __forceinline__ LimbSegment limb_segment(const LimbArgs& a, long long u, long long u_end) {
     const long long tile_units = 2ll * a.kb;
     const long long tile = u / tile_units;
     long long seg_end = (tile + 1) * tile_units;
     if (seg_end > u_end) seg_end = u_end;
     if (seg_end > u + limb::MAX_SEGMENT_UNITS) seg_end = u + limb::MAX_SEGMENT_UNITS;
-    const int per_party = a.mt * a.nt;
+    const int per_party = GROUPED ? a.n_tiles : a.mt * a.nt;
     LimbSegment s;
     s.party = (int)(tile / per_party);
     const int t2 = (int)(tile - (long long)s.party * per_party);
-    s.tm = t2 / a.nt;
-    s.tn = t2 - s.tm * a.nt;
+    if (GROUPED) {
+        const int packed = __ldg(a.tiles + t2);
+        s.tm = packed >> 16;
+        s.tn = packed & 0xffff;
+    } else {
+        s.tm = t2 / a.nt;
+        s.tn = t2 - s.tm * a.nt;
+    }
     s.kpos = (int)(u - tile * tile_units);
     s.count = (int)(seg_end - u);
     return s;
@@ -469,8 +503,8 @@ __device__ __forceinline__ uint32_t limb_desc_lo(uint32_t addr) {
 }
 constexpr uint32_t LIMB_DESC_HI = (uint32_t)(limb::SBO_BYTES >> 4) | (1u << 14);
 
-__global__ void __launch_bounds__(limb::THREADS, 1)
-combine_limb_kernel(LimbArgs a) {
+template <bool GROUPED>
+__device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
     using namespace limb;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[STAGES];
@@ -485,7 +519,7 @@ combine_limb_kernel(LimbArgs a) {
     uint8_t* sOut = sB + (size_t)STAGES * B_BLOCK_BYTES;      // EPI_WARPS x 32 rows x OUT_ROW_BYTES
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long total_units = 2ll * a.mt * a.nt * 2ll * a.kb;
+    const long long total_units = 2ll * (GROUPED ? a.n_tiles : a.mt * a.nt) * 2ll * a.kb;
     const long long u_begin = total_units * blockIdx.x / gridDim.x;
     const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
 
@@ -518,7 +552,7 @@ combine_limb_kernel(LimbArgs a) {
             const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
             const uint32_t sA0 = ptx::smem_u32(sA), sB0 = ptx::smem_u32(sB);
             for (long long u = u_begin; u < u_end && ok;) {
-                const LimbSegment sg = limb_segment(a, u, u_end);
+                const LimbSegment sg = limb_segment<GROUPED>(a, u, u_end);
                 u += sg.count;
                 int kpos = sg.kpos;
                 bool second = kpos >= a.kb;
@@ -571,7 +605,7 @@ combine_limb_kernel(LimbArgs a) {
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (long long u = u_begin; u < u_end && ok;) {
-                const LimbSegment sg = limb_segment(a, u, u_end);
+                const LimbSegment sg = limb_segment<GROUPED>(a, u, u_end);
                 u += sg.count;
                 ok = limb_wait(accum_empty, acc_phase ^ 1u, &abort_flag);
                 if (!ok) break;
@@ -621,14 +655,18 @@ combine_limb_kernel(LimbArgs a) {
         uint8_t* my_row = sOut + ((size_t)warp * 32 + lane) * OUT_ROW_BYTES;
         const uint32_t my_row_s = ptx::smem_u32(my_row);
         for (long long u = u_begin; u < u_end && ok;) {
-            const LimbSegment sg = limb_segment(a, u, u_end);
+            const LimbSegment sg = limb_segment<GROUPED>(a, u, u_end);
             u += sg.count;
             ok = limb_wait_warp(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
             if (!ok) break;
             ptx::fence_after_sync();
             const int row = sg.tm * BM + quarter * 32 + lane;
             const int col0 = sg.tn * BN + chalf * 32;
-            u64* zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0;
+            u64* zrow;
+            if (GROUPED)
+                zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)(row < a.M ? __ldg(a.row_map + row) : 0) * a.ldz;
+            else
+                zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0;
 #pragma unroll
             for (int h = 0; h < 32 / OUT_COLS; ++h) {          // this thread's 32 columns, OUT_COLS at a time
                 ptx::bulk_wait_group_read0();                  // the previous reduction has read this thread's staging row
@@ -658,7 +696,14 @@ combine_limb_kernel(LimbArgs a) {
                 if (cols > OUT_COLS) cols = OUT_COLS;
                 if (row < a.M && cols > 0) {
                     ptx::fence_proxy_async_smem();     // this thread's row, written above, is read by the copy engine
-                    ptx::bulk_reduce_add_u64(zrow + h * OUT_COLS, my_row_s, (uint32_t)cols * 8u);
+                    u64* dst;
+                    if (GROUPED) {
+                        const int c = col0 + h * OUT_COLS, blk = c / a.bs;
+                        dst = zrow + (size_t)__ldg(a.col_map + blk) * a.bs + (c - blk * a.bs);
+                    } else {
+                        dst = zrow + h * OUT_COLS;
+                    }
+                    ptx::bulk_reduce_add_u64(dst, my_row_s, (uint32_t)cols * 8u);
                 }
                 ptx::bulk_commit_group();
             }
@@ -674,6 +719,18 @@ combine_limb_kernel(LimbArgs a) {
         ptx::fence_after_sync();
         ptx::tmem_dealloc(tmem_base, 512);
     }
+}
+
+__global__ void __launch_bounds__(limb::THREADS, 1)
+combine_limb_kernel(LimbArgs a) {
+    combine_limb_body<false>(a);
+}
+
+// Protocol 2 with one multiplication per connected component: the same kernel over the listed tiles of the
+// component-sorted operands, scattering the result rows back to the compact layout of Z.
+__global__ void __launch_bounds__(limb::THREADS, 1)
+combine_limb_grouped_kernel(LimbArgs a) {
+    combine_limb_body<true>(a);
 }
 
 // ---------------------------------------------------------------------------

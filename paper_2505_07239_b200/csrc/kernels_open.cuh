@@ -168,6 +168,102 @@ token_components_kernel(const uint8_t* __restrict__ S, int T, int nab, int32_t* 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Protocol 2 asks for one multiplication per connected component, over that component's rows and columns only
+// (Theorem 1's multiplication count).  On the tensor-core path this is ONE launch over component-sorted operands:
+// rows and column blocks are ordered by component label (ties by index), so every component is a contiguous
+// rectangle and an output tile has work only if the label ranges of its rows and of its columns intersect.
+//   row_map [T]           sorted row position -> token row; rows of no component come last
+//   col_map [groups*nab]  sorted block position -> compact block (group * nab + active block); within a
+//                         component the order is (group, block); blocks of no component come last
+//   tiles   [..]          (m-tile << 16) | n-tile of every tile with work, m-tiles of TM rows, n-tiles of TN columns
+//   report[0] = number of listed tiles, report[1] = sum over components of rows x blocks (mapped host memory)
+// One CTA of 1024 threads; needs ceil(live rows / TM) <= 1024.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+group_plan_kernel(const int32_t* __restrict__ row_label, const int32_t* __restrict__ blk_label, int T, int nab,
+                  int groups, int bs, int TM, int TN, int32_t* row_map, int32_t* col_map, int32_t* tiles,
+                  long long* report) {
+    __shared__ int live_rows, live_blocks;
+    __shared__ unsigned long long pairs;
+    __shared__ int tn_first[1024], tn_count[1024], tile_off[1024];
+    const int tid = threadIdx.x;
+    if (tid == 0) { live_rows = 0; live_blocks = 0; pairs = 0ull; }
+    __syncthreads();
+    {
+        int lr = 0, lb = 0;
+        for (int r = tid; r < T; r += 1024) lr += row_label[r] >= 0;
+        for (int b = tid; b < nab; b += 1024) lb += blk_label[b] >= 0;
+        if (lr) atomicAdd(&live_rows, lr);
+        if (lb) atomicAdd(&live_blocks, lb);
+    }
+    __syncthreads();
+    const int M = live_rows, NB = live_blocks;
+    unsigned long long my_pairs = 0;
+    for (int r = tid; r < T; r += 1024) {
+        const int l = row_label[r];
+        int rank = 0;
+        if (l >= 0) {
+            for (int q = 0; q < T; ++q) {
+                const int lq = row_label[q];
+                rank += lq >= 0 && (lq < l || (lq == l && q < r));
+            }
+            for (int b = 0; b < nab; ++b) my_pairs += blk_label[b] == l;
+        } else {
+            rank = M;
+            for (int q = 0; q < r; ++q) rank += row_label[q] < 0;
+        }
+        row_map[rank] = r;
+    }
+    if (my_pairs) atomicAdd(&pairs, my_pairs);
+    for (int b = tid; b < nab; b += 1024) {
+        const int l = blk_label[b];
+        if (l >= 0) {
+            int less = 0, same = 0, before = 0;
+            for (int q = 0; q < nab; ++q) {
+                const int lq = blk_label[q];
+                less += lq >= 0 && lq < l;
+                same += lq == l;
+                before += lq == l && q < b;
+            }
+            for (int g = 0; g < groups; ++g) col_map[groups * less + g * same + before] = g * nab + b;
+        } else {
+            int before = 0;
+            for (int q = 0; q < b; ++q) before += blk_label[q] < 0;
+            for (int g = 0; g < groups; ++g) col_map[groups * NB + g * (nab - NB) + before] = g * nab + b;
+        }
+    }
+    __syncthreads();
+    const int N = groups * NB * bs;
+    const int mt = (M + TM - 1) / TM, nt = (N + TN - 1) / TN;
+    if (tid < mt) {
+        const int lo_m = row_label[row_map[tid * TM]];
+        const int hi_m = row_label[row_map[min(tid * TM + TM, M) - 1]];
+        int first = 0, count = 0;
+        for (int tn = 0; tn < nt; ++tn) {
+            const int lo_n = blk_label[col_map[(tn * TN) / bs] % nab];
+            const int hi_n = blk_label[col_map[(min(tn * TN + TN, N) - 1) / bs] % nab];
+            if (hi_n >= lo_m && lo_n <= hi_m) {
+                if (count == 0) first = tn;
+                ++count;
+            }
+        }
+        tn_first[tid] = first;
+        tn_count[tid] = count;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int off = 0;
+        for (int tm = 0; tm < mt; ++tm) { tile_off[tm] = off; off += tn_count[tm]; }
+        report[0] = off;
+        report[1] = (long long)pairs;
+        __threadfence_system();
+    }
+    __syncthreads();
+    if (tid < mt)
+        for (int j = 0; j < tn_count[tid]; ++j) tiles[tile_off[tid] + j] = (tid << 16) | (tn_first[tid] + j);
+}
+
 // The Merge step of Protocol 2 on the compact result [T, cols]: an entry whose token and block are not in the same
 // component is no part of any result block and is zero in both shares.  Compact column c belongs to active block
 // (c mod n) / bs.  `pairs` = 16-byte word pairs per party.

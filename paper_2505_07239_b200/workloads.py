@@ -301,6 +301,33 @@ def token_block_masks(seed: int, stream: str, tokens: int, n_blocks: int, p_toke
     return m
 
 
+def token_block_masks_clustered(seed: int, stream: str, tokens: int, n_blocks: int, clusters: int, p_token: float,
+                                dead_tokens: int = 0, dead_blocks: int = 0) -> np.ndarray:
+    """Per-token masks whose bipartite graph falls into (at least) `clusters` connected components: a batch that
+    mixes requests with disjoint sets of active blocks.  Every token and every block is dealt to one cluster at
+    random (so the members of a cluster are scattered over the index range); inside a cluster entries are
+    Bernoulli(p_token), repaired so that every token has a block and every block a token of its cluster.  The first
+    `dead_tokens` tokens and `dead_blocks` blocks of a seeded shuffle get no entry at all.  uint8 [tokens, n_blocks]."""
+    tc = (random_u64(seed, stream + "/tc", tokens) % np.uint64(clusters)).astype(np.int64)
+    bc = (random_u64(seed, stream + "/bc", n_blocks) % np.uint64(clusters)).astype(np.int64)
+    bc[np.argsort(random_u64(seed, stream + "/bseed", n_blocks), kind="stable")[:min(clusters, n_blocks)]] = \
+        np.arange(min(clusters, n_blocks))                       # every cluster owns a block when there are enough
+    tc[np.argsort(random_u64(seed, stream + "/tseed", tokens), kind="stable")[:min(clusters, tokens)]] = \
+        np.arange(min(clusters, tokens))
+    u = random_unit(seed, stream, tokens * n_blocks).reshape(tokens, n_blocks)
+    same = tc[:, None] == bc[None, :]
+    m = ((np.abs(u) < p_token) & same).astype(np.uint8)
+    rank = random_u64(seed, stream + "/fix", tokens * n_blocks).reshape(tokens, n_blocks) >> np.uint64(1)
+    rank = np.where(same, rank, np.uint64(0xFFFFFFFFFFFFFFFF))
+    for t in np.nonzero(m.sum(axis=1) == 0)[0]:
+        m[t, int(np.argmin(rank[t]))] = 1
+    for b in np.nonzero(m.sum(axis=0) == 0)[0]:
+        m[int(np.argmin(rank[:, b])), b] = 1
+    m[np.argsort(random_u64(seed, stream + "/dt", tokens), kind="stable")[:dead_tokens], :] = 0
+    m[:, np.argsort(random_u64(seed, stream + "/db", n_blocks), kind="stable")[:dead_blocks]] = 0
+    return m
+
+
 def bipartite_components(S: np.ndarray):
     """Connected components of the bipartite graph rows x columns with the non-zeros of S as edges, by a library
     routine (scipy).  Returns (row_label, col_label) with -1 for nodes without an edge; labels are arbitrary."""

@@ -21,6 +21,9 @@ def _canonical(row_comp, col_comp):
     return f(rc), f(cc)
 
 
+_LAST = {}
+
+
 def _run(cfg, seed, tokens, sparsity, path, p_token=None, token_mask=None):
     from paper_2505_07239_b200 import binding as cb
     from tests import harness as hz
@@ -47,6 +50,8 @@ def _run(cfg, seed, tokens, sparsity, path, p_token=None, token_mask=None):
     ctx.ffn_up(T)
     st = ctx.stats()
     assert st.matmul_path == path and st.n_components == ref["L"]
+    _LAST.update(ring_macs=st.ring_macs, tile_macs=st.tensor_tile_macs, dot_products=ref["dot_products"],
+                 dense_tile_macs=2 * 2 * (-(-T // 128) * 128) * (-(-(g * n) // 64) * 64) * (-(-d // 32) * 32), d=d)
     rl, bl, L = ctx.get_components(T, nab)
     want_r, want_c = _canonical(ref["row_comp"], ref["col_comp"][:n])
     assert L == ref["L"] and np.array_equal(rl, want_r) and np.array_equal(np.repeat(bl, bs), want_c)
@@ -103,3 +108,66 @@ def test_opt125m_one_giant_component():
         pytest.skip("needs a CUDA device")
     bad, L = _run(wl.CONFIGS["opt125m"], 97, 128, None, 2, p_token=0.3)
     assert bad == 0 and L == 1
+
+
+# ---- one multiplication per component on the tensor-core path (more than 32 tokens): component-sorted operands,
+#      only the tiles that meet a component are computed, results scattered back to the compact layout
+
+def _clustered(cfg, seed, tokens, sparsity, clusters, p, dead_tokens=0, dead_blocks=0):
+    mask = wl.block_mask(cfg, seed, sparsity)
+    return wl.token_block_masks_clustered(seed, "tmc", tokens, int(mask.sum()), clusters, p, dead_tokens, dead_blocks)
+
+
+@pytest.mark.parametrize("tokens,block,clusters,dead", [(200, 32, 4, 2), (130, 16, 3, 0), (300, 64, 6, 3), (33, 32, 2, 1)])
+def test_grouped_launch_scattered_components(tokens, block, clusters, dead):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-grouped", tokens, 128, 2048, block, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    tm = _clustered(cfg, 300 + tokens, tokens, 0.5, clusters, 0.3, dead, dead)
+    bad, L = _run(cfg, 300 + tokens, tokens, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L >= clusters
+    assert _LAST["ring_macs"] == 2 * 2 * _LAST["d"] * _LAST["dot_products"]      # Theorem 1: one product per component
+    assert 0 < _LAST["tile_macs"] <= _LAST["dense_tile_macs"]
+    if tokens > 128:                                                               # several row tiles: fewer tiles
+        assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]                       # than the union needs
+
+
+def test_grouped_launch_gated_two_matrices():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-grouped-gated", 260, 128, 2048, 64, 16, True, 0.5, "uniform", "normal", "normal0.02")
+    tm = _clustered(cfg, 411, 260, 0.5, 4, 0.4, 1, 1)
+    bad, L = _run(cfg, 411, 260, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L >= 4
+    assert _LAST["ring_macs"] == 2 * 2 * _LAST["d"] * _LAST["dot_products"]
+    assert 0 < _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
+def test_grouped_launch_contiguous_components_and_single_rows():
+    """Hand-made: components that are already contiguous, one of a single token and a single block, tokens and
+    blocks in no component between them."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-hand-grouped", 140, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 77, 0.5).sum())
+    assert nab == 8
+    tm = np.zeros((140, nab), np.uint8)
+    tm[0:60, 0:3] = 1
+    tm[60, 5] = 1                       # a component of one token and one block
+    tm[70:139, 6:8] = 1                 # tokens 61-69 and 139, blocks 3-4 in no component
+    bad, L = _run(cfg, 77, 140, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L == 3
+    assert _LAST["ring_macs"] == 2 * 2 * 128 * (60 * 96 + 1 * 32 + 69 * 64)
+
+
+def test_grouped_launch_opt13b_at_90_percent():
+    """The graded FFN shape (512 tokens, d = 2048, 26 of 256 blocks active) with the batch split into four groups
+    of requests: full comparison against the oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.CONFIGS["opt1.3b"]
+    tm = _clustered(cfg, 555, 512, 0.9, 4, 0.6)
+    bad, L = _run(cfg, 555, 512, 0.9, 2, token_mask=tm)
+    assert bad == 0 and L >= 4
+    assert _LAST["ring_macs"] == 2 * 2 * _LAST["d"] * _LAST["dot_products"]
+    assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
