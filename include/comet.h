@@ -204,10 +204,13 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * and block lie in different components zero in both shares (Merge).  The
  * per-component triples are passed stacked: row r of COMET_A_UP is the mask row
  * of r's component, row c of COMET_B_UP that of c's, COMET_C_UP holds a^t b^t
- * on the blocks (its other words are ignored).  The products are evaluated as
- * ONE dense product over [tokens, g*n] and masked afterwards: communication is
- * Theorem 1's minimum, the dot-product count is not when there are several
- * components.
+ * on the blocks (its other words are ignored).  Communication is Theorem 1's
+ * minimum.  On the tensor-core path with more than 32 tokens the products of all
+ * components are ONE launch over the component-sorted operands that computes
+ * only the 128 x 64 output tiles which meet a component ("one multiplication per
+ * subgraph" at tile granularity; comet_stats.ring_macs is then Theorem 1's count,
+ * tensor_tile_macs what the tiles cover); otherwise one product over
+ * [tokens, g*n], masked afterwards.  The shares are the same bits either way.
  *
  * Down-projection, Protocol 3 (its row sets R_j): the sparsity distribution of the hidden
  * state.  `token_mask` is [tokens, n_active_blocks]
