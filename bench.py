@@ -352,18 +352,23 @@ def main():
 
     # rotating input sets: a fresh mask (so different weight rows), X, triples and H each
     R = 4
+
+    def token_mask_for(inp, stream_name):
+        """The per-token mask of one input set (None without --token-masks)."""
+        if args.token_masks <= 0:
+            return None
+        nab = int(inp["mask"].sum())
+        return torch.from_numpy(
+            wl.token_block_masks_clustered(seed, stream_name, T, nab, args.clusters, args.token_masks)
+            if args.clusters > 1 else wl.token_block_masks(seed, stream_name, T, nab, args.token_masks))
+
     sets = []
     for s in range(R):
         inp = make_inputs(cfg, seed, sparsity, s, T)
         host = lib_tensors(inp)
         pinned = [{k: torch.from_numpy(v.view(np.int64)).pin_memory() for k, v in hp.items()} for hp in host]
         devt = [{k: v.to(dev) for k, v in hp.items()} for hp in pinned]
-        tm = None
-        if args.token_masks > 0:
-            nab = int(inp["mask"].sum())
-            tm = torch.from_numpy(
-                wl.token_block_masks_clustered(seed, f"bench/tm/{s}", T, nab, args.clusters, args.token_masks)
-                if args.clusters > 1 else wl.token_block_masks(seed, f"bench/tm/{s}", T, nab, args.token_masks))
+        tm = token_mask_for(inp, f"bench/tm/{s}")
         sets.append({"n": inp["n"], "tm_host": tm.pin_memory() if tm is not None else None,
                      "tm_dev": tm.to(dev) if tm is not None else None,
                      "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
@@ -505,7 +510,10 @@ def main():
                 pinned = [{kk: torch.from_numpy(v.view(np.int64)).pin_memory() for kk, v in hp.items()}
                           for hp in lib_tensors(inp)]
                 devt = [{kk: v.to(dev) for kk, v in hp.items()} for hp in pinned]
+                tmk = token_mask_for(inp, f"bench/tm/p{k}/{j}")
                 mine.append({"mask_dev": torch.from_numpy(inp["mask"]).to(dev), "dev": devt, "pinned": pinned,
+                             "tm_dev": tmk.to(dev) if tmk is not None else None,
+                             "tm_host": tmk.pin_memory() if tmk is not None else None,
                              "mask_host": torch.from_numpy(inp["mask"]).pin_memory(),
                              "y_host": [torch.empty((T, d), dtype=torch.int64).pin_memory() for _ in (0, 1)]})
             pctx.append((cx, sk))
@@ -516,6 +524,8 @@ def main():
             st = psets[s % C][(s // C) % 2]
             with torch.cuda.stream(sk):
                 cx.set_mask(st["mask_dev"])
+                if st["tm_dev"] is not None:
+                    cx.set_token_mask(st["tm_dev"])
                 for p in (0, 1):
                     for tid in UP_IDS:
                         cx.bind_shares(p, tid, st["dev"][p][tid])
@@ -559,6 +569,8 @@ def main():
             st = psets[s % C][(s // C) % 2]
             with torch.cuda.stream(sk):
                 cx.set_mask(st["mask_host"].numpy())
+                if st["tm_host"] is not None:
+                    cx.set_token_mask(st["tm_host"].numpy())
                 for p in (0, 1):
                     for tid in UP_IDS:
                         cx.load_shares(p, tid, st["pinned"][p][tid])

@@ -223,11 +223,15 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * n_active_blocks = 0; comet_ffn_up and comet_ffn_down must then be called with
  * the same `tokens`.  Under a token mask comet_ffn_down opens only the
  * non-zero entries (E'_i is zero elsewhere: those words are not part of the
- * message) and ignores whatever COMET_H and COMET_A_DN hold off the support;
+ * message; likewise the rows of F'_i that belong to an active block no token
+ * uses) and ignores whatever COMET_H and COMET_A_DN hold off the support;
  * the dealer's C' is sum_j a_j b_j^T scattered to the rows R_j, i.e.
- * (mask * A') B'.  The products themselves are still evaluated densely over
- * [tokens, n] on the tensor cores: communication is Theorem 2's minimum, the
- * multiply count is not.  *masked_out (may be NULL) receives the number of
+ * (mask * A') B'.  Communication is Theorem 2's minimum.  On the tensor-core
+ * path with more than 32 tokens and several components, rows and contraction
+ * index are taken in component order and every tile of 128 rows runs over the
+ * blocks of its own components only; otherwise the product runs over
+ * [tokens, n].  comet_stats.ring_macs is Theorem 2's count either way,
+ * tensor_tile_macs what the tiles cover.  *masked_out (may be NULL) receives the number of
  * non-zero entries (neurons, summed over tokens); one 8-byte device-to-host
  * report and a stream synchronise.  Errors: STATE (no block mask yet), SHAPE
  * (tokens out of range, n_active_blocks not the current count), INVALID_ARG. */

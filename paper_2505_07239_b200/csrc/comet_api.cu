@@ -50,8 +50,7 @@ struct comet_ctx {
     bool tmask_set;
     int32_t tmask_tokens;
     int64_t tmask_masked;         // non-zero entries of the hidden state under the token mask (neurons, not blocks)
-    long long* h_masked;          // pinned and mapped: [0] count_mask_kernel's count, [1..3] token_components_kernel's
-                                  // report, [4..5] group_plan_kernel's report
+    long long* h_masked;          // pinned and mapped: [0..3] token_components_kernel's report, [4..6] group_plan_kernel's
     long long* h_masked_dev;
     int32_t* d_row_label;         // component label per token row / per active block under the token mask
     int32_t* d_blk_label;
@@ -59,9 +58,11 @@ struct comet_ctx {
     // one multiplication per component on the tensor-core path: component-sorted order and the tiles with work
     int32_t* d_row_map;
     int32_t* d_col_map;
-    int32_t* d_tiles;
-    bool grouped;                 // the up-projection under the current token mask runs over the listed tiles only
-    int32_t n_tiles;
+    int32_t* d_kmap;
+    comet::LimbGroupRow* d_group_up;
+    comet::LimbGroupRow* d_group_dn;
+    bool grouped;                 // the products under the current token mask run over the component rectangles only
+    int32_t group_units_up, group_units_dn;   // k-block units per party of the two grouped launches
     int64_t component_pairs;      // sum over components of token rows x active blocks
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
@@ -231,8 +232,9 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
     a.tmask_ld = c->n_active_blocks;
     a.row_label = (!pr.down && c->tmask_set) ? c->d_row_label : nullptr;
-    a.blk_label = (!pr.down && c->tmask_set) ? c->d_blk_label : nullptr;
+    a.blk_label = c->tmask_set ? c->d_blk_label : nullptr;
     a.col_map = (!pr.down && c->grouped) ? c->d_col_map : nullptr;
+    a.kmap = (pr.down && c->grouped) ? c->d_kmap : nullptr;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
@@ -259,11 +261,15 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
         a.Z[p] = c->buf[p][pr.idZ];
     }
     a.M = pr.M; a.N = pr.N; a.K = pr.K; a.kblocks = kb;
-    if (!pr.down && c->grouped) {           // component-sorted planes of the rows and columns that lie in a component
+    if (c->grouped) {                       // component-sorted planes of the rows and columns that lie in a component
         a.M = c->live_rows;
-        a.N = c->groups * c->live_blocks * c->cfg.block;
         a.row_map = c->d_row_map;
-        a.col_map = c->d_col_map;
+        if (pr.down) {
+            a.kmap = c->d_kmap;
+        } else {
+            a.N = c->groups * c->live_blocks * c->cfg.block;
+            a.col_map = c->d_col_map;
+        }
     }
     a.left_tile_rows = limb_few(pr) ? comet::limb_few::BT : lb::BM;
     a.right_tile_rows = limb_few(pr) ? comet::limb_few::BW : lb::BN;
@@ -302,17 +308,25 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
     }
     a.M = pr.M; a.N = pr.N; a.mt = mt; a.nt = nt; a.kb = kb;
     a.error_flag = c->d_error;
-    a.ldz = pr.N; a.n_tiles = 0; a.bs = c->cfg.block;
-    a.tiles = nullptr; a.row_map = nullptr; a.col_map = nullptr;
-    const bool grouped = !pr.down && c->grouped && !few;
+    a.ldz = pr.N; a.bs = c->cfg.block; a.group_units = 0;
+    a.groups = nullptr; a.row_map = nullptr; a.col_map = nullptr;
+    const bool grouped = c->grouped && !few;
     if (grouped) {
         a.M = c->live_rows;
-        a.N = c->groups * c->live_blocks * c->cfg.block;
-        a.mt = ceil_div(a.M, lb::BM); a.nt = ceil_div(a.N, lb::BN);
-        a.n_tiles = c->n_tiles;
-        a.tiles = c->d_tiles; a.row_map = c->d_row_map; a.col_map = c->d_col_map;
+        a.mt = ceil_div(a.M, lb::BM);
+        a.row_map = c->d_row_map;
+        if (pr.down) {
+            a.groups = c->d_group_dn;
+            a.group_units = c->group_units_dn;
+        } else {
+            a.N = c->groups * c->live_blocks * c->cfg.block;
+            a.nt = ceil_div(a.N, lb::BN);
+            a.col_map = c->d_col_map;
+            a.groups = c->d_group_up;
+            a.group_units = c->group_units_up;
+        }
     }
-    const long long total_units = 2ll * (grouped ? (long long)c->n_tiles : (long long)mt * nt) * 2 * kb;
+    const long long total_units = grouped ? 2ll * a.group_units : 2ll * mt * nt * 2 * kb;
     c->stats.tensor_tile_macs = total_units * lb::KC * lb::BM * lb::BN;
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
@@ -507,13 +521,14 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_tmask, (size_t)nb * (size_t)c->cap_T) == cudaSuccess;
-    ok = ok && cudaHostAlloc((void**)&c->h_masked, 6 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_masked, 7 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_row_map, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_col_map, (size_t)c->groups * nb * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_kmap, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
     {
         const size_t mt = ceil_div((int)c->cap_T, comet::limb::BM);
-        const size_t nt = ceil_div((int)(c->groups * c->cap_n), comet::limb::BN);
-        ok = ok && cudaMalloc((void**)&c->d_tiles, mt * nt * sizeof(int32_t)) == cudaSuccess;
+        ok = ok && cudaMalloc((void**)&c->d_group_up, mt * sizeof(comet::LimbGroupRow)) == cudaSuccess;
+        ok = ok && cudaMalloc((void**)&c->d_group_dn, mt * sizeof(comet::LimbGroupRow)) == cudaSuccess;
     }
     ok = ok && cudaMalloc((void**)&c->d_row_label, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_blk_label, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
@@ -557,7 +572,9 @@ void comet_destroy(comet_ctx* c) {
     if (c->d_row_label) cudaFree(c->d_row_label);
     if (c->d_row_map) cudaFree(c->d_row_map);
     if (c->d_col_map) cudaFree(c->d_col_map);
-    if (c->d_tiles) cudaFree(c->d_tiles);
+    if (c->d_kmap) cudaFree(c->d_kmap);
+    if (c->d_group_up) cudaFree(c->d_group_up);
+    if (c->d_group_dn) cudaFree(c->d_group_dn);
     if (c->d_blk_label) cudaFree(c->d_blk_label);
     if (c->d_ids) cudaFree(c->d_ids);
     if (c->d_count) cudaFree(c->d_count);
@@ -685,6 +702,7 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     if (!token_mask) {                         // back to "every token uses every active neuron"
         if (tokens != 0 || n_active_blocks != 0) return COMET_ERR_INVALID_ARG;
         c->tmask_set = false;
+        if (c->grouped) c->dn_right_ready = false;
         c->grouped = false;
         if (masked_out) *masked_out = 0;
         return COMET_OK;
@@ -695,19 +713,23 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     if ((int64_t)tokens * c->n_active < 0 || (int64_t)tokens * c->n_active > 0x7fffffffll) return COMET_ERR_SHAPE;
     const size_t bytes = (size_t)tokens * (size_t)n_active_blocks;
     COMET_CUDA(c, cudaMemcpyAsync(c->d_tmask, token_mask, bytes, copy_kind(location, true), c->stream));
-    comet::count_mask_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, (long long)bytes, c->h_masked_dev);
-    // Protocol 2, first step: the connected components the up-projection is partitioned into
-    comet::token_components_kernel<<<1, 1024, 0, c->stream>>>(c->d_tmask, tokens, n_active_blocks, c->d_row_label,
-                                                             c->d_blk_label, c->h_masked_dev + 1);
-    c->stats.kernel_launches += 2;
+    // Protocol 2, first step: the connected components the up-projection is partitioned into (and the number of
+    // non-zero entries, Theorem 2's count)
+    {
+        const size_t label_bytes = ((size_t)tokens + (size_t)n_active_blocks) * sizeof(int);
+        const bool in_smem = label_bytes <= 40 * 1024;
+        comet::token_components_kernel<<<1, 1024, in_smem ? label_bytes : 0, c->stream>>>(
+            c->d_tmask, tokens, n_active_blocks, c->d_row_label, c->d_blk_label, c->h_masked_dev, in_smem ? 1 : 0);
+    }
+    c->stats.kernel_launches += 1;
     // ... and, for the tensor-core path, the component-sorted order and the output tiles that have work
     const bool plan = c->path == COMET_PATH_LIMB && tokens > comet::limb_few::BT &&
-                      ceil_div(tokens, comet::limb::BM) <= 1024 &&
-                      ceil_div(c->groups * c->n_active, comet::limb::BN) <= 0xffff;
+                      ceil_div(tokens, comet::limb::BM) <= 1024;
     if (plan) {
-        comet::group_plan_kernel<<<1, 1024, 0, c->stream>>>(c->d_row_label, c->d_blk_label, tokens, n_active_blocks,
-                                                           c->groups, c->cfg.block, comet::limb::BM, comet::limb::BN,
-                                                           c->d_row_map, c->d_col_map, c->d_tiles, c->h_masked_dev + 4);
+        comet::group_plan_kernel<<<1, 1024, 0, c->stream>>>(
+            c->d_row_label, c->d_blk_label, tokens, n_active_blocks, c->groups, c->cfg.block,
+            ceil_div(c->cfg.d_model, comet::limb::KC), ceil_div(c->cfg.d_model, comet::limb::BN), c->d_row_map,
+            c->d_col_map, c->d_kmap, c->d_group_up, c->d_group_dn, c->h_masked_dev + 4);
         c->stats.kernel_launches += 1;
     }
     COMET_CUDA(c, cudaGetLastError());
@@ -716,11 +738,13 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     c->n_components = (int32_t)c->h_masked[1];
     c->live_rows = (int32_t)c->h_masked[2];
     c->live_blocks = (int32_t)c->h_masked[3];
-    c->n_tiles = plan ? (int32_t)c->h_masked[4] : 0;
+    c->group_units_up = plan ? (int32_t)c->h_masked[4] : 0;
     c->component_pairs = plan ? (int64_t)c->h_masked[5] : -1;
+    c->group_units_dn = plan ? (int32_t)c->h_masked[6] : 0;
     // several components, or rows / blocks in none: compute the component rectangles only
-    c->grouped = plan && c->n_tiles > 0 &&
+    c->grouped = plan && c->group_units_up > 0 && c->group_units_dn > 0 &&
                  (c->n_components > 1 || c->live_rows < tokens || c->live_blocks < n_active_blocks);
+    c->dn_right_ready = false;    // the order of the contraction index in the down-projection's planes may change
     c->stats.n_components = c->n_components;
     c->tmask_tokens = tokens;
     c->tmask_set = true;
@@ -831,9 +855,13 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
     }
     if (c->tmask_set && c->tmask_tokens != tokens) return COMET_ERR_SHAPE;   // the token mask was given for another T
     c->stats.tokens = tokens;
-    // with a token mask only the non-zero entries of the hidden state are opened (Theorem 2's communication)
-    c->stats.message_bytes = 2ll * 8 * ((c->tmask_set ? c->tmask_masked : (int64_t)tokens * n) + (int64_t)n * d);
-    c->stats.ring_macs = 2ll * 2 * tokens * (int64_t)n * d;
+    // with a token mask only the non-zero entries of the hidden state and the rows of the weight matrix that meet
+    // a non-zero column are opened (Theorem 2's communication)
+    c->stats.message_bytes = c->tmask_set
+        ? 2ll * 8 * (c->tmask_masked + (int64_t)c->live_blocks * bs * d)
+        : 2ll * 8 * ((int64_t)tokens * n + (int64_t)n * d);
+    // Theorem 2's multiplication count under a token mask (one product row per non-zero entry), else the full product
+    c->stats.ring_macs = 2ll * 2 * (c->tmask_set ? c->tmask_masked : (int64_t)tokens * n) * d;
     c->stats.tensor_tile_macs = 0;
     c->down_tokens = tokens;
     c->down_done = true;
@@ -881,7 +909,7 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
             H, A, E, pairs, c->tmask_set ? c->d_tmask : nullptr, c->n_active_blocks, n, bs);
         const int64_t wpairs = (int64_t)d * n / 2;
         comet::open_weight_strips_kernel<<<dim3(ew_grid(c, wpairs, 256), 2), 256, 0, c->stream>>>(
-            W, B, F, c->d_ids, n, bs, d, D);
+            W, B, F, c->d_ids, n, bs, d, D, c->tmask_set ? c->d_blk_label : nullptr);
     }
     c->stats.kernel_launches += 2;
     COMET_CUDA(c, cudaGetLastError());

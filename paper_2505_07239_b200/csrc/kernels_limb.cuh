@@ -131,12 +131,17 @@ struct LimbOpenArgs {
     int tmask_ld;
     // Protocol 2 over connected components: component label per row of X and per active block (-1 = in no
     // component), or null.  A row / column outside every component is not opened: its message words are zero.
+    // Protocol 3 (down) uses blk_label alone: a block no token uses holds no non-zero column of X, and the rows of
+    // the right operand that belong to it are not opened either.
     const int32_t* row_label;
     const int32_t* blk_label;
     // With col_map (up only; one multiplication per component): row r of the plane tiles is compact row
     // col_map[r / bs] * bs + r % bs of the right operand, i.e. the planes are written in component order while the
     // message F_i keeps the compact order.
     const int32_t* col_map;
+    // With kmap (down only): contraction index k of the plane tiles is compact index kmap[k / bs] * bs + k % bs,
+    // i.e. the planes run over the active blocks in component order while F_i keeps the compact order.
+    const int32_t* kmap;
 };
 
 __global__ void __launch_bounds__(256)
@@ -175,8 +180,13 @@ limb_open_kernel(LimbOpenArgs a) {
     {
         const int kk = (tid & 15) * 2;
         const int k = kb * KC + kk;
-        // down: the strip of W that holds compact contraction indices k, k+1
-        const int kcol = a.down && k < a.K ? a.ids[k / a.bs] * a.bs + (k % a.bs) : 0;
+        int ks = k;                                   // compact contraction index of plane position k
+        if (a.kmap && k < a.K) {
+            const int sb = k / a.bs;
+            ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
+        }
+        // down: the strip of W that holds compact contraction indices ks, ks+1
+        const int kcol = a.down && k < a.K ? a.ids[ks / a.bs] * a.bs + (ks % a.bs) : 0;
 #pragma unroll
         for (int it = 0; it < PREP_ROWS / 16; ++it) {
             const int r = it * 16 + (tid >> 4);
@@ -190,6 +200,7 @@ limb_open_kernel(LimbOpenArgs a) {
                     row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
                 }
                 if (a.down) {
+                    dead = a.blk_label && a.blk_label[ks / a.bs] < 0;     // a block without a non-zero column of X
                     wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
                 } else {
                     const int grp = row / a.n, j = row - grp * a.n;
@@ -199,7 +210,7 @@ limb_open_kernel(LimbOpenArgs a) {
                                      : grp == 1 ? (party ? a.W1[1] : a.W1[0]) : (party ? a.W2g[1] : a.W2g[0])) +
                            (size_t)neuron * a.ldw + k;
                 }
-                const size_t o = (size_t)row * a.K + k;
+                const size_t o = (size_t)row * a.K + ks;
                 const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2*>(wsrc));
                 const ulonglong2 b = __ldg(reinterpret_cast<const ulonglong2*>(Bi + o));
                 *reinterpret_cast<ulonglong2*>(Fi + o) = dead ? make_ulonglong2(0ull, 0ull)
@@ -249,6 +260,8 @@ struct LimbPrepArgs {
     // rows and columns that lie in a component.  Null: identity.
     const int32_t* row_map;
     const int32_t* col_map;
+    // Down only: contraction index k of the planes is compact index kmap[k / bs] * bs + k % bs (both operands).
+    const int32_t* kmap;
 };
 
 __global__ void __launch_bounds__(256)
@@ -279,6 +292,11 @@ limb_prep_kernel(LimbPrepArgs a) {
     {
         const int kk = (tid & 15) * 2;
         const int k = kb * KC + kk;
+        int ks = k;                                   // compact contraction index of plane position k
+        if (a.kmap && k < a.K) {
+            const int sb = k / a.bs;
+            ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
+        }
 #pragma unroll
         for (int it = 0; it < PREP_ROWS / 16; ++it) {
             const int r = it * 16 + (tid >> 4);
@@ -291,12 +309,12 @@ limb_prep_kernel(LimbPrepArgs a) {
                     const int sb = row / a.bs;
                     row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
                 }
-                const size_t o = (size_t)row * a.K + k;
+                const size_t o = (size_t)row * a.K + ks;
                 const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(in0 + o));
                 const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(in1 + o));
                 s0 = x.x + y.x;                       // the exchange: both messages summed
                 s1 = x.y + y.y;
-                if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + k / a.bs] != 0)) {
+                if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + ks / a.bs] != 0)) {
                     const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(own + o));
                     w0 = z.x + (party ? s0 : 0ull);   // V_i = A_i + i*E
                     w1 = z.y + (party ? s1 : 0ull);
@@ -400,6 +418,135 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* d) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
 
+// ---------------------------------------------------------------------------
+// Protocols 2 and 3 ask for one multiplication per connected component / per non-zero column entry, over the
+// rows and columns that take part only (the multiplication counts of Theorems 1 and 2).  On the tensor cores this
+// becomes ONE launch over component-sorted operands: token rows and active blocks are ordered by component label
+// (ties by index), so every component is a contiguous rectangle, and
+//   up   (Protocol 2): an output tile has work only if the label ranges of its rows and of its columns intersect;
+//                      per row tile these column tiles form an interval;
+//   down (Protocol 3): a row tile's contraction runs only over the blocks of the components its rows belong to,
+//                      an interval of k-blocks in the sorted order of the contraction index.
+//   row_map [T]           sorted row position -> token row; rows of no component come last
+//   col_map [groups*nab]  sorted block position -> compact block (group * nab + active block) of the up-projection's
+//                         columns; within a component the order is (group, block); blocks of no component last
+//   kmap    [nab]         sorted block position -> active block, for the down-projection's contraction index
+//   up, dn  [row tiles]   the work of every tile of 128 sorted rows (LimbGroupRow)
+//   report[0] = k-block units of the up-projection per party, [1] = sum over components of rows x blocks,
+//   report[2] = units of the down-projection per party (mapped host memory)
+// One CTA of 1024 threads; needs ceil(live rows / 128) <= 1024.
+// ---------------------------------------------------------------------------
+struct LimbGroupRow {
+    int unit0;       // units (k-blocks, both operand pairs) of the row tiles before this one, per party
+    int tn0, ntn;    // interval of column tiles with work
+    int klo, kcnt;   // interval of k-blocks with work; a tile runs over 2 * kcnt units
+};
+
+__global__ void __launch_bounds__(1024)
+group_plan_kernel(const int32_t* __restrict__ row_label, const int32_t* __restrict__ blk_label, int T, int nab,
+                  int groups, int bs, int kb_up, int nt_dn, int32_t* row_map, int32_t* col_map, int32_t* kmap,
+                  LimbGroupRow* up, LimbGroupRow* dn, long long* report) {
+    constexpr int TM = limb::BM, TN = limb::BN, KC = limb::KC;
+    __shared__ int live_rows, live_blocks;
+    __shared__ unsigned long long pairs;
+    __shared__ int units_up[1024], units_dn[1024];
+    const int tid = threadIdx.x;
+    if (tid == 0) { live_rows = 0; live_blocks = 0; pairs = 0ull; }
+    __syncthreads();
+    {
+        int lr = 0, lb = 0;
+        for (int r = tid; r < T; r += 1024) lr += row_label[r] >= 0;
+        for (int b = tid; b < nab; b += 1024) lb += blk_label[b] >= 0;
+        if (lr) atomicAdd(&live_rows, lr);
+        if (lb) atomicAdd(&live_blocks, lb);
+    }
+    __syncthreads();
+    const int M = live_rows, NB = live_blocks;
+    unsigned long long my_pairs = 0;
+    for (int r = tid; r < T; r += 1024) {
+        const int l = row_label[r];
+        int rank = 0;
+        if (l >= 0) {
+            for (int q = 0; q < T; ++q) {
+                const int lq = row_label[q];
+                rank += lq >= 0 && (lq < l || (lq == l && q < r));
+            }
+            for (int b = 0; b < nab; ++b) my_pairs += blk_label[b] == l;
+        } else {
+            rank = M;
+            for (int q = 0; q < r; ++q) rank += row_label[q] < 0;
+        }
+        row_map[rank] = r;
+    }
+    if (my_pairs) atomicAdd(&pairs, my_pairs);
+    for (int b = tid; b < nab; b += 1024) {
+        const int l = blk_label[b];
+        if (l >= 0) {
+            int less = 0, same = 0, before = 0;
+            for (int q = 0; q < nab; ++q) {
+                const int lq = blk_label[q];
+                less += lq >= 0 && lq < l;
+                same += lq == l;
+                before += lq == l && q < b;
+            }
+            for (int g = 0; g < groups; ++g) col_map[groups * less + g * same + before] = g * nab + b;
+            kmap[less + before] = b;
+        } else {
+            int before = 0;
+            for (int q = 0; q < b; ++q) before += blk_label[q] < 0;
+            for (int g = 0; g < groups; ++g) col_map[groups * NB + g * (nab - NB) + before] = g * nab + b;
+            kmap[NB + before] = b;
+        }
+    }
+    __syncthreads();
+    const int N = groups * NB * bs;
+    const int mt = (M + TM - 1) / TM, nt = (N + TN - 1) / TN;
+    if (tid < mt) {
+        const int lo_m = row_label[row_map[tid * TM]];
+        const int hi_m = row_label[row_map[min(tid * TM + TM, M) - 1]];
+        int first = 0, count = 0;
+        for (int tn = 0; tn < nt; ++tn) {
+            const int lo_n = blk_label[col_map[(tn * TN) / bs] % nab];
+            const int hi_n = blk_label[col_map[(min(tn * TN + TN, N) - 1) / bs] % nab];
+            if (hi_n >= lo_m && lo_n <= hi_m) {
+                if (count == 0) first = tn;
+                ++count;
+            }
+        }
+        up[tid].tn0 = first;
+        up[tid].ntn = count;
+        up[tid].klo = 0;
+        up[tid].kcnt = kb_up;
+        units_up[tid] = count * 2 * kb_up;
+        int blk_begin = 0, blk_end = 0;          // sorted block positions of the components lo_m .. hi_m
+        for (int q = 0; q < nab; ++q) {
+            const int lq = blk_label[q];
+            blk_begin += lq >= 0 && lq < lo_m;
+            blk_end += lq >= 0 && lq <= hi_m;
+        }
+        const int klo = (blk_begin * bs) / KC, khi = (blk_end * bs + KC - 1) / KC;
+        dn[tid].tn0 = 0;
+        dn[tid].ntn = nt_dn;
+        dn[tid].klo = klo;
+        dn[tid].kcnt = khi - klo;
+        units_dn[tid] = nt_dn * 2 * (khi - klo);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int off_up = 0, off_dn = 0;
+        for (int tm = 0; tm < mt; ++tm) {
+            up[tm].unit0 = off_up;
+            dn[tm].unit0 = off_dn;
+            off_up += units_up[tm];
+            off_dn += units_dn[tm];
+        }
+        report[0] = off_up;
+        report[1] = (long long)pairs;
+        report[2] = off_dn;
+        __threadfence_system();
+    }
+}
+
 struct LimbArgs {
     const uint8_t* Epl[2];   // left planes of E = E_0 + E_1, per party: [m-tile][k-block][32 KiB]
     const uint8_t* Vpl[2];   // left planes of V_i = A_i + i*E
@@ -409,14 +556,17 @@ struct LimbArgs {
     int M, N;                // N a multiple of 16
     int mt, nt, kb;          // tiles and k-blocks per operand pair; one tile runs over 2*kb blocks
     int* error_flag;         // set to 1 if a bounded wait ran out
-    // Only read by the grouped kernel (Protocol 2 with one multiplication per connected component): the planes
-    // hold the rows and columns of the components sorted by component, M and N count those, and only the listed
-    // tiles are computed.  A finished row piece goes to row row_map[r] of Z, whose rows are ldz words long, and
-    // the 16 columns from sorted column c on to compact columns col_map[c / bs] * bs + c % bs.. (bs is a multiple of 16).
-    int ldz, n_tiles, bs;
-    const int32_t* tiles;    // [n_tiles] (m-tile << 16) | n-tile
-    const int32_t* row_map;  // [M] sorted row -> row of Z
-    const int32_t* col_map;  // [N / bs] sorted block -> compact block of Z
+    // Only read by the grouped kernel (one multiplication per connected component): the planes hold the operands
+    // in component-sorted order, M counts the rows that lie in a component (and N the columns, when col_map is
+    // given), and every row tile runs over the column tiles and k-blocks its LimbGroupRow names.  kb stays the
+    // number of k-blocks per plane tile in memory.  A finished row piece goes to row row_map[r] of Z, whose rows are
+    // ldz words long, and the 16 columns from sorted column c on to compact columns
+    // col_map[c / bs] * bs + c % bs.. (bs is a multiple of 16; col_map null: column c itself).
+    int ldz, bs;
+    int group_units;             // units per party: sum over row tiles of ntn * 2 * kcnt
+    const LimbGroupRow* groups;  // [mt]
+    const int32_t* row_map;      // [M] sorted row -> row of Z
+    const int32_t* col_map;      // [N / bs] sorted block -> compact block of Z, or null
 };
 
 // Slow path of a bounded wait, kept out of line so that the polling loops of the three roles stay short.
@@ -469,28 +619,41 @@ struct LimbSegment {
     int party, tm, tn;
     int kpos;        // first k-block, in [0, 2*kb): blocks [0,kb) pair E with B_i, [kb,2kb) pair V_i with F
     int count;       // k-blocks in this segment, <= MAX_SEGMENT_UNITS
+    int kb, klo;     // grouped kernel only: k-blocks per operand pair of this tile and the first of them
 };
 
 template <bool GROUPED = false>
 __device__ __forceinline__ LimbSegment limb_segment(const LimbArgs& a, long long u, long long u_end) {
-    const long long tile_units = 2ll * a.kb;
-    const long long tile = u / tile_units;
-    long long seg_end = (tile + 1) * tile_units;
-    if (seg_end > u_end) seg_end = u_end;
-    if (seg_end > u + limb::MAX_SEGMENT_UNITS) seg_end = u + limb::MAX_SEGMENT_UNITS;
-    const int per_party = GROUPED ? a.n_tiles : a.mt * a.nt;
     LimbSegment s;
-    s.party = (int)(tile / per_party);
-    const int t2 = (int)(tile - (long long)s.party * per_party);
+    long long seg_end;
     if (GROUPED) {
-        const int packed = __ldg(a.tiles + t2);
-        s.tm = packed >> 16;
-        s.tn = packed & 0xffff;
+        s.party = (int)(u / a.group_units);
+        const int ul = (int)(u - (long long)s.party * a.group_units);
+        int tm = 0;
+        while (tm + 1 < a.mt && __ldg(&a.groups[tm + 1].unit0) <= ul) ++tm;     // row tiles without work are passed over
+        const int unit0 = __ldg(&a.groups[tm].unit0);
+        s.kb = __ldg(&a.groups[tm].kcnt);
+        s.klo = __ldg(&a.groups[tm].klo);
+        const int tile_units = 2 * s.kb, r = ul - unit0, ti = r / tile_units;
+        s.tm = tm;
+        s.tn = __ldg(&a.groups[tm].tn0) + ti;
+        s.kpos = r - ti * tile_units;
+        seg_end = u - s.kpos + tile_units;
     } else {
+        const long long tile_units = 2ll * a.kb;
+        const long long tile = u / tile_units;
+        seg_end = (tile + 1) * tile_units;
+        const int per_party = a.mt * a.nt;
+        s.party = (int)(tile / per_party);
+        const int t2 = (int)(tile - (long long)s.party * per_party);
         s.tm = t2 / a.nt;
         s.tn = t2 - s.tm * a.nt;
+        s.kpos = (int)(u - tile * tile_units);
+        s.kb = a.kb;
+        s.klo = 0;
     }
-    s.kpos = (int)(u - tile * tile_units);
+    if (seg_end > u_end) seg_end = u_end;
+    if (seg_end > u + limb::MAX_SEGMENT_UNITS) seg_end = u + limb::MAX_SEGMENT_UNITS;
     s.count = (int)(seg_end - u);
     return s;
 }
@@ -519,7 +682,7 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
     uint8_t* sOut = sB + (size_t)STAGES * B_BLOCK_BYTES;      // EPI_WARPS x 32 rows x OUT_ROW_BYTES
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long total_units = 2ll * (GROUPED ? a.n_tiles : a.mt * a.nt) * 2ll * a.kb;
+    const long long total_units = GROUPED ? 2ll * a.group_units : 2ll * a.mt * a.nt * 2ll * a.kb;
     const long long u_begin = total_units * blockIdx.x / gridDim.x;
     const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
 
@@ -555,12 +718,14 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                 const LimbSegment sg = limb_segment<GROUPED>(a, u, u_end);
                 u += sg.count;
                 int kpos = sg.kpos;
-                bool second = kpos >= a.kb;
-                if (second) kpos -= a.kb;
+                const int kbe = GROUPED ? sg.kb : a.kb;       // k-blocks per operand pair of this tile
+                const int klo = GROUPED ? sg.klo : 0;         // and where they start in the plane tile
+                bool second = kpos >= kbe;
+                if (second) kpos -= kbe;
                 const uint8_t* left = (second ? (sg.party ? a.Vpl[1] : a.Vpl[0]) : (sg.party ? a.Epl[1] : a.Epl[0])) +
-                                      ((size_t)sg.tm * a.kb + kpos) * A_BLOCK_BYTES;
+                                      ((size_t)sg.tm * a.kb + klo + kpos) * A_BLOCK_BYTES;
                 const uint8_t* right = (second ? (sg.party ? a.Fpl[1] : a.Fpl[0]) : (sg.party ? a.Bpl[1] : a.Bpl[0])) +
-                                       ((size_t)sg.tn * a.kb + kpos) * B_BLOCK_BYTES;
+                                       ((size_t)sg.tn * a.kb + klo + kpos) * B_BLOCK_BYTES;
                 for (int it = 0; it < sg.count; ++it) {
                     ok = limb_wait(empty0 + 8 * stage, phase ^ 1u, &abort_flag);
                     if (!ok) break;
@@ -572,12 +737,12 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     left += A_BLOCK_BYTES;
                     right += B_BLOCK_BYTES;
-                    if (++kpos == a.kb && !second) {
+                    if (++kpos == kbe && !second) {
                         // the tile's first product (E with B_i) is done: go on with the second (V_i with F)
                         second = true;
                         kpos = 0;
-                        left = (sg.party ? a.Vpl[1] : a.Vpl[0]) + (size_t)sg.tm * a.kb * A_BLOCK_BYTES;
-                        right = (sg.party ? a.Fpl[1] : a.Fpl[0]) + (size_t)sg.tn * a.kb * B_BLOCK_BYTES;
+                        left = (sg.party ? a.Vpl[1] : a.Vpl[0]) + ((size_t)sg.tm * a.kb + klo) * A_BLOCK_BYTES;
+                        right = (sg.party ? a.Fpl[1] : a.Fpl[0]) + ((size_t)sg.tn * a.kb + klo) * B_BLOCK_BYTES;
                     }
                 }
             }
@@ -699,7 +864,7 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                     u64* dst;
                     if (GROUPED) {
                         const int c = col0 + h * OUT_COLS, blk = c / a.bs;
-                        dst = zrow + (size_t)__ldg(a.col_map + blk) * a.bs + (c - blk * a.bs);
+                        dst = a.col_map ? zrow + (size_t)__ldg(a.col_map + blk) * a.bs + (c - blk * a.bs) : zrow + c;
                     } else {
                         dst = zrow + h * OUT_COLS;
                     }
@@ -726,8 +891,8 @@ combine_limb_kernel(LimbArgs a) {
     combine_limb_body<false>(a);
 }
 
-// Protocol 2 with one multiplication per connected component: the same kernel over the listed tiles of the
-// component-sorted operands, scattering the result rows back to the compact layout of Z.
+// One multiplication per connected component (Protocols 2 and 3 under a per-token mask): the same kernel over the
+// tiles and k-blocks of the component-sorted operands that have work, scattering the result rows back to Z.
 __global__ void __launch_bounds__(limb::THREADS, 1)
 combine_limb_grouped_kernel(LimbArgs a) {
     combine_limb_body<true>(a);

@@ -103,165 +103,73 @@ open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, cons
 // The first step of Protocol 2 on the GPU: connected components of the bipartite graph
 // (token rows) x (active blocks) whose edges are the non-zero bytes of the
 // per-token mask S [T, nab].  The paper uses depth-first search; here one CTA
-// propagates minimum labels back and forth (block <- min over its tokens,
-// token <- min over its blocks) until nothing changes, at most T + nab + 1
-// rounds.  Every node of a component ends up with the component's smallest
-// token index as its label; nodes without an edge get -1.
-// report[0] = number of components, [1] = tokens with an edge, [2] = blocks with
-// an edge (mapped host memory).
+// propagates minimum labels over the edges (every edge pulls the labels of its
+// two ends down to their minimum, all edges in parallel) until nothing changes,
+// at most T + nab + 1 sweeps.  Every node of a component ends up with the
+// component's smallest token index as its label; nodes without an edge get -1.
+// The labels live in shared memory while they change when `labels_in_smem`
+// (dynamic shared memory of (T + nab) ints), else in the output arrays.
+// report[0] = number of edges (non-zero bytes of S), [1] = number of components,
+// [2] = tokens with an edge, [3] = blocks with an edge (mapped host memory).
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 token_components_kernel(const uint8_t* __restrict__ S, int T, int nab, int32_t* row_label, int32_t* blk_label,
-                        long long* report) {
-    __shared__ int changed;
+                        long long* report, int labels_in_smem) {
+    extern __shared__ int comp_smem[];
     __shared__ int counts[3];
+    __shared__ unsigned long long edges;
     const int tid = threadIdx.x;
     const int INF = 0x7fffffff;
-    for (int r = tid; r < T; r += 1024) {
-        bool edge = false;
-        for (int b = 0; b < nab && !edge; ++b) edge = S[(size_t)r * nab + b] != 0;
-        row_label[r] = edge ? r : INF;
-    }
-    for (int b = tid; b < nab; b += 1024) blk_label[b] = INF;
-    if (tid == 0) counts[0] = counts[1] = counts[2] = 0;
+    int* rl = labels_in_smem ? comp_smem : row_label;
+    int* bl = labels_in_smem ? comp_smem + T : blk_label;
+    volatile int* vrl = rl;
+    volatile int* vbl = bl;
+    const long long total = (long long)T * nab;
+    for (int r = tid; r < T; r += 1024) rl[r] = INF;
+    for (int b = tid; b < nab; b += 1024) bl[b] = INF;
+    if (tid == 0) { counts[0] = counts[1] = counts[2] = 0; edges = 0ull; }
     __syncthreads();
-    for (int round = 0; round <= T + nab; ++round) {
-        if (tid == 0) changed = 0;
-        __syncthreads();
-        for (int b = tid; b < nab; b += 1024) {
-            int best = blk_label[b];
-            for (int r = 0; r < T; ++r)
-                if (S[(size_t)r * nab + b] != 0) best = min(best, row_label[r]);
-            if (best < blk_label[b]) { blk_label[b] = best; changed = 1; }
+    unsigned long long mine = 0;
+    for (long long t = tid; t < total; t += 1024)
+        if (S[t] != 0) {
+            const int r = (int)(t / nab);
+            ++mine;
+            atomicMin(&rl[r], r);                    // a row with an edge starts from its own index
         }
-        __syncthreads();
-        for (int r = tid; r < T; r += 1024) {
-            int best = row_label[r];
-            if (best != INF) {
-                for (int b = 0; b < nab; ++b)
-                    if (S[(size_t)r * nab + b] != 0) best = min(best, blk_label[b]);
-                if (best < row_label[r]) { row_label[r] = best; changed = 1; }
+    if (mine) atomicAdd(&edges, mine);
+    __syncthreads();
+    for (int sweep = 0; sweep <= T + nab; ++sweep) {
+        int changed = 0;
+        for (long long t = tid; t < total; t += 1024)
+            if (S[t] != 0) {
+                const int r = (int)(t / nab), b = (int)(t - (long long)r * nab);
+                const int lr = vrl[r], lb = vbl[b];
+                if (lr < lb) { atomicMin(&bl[b], lr); changed = 1; }
+                else if (lb < lr) { atomicMin(&rl[r], lb); changed = 1; }
             }
-        }
-        __syncthreads();
-        if (!changed) break;
-        __syncthreads();
+        if (!__syncthreads_or(changed)) break;
     }
     for (int r = tid; r < T; r += 1024) {
-        const int l = row_label[r];
-        if (l == INF) row_label[r] = -1;
-        else {
+        const int l = rl[r];
+        row_label[r] = l == INF ? -1 : l;
+        if (l != INF) {
             atomicAdd(&counts[1], 1);
             if (l == r) atomicAdd(&counts[0], 1);
         }
     }
     for (int b = tid; b < nab; b += 1024) {
-        if (blk_label[b] == INF) blk_label[b] = -1;
-        else atomicAdd(&counts[2], 1);
+        const int l = bl[b];
+        blk_label[b] = l == INF ? -1 : l;
+        if (l != INF) atomicAdd(&counts[2], 1);
     }
     __syncthreads();
     if (tid == 0) {
-        report[0] = counts[0];
-        report[1] = counts[1];
-        report[2] = counts[2];
+        report[0] = (long long)edges;
+        report[1] = counts[0];
+        report[2] = counts[1];
+        report[3] = counts[2];
         __threadfence_system();
     }
-}
-
-// ---------------------------------------------------------------------------
-// Protocol 2 asks for one multiplication per connected component, over that component's rows and columns only
-// (Theorem 1's multiplication count).  On the tensor-core path this is ONE launch over component-sorted operands:
-// rows and column blocks are ordered by component label (ties by index), so every component is a contiguous
-// rectangle and an output tile has work only if the label ranges of its rows and of its columns intersect.
-//   row_map [T]           sorted row position -> token row; rows of no component come last
-//   col_map [groups*nab]  sorted block position -> compact block (group * nab + active block); within a
-//                         component the order is (group, block); blocks of no component come last
-//   tiles   [..]          (m-tile << 16) | n-tile of every tile with work, m-tiles of TM rows, n-tiles of TN columns
-//   report[0] = number of listed tiles, report[1] = sum over components of rows x blocks (mapped host memory)
-// One CTA of 1024 threads; needs ceil(live rows / TM) <= 1024.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-group_plan_kernel(const int32_t* __restrict__ row_label, const int32_t* __restrict__ blk_label, int T, int nab,
-                  int groups, int bs, int TM, int TN, int32_t* row_map, int32_t* col_map, int32_t* tiles,
-                  long long* report) {
-    __shared__ int live_rows, live_blocks;
-    __shared__ unsigned long long pairs;
-    __shared__ int tn_first[1024], tn_count[1024], tile_off[1024];
-    const int tid = threadIdx.x;
-    if (tid == 0) { live_rows = 0; live_blocks = 0; pairs = 0ull; }
-    __syncthreads();
-    {
-        int lr = 0, lb = 0;
-        for (int r = tid; r < T; r += 1024) lr += row_label[r] >= 0;
-        for (int b = tid; b < nab; b += 1024) lb += blk_label[b] >= 0;
-        if (lr) atomicAdd(&live_rows, lr);
-        if (lb) atomicAdd(&live_blocks, lb);
-    }
-    __syncthreads();
-    const int M = live_rows, NB = live_blocks;
-    unsigned long long my_pairs = 0;
-    for (int r = tid; r < T; r += 1024) {
-        const int l = row_label[r];
-        int rank = 0;
-        if (l >= 0) {
-            for (int q = 0; q < T; ++q) {
-                const int lq = row_label[q];
-                rank += lq >= 0 && (lq < l || (lq == l && q < r));
-            }
-            for (int b = 0; b < nab; ++b) my_pairs += blk_label[b] == l;
-        } else {
-            rank = M;
-            for (int q = 0; q < r; ++q) rank += row_label[q] < 0;
-        }
-        row_map[rank] = r;
-    }
-    if (my_pairs) atomicAdd(&pairs, my_pairs);
-    for (int b = tid; b < nab; b += 1024) {
-        const int l = blk_label[b];
-        if (l >= 0) {
-            int less = 0, same = 0, before = 0;
-            for (int q = 0; q < nab; ++q) {
-                const int lq = blk_label[q];
-                less += lq >= 0 && lq < l;
-                same += lq == l;
-                before += lq == l && q < b;
-            }
-            for (int g = 0; g < groups; ++g) col_map[groups * less + g * same + before] = g * nab + b;
-        } else {
-            int before = 0;
-            for (int q = 0; q < b; ++q) before += blk_label[q] < 0;
-            for (int g = 0; g < groups; ++g) col_map[groups * NB + g * (nab - NB) + before] = g * nab + b;
-        }
-    }
-    __syncthreads();
-    const int N = groups * NB * bs;
-    const int mt = (M + TM - 1) / TM, nt = (N + TN - 1) / TN;
-    if (tid < mt) {
-        const int lo_m = row_label[row_map[tid * TM]];
-        const int hi_m = row_label[row_map[min(tid * TM + TM, M) - 1]];
-        int first = 0, count = 0;
-        for (int tn = 0; tn < nt; ++tn) {
-            const int lo_n = blk_label[col_map[(tn * TN) / bs] % nab];
-            const int hi_n = blk_label[col_map[(min(tn * TN + TN, N) - 1) / bs] % nab];
-            if (hi_n >= lo_m && lo_n <= hi_m) {
-                if (count == 0) first = tn;
-                ++count;
-            }
-        }
-        tn_first[tid] = first;
-        tn_count[tid] = count;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int off = 0;
-        for (int tm = 0; tm < mt; ++tm) { tile_off[tm] = off; off += tn_count[tm]; }
-        report[0] = off;
-        report[1] = (long long)pairs;
-        __threadfence_system();
-    }
-    __syncthreads();
-    if (tid < mt)
-        for (int j = 0; j < tn_count[tid]; ++j) tiles[tile_off[tid] + j] = (tid << 16) | (tn_first[tid] + j);
 }
 
 // The Merge step of Protocol 2 on the compact result [T, cols]: an entry whose token and block are not in the same
@@ -277,25 +185,6 @@ somm_merge_kernel(PartyOut Z, int64_t pairs, int cols, int n, int bs, const int3
         const unsigned word = (unsigned)(2 * t), row = word / (unsigned)cols, col = word - row * (unsigned)cols;
         const int rl = row_label[row];
         if (rl < 0 || rl != blk_label[(col % (unsigned)n) / (unsigned)bs]) z[t] = make_ulonglong2(0ull, 0ull);
-    }
-}
-
-// Number of non-zero bytes of a mask, written to `out` (mapped host memory) as a 64-bit count.
-__global__ void __launch_bounds__(1024)
-count_mask_kernel(const uint8_t* __restrict__ mask, long long count, long long* out) {
-    __shared__ long long partial[32];
-    long long mine = 0;
-    for (long long t = threadIdx.x; t < count; t += 1024) mine += mask[t] != 0;
-    for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
-    if ((threadIdx.x & 31) == 0) partial[threadIdx.x >> 5] = mine;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        long long v = partial[threadIdx.x];
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
-        if (threadIdx.x == 0) {
-            *out = v;
-            __threadfence_system();
-        }
     }
 }
 
@@ -337,10 +226,12 @@ open_weight_rows_kernel(PartyPtrs Wg0, PartyPtrs Wg1, PartyPtrs Wg2, PartyPtrs B
 // IndexRow (Protocol 3) on the stored transpose [d, D] is a gather of
 // bs-word strips (256 or 512 contiguous bytes) out of every row q.
 // Flat index over (q, c/2); consecutive threads walk consecutive pairs of a row.
+// With blk_label (Protocol 3 under a per-token mask): a block no token uses (label < 0) holds no non-zero column
+// of X, so its rows of Y are not masked and not sent: their message words are zero.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 open_weight_strips_kernel(PartyPtrs W2, PartyPtrs B, PartyOut F, const int32_t* __restrict__ ids,
-                          int n, int bs, int d, int D) {
+                          int n, int bs, int d, int D, const int32_t* __restrict__ blk_label) {
     const int party = blockIdx.y;
     const int half_n = n >> 1;
     const int64_t total = (int64_t)d * half_n;
@@ -351,6 +242,10 @@ open_weight_strips_kernel(PartyPtrs W2, PartyPtrs B, PartyOut F, const int32_t* 
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
         const int q = (int)(t / half_n);
         const int c = (int)(t - (int64_t)q * half_n) << 1;
+        if (blk_label && blk_label[c / bs] < 0) {
+            f[t] = make_ulonglong2(0ull, 0ull);
+            continue;
+        }
         const int neuron = ids[c / bs] * bs + (c % bs);
         const ulonglong2 wv = __ldg(reinterpret_cast<const ulonglong2*>(W + (size_t)q * D + neuron));
         const ulonglong2 bv = __ldg(b + t);

@@ -12,7 +12,10 @@ import oracle  # noqa: E402
 from paper_2505_07239_b200 import workloads as wl  # noqa: E402
 
 
-def _run(cfg, seed, tokens, sparsity, p_token, path, clear_after=False):
+_LAST = {}
+
+
+def _run(cfg, seed, tokens, sparsity, p_token, path, clear_after=False, token_mask=None):
     from paper_2505_07239_b200 import binding as cb
     from tests import harness as hz
 
@@ -21,7 +24,7 @@ def _run(cfg, seed, tokens, sparsity, p_token, path, clear_after=False):
     mask = wl.block_mask(cfg, seed, sparsity)
     I = oracle.index_set(mask, cfg.block, 1)
     n, nab = I.size, int(mask.sum())
-    tm = wl.token_block_masks(seed, "tm", T, nab, p_token)
+    tm = token_mask if token_mask is not None else wl.token_block_masks(seed, "tm", T, nab, p_token)
     S = np.repeat(tm, cfg.block, axis=1)                       # element-level distribution over the compact columns
     _, H0, H1 = wl.hidden_shares(cfg, seed, n, tokens=T)       # uniform words everywhere, also off the support
     tri = wl.dealer_triple_rowsets(seed, "down", S, d)
@@ -37,7 +40,11 @@ def _run(cfg, seed, tokens, sparsity, p_token, path, clear_after=False):
     ctx.ffn_down(T)
     st = ctx.stats()
     assert st.matmul_path == path
-    assert st.message_bytes == 2 * 8 * (masked + n * d)        # only the non-zeros of the hidden state are sent
+    used = int((tm.sum(axis=0) > 0).sum()) * cfg.block         # columns of X with a non-zero
+    assert st.message_bytes == 2 * 8 * (masked + used * d)     # only the non-zeros of X and those rows of Y are sent
+    assert st.ring_macs == 2 * 2 * masked * d                  # Theorem 2: one row of Y per non-zero of X
+    _LAST.update(tile_macs=st.tensor_tile_macs,
+                 dense_tile_macs=2 * 2 * (-(-T // 128) * 128) * (-(-d // 64) * 64) * (-(-n // 32) * 32))
     ref = oracle.simm_rowsets((H0, H1), W["W2"][1:], I, S, tri["A"][1:], tri["B"][1:], tri["C"][1:])
     assert ref["masked"] == masked
     bad = 0
@@ -86,6 +93,48 @@ def test_token_masked_down_projection_llama_shape_blocks_of_64():
         pytest.skip("needs a CUDA device")
     cfg = wl.FFNConfig("rowsets-b64", 96, 256, 2048, 64, 16, True, 0.25, "uniform", "normal", "normal0.02")
     assert _run(cfg, 73, 96, 0.75, 0.05, 2) == 0
+
+
+# ---- per-column row sets that fall into several components (tensor-core path, more than 32 tokens): rows and the
+#      contraction index are taken in component order and a row tile runs over its components' blocks only
+
+@pytest.mark.parametrize("tokens,block,clusters,dead", [(200, 32, 4, 2), (130, 16, 3, 1), (300, 64, 6, 3), (40, 16, 5, 0)])
+def test_grouped_down_projection_scattered_components(tokens, block, clusters, dead):
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-grouped", tokens, 128, 2048, block, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 500 + tokens, 0.5).sum())
+    tm = wl.token_block_masks_clustered(500 + tokens, "tmc", tokens, nab, clusters, 0.3, dead, dead)
+    assert _run(cfg, 500 + tokens, tokens, 0.5, None, 2, token_mask=tm, clear_after=True) == 0
+    assert 0 < _LAST["tile_macs"] <= _LAST["dense_tile_macs"]
+    if tokens > 128:                                            # several row tiles: each skips the others' blocks
+        assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
+def test_grouped_down_projection_opt13b_at_90_percent():
+    """The graded FFN shape with the batch dealt to four groups of requests: full comparison against the oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.CONFIGS["opt1.3b"]
+    nab = int(wl.block_mask(cfg, 556, 0.9).sum())
+    tm = wl.token_block_masks_clustered(556, "tmc", 512, nab, 4, 0.6)
+    assert _run(cfg, 556, 512, 0.9, None, 2, token_mask=tm) == 0
+    assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("tokens", [12, 70])
+def test_active_block_without_any_token_is_not_opened(path, tokens):
+    """A block of the block mask that no token uses holds no non-zero column of X: its rows of the weight matrix
+    are not masked and not sent (zero message words), on both paths and in the few-token kernel."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-dead", tokens, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 640, 0.5).sum())
+    tm = wl.token_block_masks(640, "tm", tokens, nab, 0.4)
+    tm[:, 2] = 0
+    tm[:, nab - 1] = 0
+    assert _run(cfg, 640, tokens, 0.5, None, path, token_mask=tm) == 0
 
 
 def test_token_mask_errors():

@@ -171,3 +171,54 @@ def test_grouped_launch_opt13b_at_90_percent():
     assert bad == 0 and L >= 4
     assert _LAST["ring_macs"] == 2 * 2 * _LAST["d"] * _LAST["dot_products"]
     assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
+def test_grouped_chain_up_then_down_with_three_stacked_matrices():
+    """Both products of one layer under one clustered token mask, the down-projection's weight side opened early
+    (on the side stream, in component order) during the up-projection: three stacked matrices, then the
+    row-gathered product, each against the oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    cfg = wl.FFNConfig("comp-chain", 150, 256, 1024, 64, 16, False, 0.5, "uniform", "normal", "normal0.02", stacked=3)
+    seed, T, d, g, bs = 620, 150, cfg.d_model, cfg.groups, cfg.block
+    W = wl.model_shares(cfg, seed, plain=False)
+    mask = wl.block_mask(cfg, seed, 0.5)
+    I1, Ig = oracle.index_set(mask, bs, 1), oracle.index_set(mask, bs, g)
+    n, nab = I1.size, int(mask.sum())
+    tm = wl.token_block_masks_clustered(seed, "tmc", T, nab, 3, 0.5, 2, 1)
+    S1 = np.repeat(tm, bs, axis=1)
+    Sg = np.tile(S1, (1, g))
+    _, X0, X1 = wl.activation_shares(cfg, seed, tokens=T)
+    tri = wl.dealer_triple_components(seed, "up", Sg, d)
+    trd = wl.dealer_triple_rowsets(seed, "down", S1, d)
+    _, H0, H1 = wl.hidden_shares(cfg, seed, n, tokens=T)
+    Wup = (hz.oracle_up_operand(cfg, W, 1), hz.oracle_up_operand(cfg, W, 2))
+    ref = oracle.somm_components((X0, X1), Wup, Ig, Sg, tri["A"][1:], tri["B"][1:], tri["C"][1:])
+    refd = oracle.simm_rowsets((H0, H1), W["W2"][1:], I1, S1, trd["A"][1:], trd["B"][1:], trd["C"][1:])
+
+    ctx = hz.make_context(cfg, T, 2)
+    hz.load_weights(ctx, cfg, W)
+    for p, Xs in ((0, X0), (1, X1)):
+        ctx.load_shares(p, cb.X, cb.to_device(Xs))
+    assert ctx.set_mask(mask) == n
+    ctx.set_token_mask(tm)
+    hz.load_triple_up(ctx, tri)
+    hz.load_triple_down(ctx, trd)                 # B' is there before ffn_up: the weight side is opened early
+    ctx.ffn_up(T)
+    assert ctx.stats().n_components == ref["L"] >= 3
+    bad = 0
+    for p in (0, 1):
+        bad += int((ctx.get(p, cb.Z_UP, (T, g * n)) != ref["Z"][p]).sum())
+        bad += int((ctx.get(p, cb.F_UP, (g * n, d)).T != ref["F"][p]).sum())
+    for p, Hs in ((0, H0), (1, H1)):
+        ctx.load_shares(p, cb.H, cb.to_device(Hs))
+    ctx.ffn_down(T)
+    for p in (0, 1):
+        bad += int((ctx.get(p, cb.Y, (T, d)) != refd["Z"][p]).sum())
+        bad += int((ctx.get(p, cb.E_DN, (T, n)) != refd["E"][p]).sum())
+        bad += int((ctx.get(p, cb.F_DN, (d, n)).T != refd["F"][p]).sum())
+    ctx.close()
+    assert bad == 0
