@@ -50,7 +50,8 @@ struct comet_ctx {
     bool tmask_set;
     int32_t tmask_tokens;
     int64_t tmask_masked;         // non-zero entries of the hidden state under the token mask (neurons, not blocks)
-    long long* h_masked;          // pinned and mapped: [0..3] token_components_kernel's report, [4..6] group_plan_kernel's
+    long long* h_masked;          // pinned and mapped: token_plan_kernel's report [0..6]
+    uint32_t* d_plan_scratch;     // its working storage when that does not fit into shared memory
     long long* h_masked_dev;
     int32_t* d_row_label;         // component label per token row / per active block under the token mask
     int32_t* d_blk_label;
@@ -525,6 +526,8 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     ok = ok && cudaMalloc((void**)&c->d_row_map, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_col_map, (size_t)c->groups * nb * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_kmap, (size_t)nb * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->d_plan_scratch,
+                          ((size_t)c->cap_T * ceil_div(nb, 32) + (size_t)c->groups * nb) * sizeof(uint32_t)) == cudaSuccess;
     {
         const size_t mt = ceil_div((int)c->cap_T, comet::limb::BM);
         ok = ok && cudaMalloc((void**)&c->d_group_up, mt * sizeof(comet::LimbGroupRow)) == cudaSuccess;
@@ -573,6 +576,7 @@ void comet_destroy(comet_ctx* c) {
     if (c->d_row_map) cudaFree(c->d_row_map);
     if (c->d_col_map) cudaFree(c->d_col_map);
     if (c->d_kmap) cudaFree(c->d_kmap);
+    if (c->d_plan_scratch) cudaFree(c->d_plan_scratch);
     if (c->d_group_up) cudaFree(c->d_group_up);
     if (c->d_group_dn) cudaFree(c->d_group_dn);
     if (c->d_blk_label) cudaFree(c->d_blk_label);
@@ -713,25 +717,29 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     if ((int64_t)tokens * c->n_active < 0 || (int64_t)tokens * c->n_active > 0x7fffffffll) return COMET_ERR_SHAPE;
     const size_t bytes = (size_t)tokens * (size_t)n_active_blocks;
     COMET_CUDA(c, cudaMemcpyAsync(c->d_tmask, token_mask, bytes, copy_kind(location, true), c->stream));
-    // Protocol 2, first step: the connected components the up-projection is partitioned into (and the number of
-    // non-zero entries, Theorem 2's count)
+    // Protocol 2, first step: the connected components the up-projection is partitioned into, the number of
+    // non-zero entries (Theorem 2's count) and, for the tensor-core path, the component-sorted order and the work
+    // of every row tile, in one launch
+    const bool plan = c->path == COMET_PATH_LIMB && tokens > comet::limb_few::BT && tokens <= 32768;
     {
-        const size_t label_bytes = ((size_t)tokens + (size_t)n_active_blocks) * sizeof(int);
-        const bool in_smem = label_bytes <= 40 * 1024;
-        comet::token_components_kernel<<<1, 1024, in_smem ? label_bytes : 0, c->stream>>>(
-            c->d_tmask, tokens, n_active_blocks, c->d_row_label, c->d_blk_label, c->h_masked_dev, in_smem ? 1 : 0);
+        comet::TokenPlanArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.S = c->d_tmask;
+        a.T = tokens; a.nab = n_active_blocks; a.wpr = ceil_div(n_active_blocks, 32);
+        a.row_label = c->d_row_label; a.blk_label = c->d_blk_label;
+        a.report = c->h_masked_dev;
+        a.scratch = c->d_plan_scratch;
+        a.plan = plan ? 1 : 0;
+        a.groups = c->groups; a.bs = c->cfg.block;
+        a.kb_up = ceil_div(c->cfg.d_model, comet::limb::KC);
+        a.nt_dn = ceil_div(c->cfg.d_model, comet::limb::BN);
+        a.row_map = c->d_row_map; a.col_map = c->d_col_map; a.kmap = c->d_kmap;
+        a.up = c->d_group_up; a.dn = c->d_group_dn;
+        const size_t words = (size_t)tokens * a.wpr + tokens + (size_t)n_active_blocks * (1 + c->groups);
+        a.in_smem = words * sizeof(uint32_t) <= 36 * 1024 ? 1 : 0;
+        comet::token_plan_kernel<<<1, 1024, a.in_smem ? words * sizeof(uint32_t) : 0, c->stream>>>(a);
     }
     c->stats.kernel_launches += 1;
-    // ... and, for the tensor-core path, the component-sorted order and the output tiles that have work
-    const bool plan = c->path == COMET_PATH_LIMB && tokens > comet::limb_few::BT &&
-                      ceil_div(tokens, comet::limb::BM) <= 1024;
-    if (plan) {
-        comet::group_plan_kernel<<<1, 1024, 0, c->stream>>>(
-            c->d_row_label, c->d_blk_label, tokens, n_active_blocks, c->groups, c->cfg.block,
-            ceil_div(c->cfg.d_model, comet::limb::KC), ceil_div(c->cfg.d_model, comet::limb::BN), c->d_row_map,
-            c->d_col_map, c->d_kmap, c->d_group_up, c->d_group_dn, c->h_masked_dev + 4);
-        c->stats.kernel_launches += 1;
-    }
     COMET_CUDA(c, cudaGetLastError());
     COMET_CUDA(c, cudaStreamSynchronize(c->stream));
     c->tmask_masked = (int64_t)c->h_masked[0] * c->cfg.block;

@@ -419,22 +419,35 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 }  // namespace ptx
 
 // ---------------------------------------------------------------------------
-// Protocols 2 and 3 ask for one multiplication per connected component / per non-zero column entry, over the
-// rows and columns that take part only (the multiplication counts of Theorems 1 and 2).  On the tensor cores this
-// becomes ONE launch over component-sorted operands: token rows and active blocks are ordered by component label
-// (ties by index), so every component is a contiguous rectangle, and
-//   up   (Protocol 2): an output tile has work only if the label ranges of its rows and of its columns intersect;
-//                      per row tile these column tiles form an interval;
-//   down (Protocol 3): a row tile's contraction runs only over the blocks of the components its rows belong to,
-//                      an interval of k-blocks in the sorted order of the contraction index.
-//   row_map [T]           sorted row position -> token row; rows of no component come last
-//   col_map [groups*nab]  sorted block position -> compact block (group * nab + active block) of the up-projection's
-//                         columns; within a component the order is (group, block); blocks of no component last
-//   kmap    [nab]         sorted block position -> active block, for the down-projection's contraction index
-//   up, dn  [row tiles]   the work of every tile of 128 sorted rows (LimbGroupRow)
-//   report[0] = k-block units of the up-projection per party, [1] = sum over components of rows x blocks,
-//   report[2] = units of the down-projection per party (mapped host memory)
-// One CTA of 1024 threads; needs ceil(live rows / 128) <= 1024.
+// What a per-token mask S [T, nab] (non-zero byte = token t uses active block b) implies, in one launch of one CTA.
+//
+// 1. The first step of Protocol 2: the connected components of the bipartite graph (token rows) x (active
+//    blocks) with the non-zero bytes as edges.  The paper uses depth-first search; here S becomes a bit matrix
+//    and minimum labels are propagated: every row takes the minimum over its blocks and pushes it to them, all
+//    rows in parallel, until nothing changes (at most T + nab + 1 sweeps).  Every node of a component ends up with
+//    the component's smallest token index as its label; nodes without an edge get -1.
+//
+// 2. (plan != 0) Protocols 2 and 3 ask for one multiplication per component / per non-zero column entry, over the
+//    rows and columns that take part only (the multiplication counts of Theorems 1 and 2).  On the tensor cores
+//    this becomes ONE launch over component-sorted operands: token rows and active blocks are ordered by
+//    component label (ties by index), so every component is a contiguous rectangle, and
+//      up   (Protocol 2): an output tile has work only if the label ranges of its rows and of its columns
+//                         intersect; per row tile these column tiles form an interval;
+//      down (Protocol 3): a row tile's contraction runs only over the blocks of the components its rows belong
+//                         to, an interval of k-blocks in the sorted order of the contraction index.
+//    row_map [T]           sorted row position -> token row; rows of no component come last
+//    col_map [groups*nab]  sorted block position -> compact block (group * nab + active block) of the
+//                          up-projection's columns; inside a component the order is (group, block); blocks of no
+//                          component last
+//    kmap    [nab]         sorted block position -> active block, for the down-projection's contraction index
+//    up, dn  [row tiles]   the work of every tile of 128 sorted rows (LimbGroupRow); needs at most 32768 tokens
+//
+// report (mapped host memory): [0] edges, [1] components, [2] rows with an edge, [3] blocks with an edge,
+// [4] k-block units of the up-projection per party, [5] sum over components of rows x blocks, [6] units of the
+// down-projection per party ([4..6] only with plan).
+// Working storage: bit matrix [T, wpr] words, labels, and the labels of the sorted column blocks, in dynamic
+// shared memory when `in_smem` (T*wpr + T + nab + groups*nab words), else in `scratch` (global, same size) with
+// the labels kept in the output arrays.
 // ---------------------------------------------------------------------------
 struct LimbGroupRow {
     int unit0;       // units (k-blocks, both operand pairs) of the row tiles before this one, per party
@@ -442,107 +455,229 @@ struct LimbGroupRow {
     int klo, kcnt;   // interval of k-blocks with work; a tile runs over 2 * kcnt units
 };
 
-__global__ void __launch_bounds__(1024)
-group_plan_kernel(const int32_t* __restrict__ row_label, const int32_t* __restrict__ blk_label, int T, int nab,
-                  int groups, int bs, int kb_up, int nt_dn, int32_t* row_map, int32_t* col_map, int32_t* kmap,
-                  LimbGroupRow* up, LimbGroupRow* dn, long long* report) {
+struct TokenPlanArgs {
+    const uint8_t* S;
+    int T, nab, wpr;             // wpr = ceil(nab / 32)
+    int32_t* row_label;          // out [T]
+    int32_t* blk_label;          // out [nab]
+    long long* report;
+    int in_smem;
+    uint32_t* scratch;
+    int plan, groups, bs, kb_up, nt_dn;
+    int32_t* row_map;
+    int32_t* col_map;
+    int32_t* kmap;
+    LimbGroupRow* up;
+    LimbGroupRow* dn;
+};
+
+__global__ void __launch_bounds__(1024, 1)
+token_plan_kernel(TokenPlanArgs a) {
     constexpr int TM = limb::BM, TN = limb::BN, KC = limb::KC;
-    __shared__ int live_rows, live_blocks;
-    __shared__ unsigned long long pairs;
+    extern __shared__ uint32_t plan_smem[];
+    __shared__ int counts[3];
+    __shared__ unsigned long long edges, pairs;
     __shared__ int units_up[1024], units_dn[1024];
     const int tid = threadIdx.x;
-    if (tid == 0) { live_rows = 0; live_blocks = 0; pairs = 0ull; }
+    const int T = a.T, nab = a.nab, wpr = a.wpr;
+    const int INF = 0x7fffffff;
+    uint32_t* bits = a.in_smem ? plan_smem : a.scratch;
+    int* rl = a.in_smem ? reinterpret_cast<int*>(plan_smem + (size_t)T * wpr) : a.row_label;
+    int* bl = a.in_smem ? rl + T : a.blk_label;
+    int* sorted_bl = a.in_smem ? bl + nab : reinterpret_cast<int*>(a.scratch + (size_t)T * wpr);
+
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int w = tid; w < T * wpr; w += 1024) bits[w] = 0u;
+    for (int b = tid; b < nab; b += 1024) bl[b] = INF;
+    if (tid == 0) { counts[0] = counts[1] = counts[2] = 0; edges = 0ull; pairs = 0ull; }
     __syncthreads();
     {
-        int lr = 0, lb = 0;
-        for (int r = tid; r < T; r += 1024) lr += row_label[r] >= 0;
-        for (int b = tid; b < nab; b += 1024) lb += blk_label[b] >= 0;
-        if (lr) atomicAdd(&live_rows, lr);
-        if (lb) atomicAdd(&live_blocks, lb);
+        // S is read four bytes at a time (its buffer is 256-byte aligned); the last 0-3 bytes singly
+        const int total = T * nab, words = total >> 2;
+        const uint32_t* S4 = reinterpret_cast<const uint32_t*>(a.S);
+        for (int q = tid; q < words; q += 1024) {
+            uint32_t v = __ldg(S4 + q);
+            if (v == 0u) continue;
+#pragma unroll
+            for (int k = 0; k < 4; ++k, v >>= 8)
+                if (v & 0xffu) {
+                    const int t = 4 * q + k, r = t / nab, b = t - r * nab;
+                    atomicOr(&bits[r * wpr + (b >> 5)], 1u << (b & 31));
+                }
+        }
+        for (int t = 4 * words + tid; t < total; t += 1024)
+            if (a.S[t] != 0) {
+                const int r = t / nab, b = t - r * nab;
+                atomicOr(&bits[r * wpr + (b >> 5)], 1u << (b & 31));
+            }
     }
     __syncthreads();
-    const int M = live_rows, NB = live_blocks;
+    {
+        int mine = 0;
+        for (int r = tid; r < T; r += 1024) {
+            int deg = 0;
+            for (int w = 0; w < wpr; ++w) deg += __popc(bits[r * wpr + w]);
+            rl[r] = deg ? r : INF;               // a row with an edge starts from its own index
+            mine += deg;
+        }
+        mine = __reduce_add_sync(0xffffffffu, mine);
+        if (lane == 0 && mine) atomicAdd(&edges, (unsigned long long)mine);
+    }
+    __syncthreads();
+    for (int sweep = 0; sweep <= T + nab; ++sweep) {
+        int changed = 0;
+        // blocks take the minimum over their rows: one warp per block, no atomics
+        for (int b = warp; b < nab; b += 32) {
+            const int w = b >> 5;
+            const uint32_t bit = 1u << (b & 31);
+            int m = INF;
+            for (int r = lane; r < T; r += 32)
+                if (bits[r * wpr + w] & bit) m = min(m, rl[r]);
+            m = __reduce_min_sync(0xffffffffu, m);
+            if (lane == 0 && m < bl[b]) { bl[b] = m; changed = 1; }
+        }
+        __syncthreads();
+        // rows take the minimum over their blocks
+        for (int r = tid; r < T; r += 1024) {
+            const int mine = rl[r];
+            if (mine == INF) continue;
+            int m = mine;
+            for (int w = 0; w < wpr; ++w)
+                for (uint32_t v = bits[r * wpr + w]; v; v &= v - 1) m = min(m, bl[w * 32 + __ffs(v) - 1]);
+            if (m < mine) { rl[r] = m; changed = 1; }
+        }
+        if (!__syncthreads_or(changed)) break;
+    }
+    {
+        int comps = 0, live_r = 0, live_b = 0;
+        for (int r = tid; r < T; r += 1024) {
+            const int l = rl[r];
+            if (l == INF) rl[r] = -1;
+            else {
+                ++live_r;
+                comps += l == r;
+            }
+            a.row_label[r] = l == INF ? -1 : l;
+        }
+        for (int b = tid; b < nab; b += 1024) {
+            const int l = bl[b];
+            if (l == INF) bl[b] = -1;
+            else ++live_b;
+            a.blk_label[b] = l == INF ? -1 : l;
+        }
+        comps = __reduce_add_sync(0xffffffffu, comps);
+        live_r = __reduce_add_sync(0xffffffffu, live_r);
+        live_b = __reduce_add_sync(0xffffffffu, live_b);
+        if (lane == 0) {
+            if (comps) atomicAdd(&counts[0], comps);
+            if (live_r) atomicAdd(&counts[1], live_r);
+            if (live_b) atomicAdd(&counts[2], live_b);
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        a.report[0] = (long long)edges;
+        a.report[1] = counts[0];
+        a.report[2] = counts[1];
+        a.report[3] = counts[2];
+        if (!a.plan) __threadfence_system();
+    }
+    if (!a.plan) return;
+
+    // ---- component-sorted order
+    const int M = counts[1], NB = counts[2], groups = a.groups, bs = a.bs;
+    // rank of a row = number of rows with a smaller key label * T + row; rows of no component take T for the
+    // label and so come last, in index order.  T <= 32768 keeps the key within 32 bits.
     unsigned long long my_pairs = 0;
     for (int r = tid; r < T; r += 1024) {
-        const int l = row_label[r];
-        int rank = 0;
-        if (l >= 0) {
-            for (int q = 0; q < T; ++q) {
-                const int lq = row_label[q];
-                rank += lq >= 0 && (lq < l || (lq == l && q < r));
-            }
-            for (int b = 0; b < nab; ++b) my_pairs += blk_label[b] == l;
-        } else {
-            rank = M;
-            for (int q = 0; q < r; ++q) rank += row_label[q] < 0;
+        const int l = rl[r];
+        const unsigned key = (l >= 0 ? (unsigned)l : (unsigned)T) * (unsigned)T + (unsigned)r;
+        int rank0 = 0, rank1 = 0;
+        int q = 0;
+        for (; q + 1 < T; q += 2) {
+            const int l0 = rl[q], l1 = rl[q + 1];
+            rank0 += (l0 >= 0 ? (unsigned)l0 : (unsigned)T) * (unsigned)T + (unsigned)q < key;
+            rank1 += (l1 >= 0 ? (unsigned)l1 : (unsigned)T) * (unsigned)T + (unsigned)(q + 1) < key;
         }
-        row_map[rank] = r;
+        if (q < T) rank0 += (rl[q] >= 0 ? (unsigned)rl[q] : (unsigned)T) * (unsigned)T + (unsigned)q < key;
+        a.row_map[rank0 + rank1] = r;
+        if (l >= 0)
+            for (int b = 0; b < nab; ++b) my_pairs += bl[b] == l;
     }
-    if (my_pairs) atomicAdd(&pairs, my_pairs);
+    my_pairs = __reduce_add_sync(0xffffffffu, (unsigned)my_pairs);
+    if (lane == 0 && my_pairs) atomicAdd(&pairs, my_pairs);
     for (int b = tid; b < nab; b += 1024) {
-        const int l = blk_label[b];
+        const int l = bl[b];
         if (l >= 0) {
             int less = 0, same = 0, before = 0;
             for (int q = 0; q < nab; ++q) {
-                const int lq = blk_label[q];
+                const int lq = bl[q];
                 less += lq >= 0 && lq < l;
                 same += lq == l;
                 before += lq == l && q < b;
             }
-            for (int g = 0; g < groups; ++g) col_map[groups * less + g * same + before] = g * nab + b;
-            kmap[less + before] = b;
+            for (int g = 0; g < groups; ++g) {
+                a.col_map[groups * less + g * same + before] = g * nab + b;
+                sorted_bl[groups * less + g * same + before] = l;
+            }
+            a.kmap[less + before] = b;
         } else {
             int before = 0;
-            for (int q = 0; q < b; ++q) before += blk_label[q] < 0;
-            for (int g = 0; g < groups; ++g) col_map[groups * NB + g * (nab - NB) + before] = g * nab + b;
-            kmap[NB + before] = b;
+            for (int q = 0; q < b; ++q) before += bl[q] < 0;
+            for (int g = 0; g < groups; ++g) {
+                a.col_map[groups * NB + g * (nab - NB) + before] = g * nab + b;
+                sorted_bl[groups * NB + g * (nab - NB) + before] = -1;
+            }
+            a.kmap[NB + before] = b;
         }
     }
     __syncthreads();
+
+    // ---- the work of every row tile
     const int N = groups * NB * bs;
     const int mt = (M + TM - 1) / TM, nt = (N + TN - 1) / TN;
     if (tid < mt) {
-        const int lo_m = row_label[row_map[tid * TM]];
-        const int hi_m = row_label[row_map[min(tid * TM + TM, M) - 1]];
+        const int lo_m = rl[a.row_map[tid * TM]];
+        const int hi_m = rl[a.row_map[min(tid * TM + TM, M) - 1]];
         int first = 0, count = 0;
         for (int tn = 0; tn < nt; ++tn) {
-            const int lo_n = blk_label[col_map[(tn * TN) / bs] % nab];
-            const int hi_n = blk_label[col_map[(min(tn * TN + TN, N) - 1) / bs] % nab];
+            const int lo_n = sorted_bl[(tn * TN) / bs];
+            const int hi_n = sorted_bl[(min(tn * TN + TN, N) - 1) / bs];
             if (hi_n >= lo_m && lo_n <= hi_m) {
                 if (count == 0) first = tn;
                 ++count;
             }
         }
-        up[tid].tn0 = first;
-        up[tid].ntn = count;
-        up[tid].klo = 0;
-        up[tid].kcnt = kb_up;
-        units_up[tid] = count * 2 * kb_up;
+        a.up[tid].tn0 = first;
+        a.up[tid].ntn = count;
+        a.up[tid].klo = 0;
+        a.up[tid].kcnt = a.kb_up;
+        units_up[tid] = count * 2 * a.kb_up;
         int blk_begin = 0, blk_end = 0;          // sorted block positions of the components lo_m .. hi_m
         for (int q = 0; q < nab; ++q) {
-            const int lq = blk_label[q];
+            const int lq = bl[q];
             blk_begin += lq >= 0 && lq < lo_m;
             blk_end += lq >= 0 && lq <= hi_m;
         }
         const int klo = (blk_begin * bs) / KC, khi = (blk_end * bs + KC - 1) / KC;
-        dn[tid].tn0 = 0;
-        dn[tid].ntn = nt_dn;
-        dn[tid].klo = klo;
-        dn[tid].kcnt = khi - klo;
-        units_dn[tid] = nt_dn * 2 * (khi - klo);
+        a.dn[tid].tn0 = 0;
+        a.dn[tid].ntn = a.nt_dn;
+        a.dn[tid].klo = klo;
+        a.dn[tid].kcnt = khi - klo;
+        units_dn[tid] = a.nt_dn * 2 * (khi - klo);
     }
     __syncthreads();
     if (tid == 0) {
         int off_up = 0, off_dn = 0;
         for (int tm = 0; tm < mt; ++tm) {
-            up[tm].unit0 = off_up;
-            dn[tm].unit0 = off_dn;
+            a.up[tm].unit0 = off_up;
+            a.dn[tm].unit0 = off_dn;
             off_up += units_up[tm];
             off_dn += units_dn[tm];
         }
-        report[0] = off_up;
-        report[1] = (long long)pairs;
-        report[2] = off_dn;
+        a.report[4] = off_up;
+        a.report[5] = (long long)pairs;
+        a.report[6] = off_dn;
         __threadfence_system();
     }
 }

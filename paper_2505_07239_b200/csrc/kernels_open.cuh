@@ -99,79 +99,6 @@ open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, cons
     }
 }
 
-// ---------------------------------------------------------------------------
-// The first step of Protocol 2 on the GPU: connected components of the bipartite graph
-// (token rows) x (active blocks) whose edges are the non-zero bytes of the
-// per-token mask S [T, nab].  The paper uses depth-first search; here one CTA
-// propagates minimum labels over the edges (every edge pulls the labels of its
-// two ends down to their minimum, all edges in parallel) until nothing changes,
-// at most T + nab + 1 sweeps.  Every node of a component ends up with the
-// component's smallest token index as its label; nodes without an edge get -1.
-// The labels live in shared memory while they change when `labels_in_smem`
-// (dynamic shared memory of (T + nab) ints), else in the output arrays.
-// report[0] = number of edges (non-zero bytes of S), [1] = number of components,
-// [2] = tokens with an edge, [3] = blocks with an edge (mapped host memory).
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-token_components_kernel(const uint8_t* __restrict__ S, int T, int nab, int32_t* row_label, int32_t* blk_label,
-                        long long* report, int labels_in_smem) {
-    extern __shared__ int comp_smem[];
-    __shared__ int counts[3];
-    __shared__ unsigned long long edges;
-    const int tid = threadIdx.x;
-    const int INF = 0x7fffffff;
-    int* rl = labels_in_smem ? comp_smem : row_label;
-    int* bl = labels_in_smem ? comp_smem + T : blk_label;
-    volatile int* vrl = rl;
-    volatile int* vbl = bl;
-    const long long total = (long long)T * nab;
-    for (int r = tid; r < T; r += 1024) rl[r] = INF;
-    for (int b = tid; b < nab; b += 1024) bl[b] = INF;
-    if (tid == 0) { counts[0] = counts[1] = counts[2] = 0; edges = 0ull; }
-    __syncthreads();
-    unsigned long long mine = 0;
-    for (long long t = tid; t < total; t += 1024)
-        if (S[t] != 0) {
-            const int r = (int)(t / nab);
-            ++mine;
-            atomicMin(&rl[r], r);                    // a row with an edge starts from its own index
-        }
-    if (mine) atomicAdd(&edges, mine);
-    __syncthreads();
-    for (int sweep = 0; sweep <= T + nab; ++sweep) {
-        int changed = 0;
-        for (long long t = tid; t < total; t += 1024)
-            if (S[t] != 0) {
-                const int r = (int)(t / nab), b = (int)(t - (long long)r * nab);
-                const int lr = vrl[r], lb = vbl[b];
-                if (lr < lb) { atomicMin(&bl[b], lr); changed = 1; }
-                else if (lb < lr) { atomicMin(&rl[r], lb); changed = 1; }
-            }
-        if (!__syncthreads_or(changed)) break;
-    }
-    for (int r = tid; r < T; r += 1024) {
-        const int l = rl[r];
-        row_label[r] = l == INF ? -1 : l;
-        if (l != INF) {
-            atomicAdd(&counts[1], 1);
-            if (l == r) atomicAdd(&counts[0], 1);
-        }
-    }
-    for (int b = tid; b < nab; b += 1024) {
-        const int l = bl[b];
-        blk_label[b] = l == INF ? -1 : l;
-        if (l != INF) atomicAdd(&counts[2], 1);
-    }
-    __syncthreads();
-    if (tid == 0) {
-        report[0] = (long long)edges;
-        report[1] = counts[0];
-        report[2] = counts[1];
-        report[3] = counts[2];
-        __threadfence_system();
-    }
-}
-
 // The Merge step of Protocol 2 on the compact result [T, cols]: an entry whose token and block are not in the same
 // component is no part of any result block and is zero in both shares.  Compact column c belongs to active block
 // (c mod n) / bs.  `pairs` = 16-byte word pairs per party.

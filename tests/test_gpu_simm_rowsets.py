@@ -111,6 +111,16 @@ def test_grouped_down_projection_scattered_components(tokens, block, clusters, d
         assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
 
 
+def test_grouped_down_projection_token_mask_too_large_for_shared_memory():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-large-mask", 1400, 128, 8192, 16, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 432, 0.5).sum())
+    tm = wl.token_block_masks_clustered(432, "tmc", 1400, nab, 5, 0.05, 3, 2)
+    assert _run(cfg, 432, 1400, 0.5, None, 2, token_mask=tm) == 0
+    assert 0 < _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
 def test_grouped_down_projection_opt13b_at_90_percent():
     """The graded FFN shape with the batch dealt to four groups of requests: full comparison against the oracle."""
     if not torch.cuda.is_available():

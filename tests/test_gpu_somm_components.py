@@ -132,6 +132,18 @@ def test_grouped_launch_scattered_components(tokens, block, clusters, dead):
         assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]                       # than the union needs
 
 
+def test_grouped_launch_token_mask_too_large_for_shared_memory():
+    """1400 tokens x 256 active blocks: the planning kernel's bit matrix and labels (52 KB) work in global memory."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-large-mask", 1400, 128, 8192, 16, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    tm = _clustered(cfg, 431, 1400, 0.5, 5, 0.05, 3, 2)
+    bad, L = _run(cfg, 431, 1400, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L >= 5
+    assert _LAST["ring_macs"] == 2 * 2 * _LAST["d"] * _LAST["dot_products"]
+    assert 0 < _LAST["tile_macs"] < _LAST["dense_tile_macs"]
+
+
 def test_grouped_launch_gated_two_matrices():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
