@@ -207,8 +207,8 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * on the blocks (its other words are ignored).  Communication is Theorem 1's
  * minimum.  On the tensor-core path with more than 32 tokens the products of all
  * components are ONE launch over the component-sorted operands that computes
- * only the 128 x 64 output tiles which meet a component ("one multiplication per
- * subgraph" at tile granularity; comet_stats.ring_macs is then Theorem 1's count,
+ * only the 128 x 64 output tiles which meet a component (a separate product for
+ * every component, at tile granularity; comet_stats.ring_macs is then Theorem 1's count,
  * tensor_tile_macs what the tiles cover); otherwise one product over
  * [tokens, g*n], masked afterwards.  The shares are the same bits either way.
  *
