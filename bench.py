@@ -77,12 +77,16 @@ def ffn_bytes(cfg, T, n):
 
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
+    """`nvidia-smi` polled every 20 ms by a child process for the whole run; every sample is stamped on arrival and
+    a timed region is summarised from the samples that fell inside it.  The child is started long before the first
+    timed region (its start-up takes longer than a region lasts) and adds no work to the device."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.lines, self.proc = index, [], None
+        self.index, self.samples, self.proc = index, [], None
 
     def start(self):
         try:
@@ -93,26 +97,28 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def warm(self, step, limit_s: float = 3.0):
-        """Keep the device under the timed load (untimed calls of `step`) until the first sample has
-        arrived, so that a timed region shorter than the tool's start-up still has samples inside it."""
-        t0, s = time.perf_counter(), 0
-        while self.proc is not None and not self.lines and time.perf_counter() - t0 < limit_s:
-            step(s)
-            s += 1
-
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.samples.append((time.perf_counter(), line.strip()))
 
-    def stop(self) -> dict:
+    def wait_ready(self, limit_s: float = 5.0):
+        """Wait (device idle) until the first sample has arrived."""
+        t0 = time.perf_counter()
+        while self.proc is not None and not self.samples and time.perf_counter() - t0 < limit_s:
+            time.sleep(0.01)
+
+    def region(self, t0: float, t1: float) -> dict:
+        """Summary of the samples taken between the host times t0 and t1 (a sample shows up some milliseconds after
+        it was taken, so arrivals up to 30 ms after t1 count, and a region shorter than the polling period takes
+        the first sample after it began)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
+        time.sleep(0.05)
+        inside = [ln for t, ln in list(self.samples) if t0 <= t <= t1 + 0.03]
+        if not inside:
+            inside = [ln for t, ln in list(self.samples) if t >= t0][:1]
         sm, mx, reasons = [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        for line in inside:
             f = [x.strip() for x in line.split(",")]
             if len(f) < 8:
                 continue
@@ -121,11 +127,15 @@ class ClockSampler:
                 mx.append(float(f[1]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[4:8]):
+            for name, val in zip(self.NAMES, f[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
 
 
 # --------------------------------------------------------------------------- inputs
@@ -255,7 +265,9 @@ def run_shuffle(args, cfg):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        sampler.wait_ready()
     evs = []
+    host0 = time.perf_counter()
     for s in range(args.steps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -263,7 +275,8 @@ def run_shuffle(args, cfg):
         e1.record(stream)
         evs.append((e0, e1))
     torch.cuda.synchronize(dev)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.region(host0, time.perf_counter()) if rank == 0 else None
+    sampler.stop()
     total_ms = float(sum(a.elapsed_time(b) for a, b in evs))
     (total_ms,) = ranks.max_over_ranks([total_ms], dev)
     if rank != 0:
@@ -336,6 +349,9 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     T, d, g = cfg.tokens, cfg.d_model, cfg.groups
+    sampler = ClockSampler(local)        # polls for the whole run; the timed regions pick their samples by time
+    if rank == 0:
+        sampler.start()
     seed = ranks.rank_seed(1000, rank)   # every rank runs its own independent FFN problems (weak scaling, no collective)
     path = {"auto": cb.PATH_AUTO, "simt": cb.PATH_SIMT, "limb": cb.PATH_LIMB}[args.path]
     stream = torch.cuda.Stream(device=dev)
@@ -448,16 +464,14 @@ def main():
         device_step(s, False)
     barrier()
     launches0 = ctx.stats().kernel_launches
-    sampler = ClockSampler(local)
     if rank == 0:
-        sampler.start()
-        sampler.warm(lambda s: device_step(s, False))
+        sampler.wait_ready()
     barrier()
     wall0 = time.perf_counter()
     events = [device_step(args.warmup + s, True) for s in range(args.steps)]
     barrier()
     wall = time.perf_counter() - wall0
-    clocks_single = sampler.stop() if rank == 0 else None
+    clocks_single = sampler.region(wall0, wall0 + wall) if rank == 0 else None
     launches = ctx.stats().kernel_launches - launches0
     step_ms = [e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) + e[4].elapsed_time(e[5]) for e in events]
     total_ms = float(sum(step_ms))
@@ -540,11 +554,7 @@ def main():
             piped_step(s)
         barrier()
         launched0 = sum(cx.stats().kernel_launches for cx, _ in pctx)
-        sampler2 = ClockSampler(local)
-        if rank == 0:
-            sampler2.start()
-            sampler2.warm(piped_step)
-        barrier()
+        host0 = time.perf_counter()
         p0, p1 = ev(), ev()
         p0.record(tstream)
         for s in range(args.steps):
@@ -555,7 +565,7 @@ def main():
             tstream.wait_event(done)
         p1.record(tstream)
         barrier()
-        clocks_piped = sampler2.stop() if rank == 0 else None
+        clocks_piped = sampler.region(host0, time.perf_counter()) if rank == 0 else None
         (piped_ms,) = ranks.max_over_ranks([p0.elapsed_time(p1)], dev)
         piped = {"in_flight": C, "ms_per_step": piped_ms / args.steps,
                  "launches": int(sum(cx.stats().kernel_launches for cx, _ in pctx) - launched0),
@@ -608,6 +618,7 @@ def main():
     pairs = [e2e_step(3 + s) for s in range(args.steps)]
     barrier()
     e2e_ms = float(sum(a.elapsed_time(b) for a, b in pairs))
+    sampler.stop()
     h2d = sum(t.numel() * 8 for p in (0, 1) for t in sets[0]["pinned"][p].values()) + sets[0]["mask_host"].numel()
     d2h = 2 * T * d * 8 + 4
 
