@@ -111,6 +111,16 @@ def test_grouped_down_projection_scattered_components(tokens, block, clusters, d
         assert _LAST["tile_macs"] < _LAST["dense_tile_macs"]
 
 
+def test_down_projection_token_mask_without_any_entry():
+    """No non-zero in the hidden state at all: nothing is opened and Y_i = C'_i."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("rowsets-empty", 140, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 89, 0.5).sum())
+    for path in (1, 2):
+        assert _run(cfg, 89, 140, 0.5, None, path, token_mask=np.zeros((140, nab), np.uint8)) == 0
+
+
 def test_grouped_down_projection_token_mask_too_large_for_shared_memory():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")

@@ -144,6 +144,39 @@ def test_grouped_launch_token_mask_too_large_for_shared_memory():
     assert 0 < _LAST["tile_macs"] < _LAST["dense_tile_macs"]
 
 
+def test_token_mask_without_any_entry_and_with_a_single_one():
+    """Degenerate distributions on the tensor-core path with more than 32 tokens: no entry at all (nothing is opened,
+    every result share is zero) and a single (token, block) entry."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-degenerate", 140, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 88, 0.5).sum())
+    tm = np.zeros((140, nab), np.uint8)
+    bad, L = _run(cfg, 88, 140, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L == 0 and _LAST["ring_macs"] == 0
+    tm[137, nab - 1] = 1
+    bad, L = _run(cfg, 88, 140, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L == 1 and _LAST["ring_macs"] == 2 * 2 * 128 * 32
+    assert _LAST["tile_macs"] == 2 * 2 * 128 * 64 * 128            # one output tile per party and operand pair
+
+
+@pytest.mark.parametrize("live", [127, 128, 129])
+def test_grouped_launch_row_tile_boundaries(live):
+    """Exactly 127 / 128 / 129 tokens lie in a component (of 200): the sorted rows fill one tile, or one and one row."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    cfg = wl.FFNConfig("comp-boundary", 200, 128, 1024, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    nab = int(wl.block_mask(cfg, 90 + live, 0.5).sum())
+    tm = wl.token_block_masks_clustered(90 + live, "tmc", 200, nab, 3, 0.4)
+    order = np.argsort(wl.random_u64(90 + live, "kill", 200), kind="stable")
+    tm[order[:200 - live], :] = 0
+    tm[:, tm.sum(axis=0) == 0] = 0
+    rows_alive = int((tm.sum(axis=1) > 0).sum())
+    assert rows_alive == live
+    bad, L = _run(cfg, 90 + live, 200, 0.5, 2, token_mask=tm)
+    assert bad == 0 and L >= 1
+
+
 def test_grouped_launch_gated_two_matrices():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
