@@ -135,8 +135,9 @@ typedef struct {
     int32_t n_components;    /* connected components under the current token mask (0 without one) */
     int32_t reserved;
     int64_t tensor_tile_macs; /* 64-bit multiply-adds the tensor-core kernel of the last ffn call covered, counted
-                                 in whole 128 x 64 output tiles, both parties (0 on the CUDA-core path): under a
-                                 token mask with several components only the tiles that meet a component */
+                                 in whole output tiles (128 x 64, or 32 tokens x 128 for at most 32 tokens) and
+                                 32-deep steps, both parties (0 on the CUDA-core path): under a token mask with
+                                 several components only the tiles and steps that meet a component */
 } comet_stats_t;
 
 /* Create a context: validates the configuration, selects the device, and

@@ -328,7 +328,7 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
         }
     }
     const long long total_units = grouped ? 2ll * a.group_units : 2ll * mt * nt * 2 * kb;
-    c->stats.tensor_tile_macs = total_units * lb::KC * lb::BM * lb::BN;
+    c->stats.tensor_tile_macs = total_units * lb::KC * (few ? lf::BW * lf::BT : lb::BM * lb::BN);
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
         PhaseTimer timer(c, COMET_PHASE_COMBINE, 1);
