@@ -267,3 +267,72 @@ def test_grouped_chain_up_then_down_with_three_stacked_matrices():
         bad += int((ctx.get(p, cb.F_DN, (d, n)).T != refd["F"][p]).sum())
     ctx.close()
     assert bad == 0
+
+
+def test_one_context_through_grouped_cleared_and_regrouped_masks():
+    """State carried by a context across calls: a clustered token mask (grouped launches, the down-projection's
+    weight side opened early in component order), the mask cleared (products over the union again), a token mask
+    with one component, then a new block mask with another clustered token mask.  Every product is compared with
+    the oracle, so nothing of an earlier plan may leak into a later call."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    cfg = wl.FFNConfig("comp-states", 160, 128, 1024, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    T, d, bs = 160, cfg.d_model, cfg.block
+    seed = 700
+    W = wl.model_shares(cfg, seed, plain=False)
+    Wup = (hz.oracle_up_operand(cfg, W, 1), hz.oracle_up_operand(cfg, W, 2))
+    ctx = hz.make_context(cfg, T, 2)
+    hz.load_weights(ctx, cfg, W)
+    bad = 0
+
+    def both(step, mask, tm):
+        """One up- and one down-projection under (mask, tm); tm None = no token mask."""
+        nonlocal bad
+        I = oracle.index_set(mask, bs, 1)
+        n, nab = I.size, int(mask.sum())
+        _, X0, X1 = wl.activation_shares(cfg, seed, step=step, tokens=T)
+        _, H0, H1 = wl.hidden_shares(cfg, seed, n, step=step, tokens=T)
+        assert ctx.set_mask(mask) == n
+        if tm is None:
+            tri = wl.dealer_triple(seed, f"up/{step}", T, d, n, valid=False)
+            trd = wl.dealer_triple(seed, f"dn/{step}", T, n, d, valid=False)
+            ref = oracle.somm((X0, X1), Wup, I, tri["A"][1:], tri["B"][1:], tri["C"][1:])
+            refd = oracle.simm((H0, H1), W["W2"][1:], I, trd["A"][1:], trd["B"][1:], trd["C"][1:])
+        else:
+            S = np.repeat(tm, bs, axis=1)
+            tri = wl.dealer_triple_components(seed, f"up/{step}", S, d)
+            trd = wl.dealer_triple_rowsets(seed, f"dn/{step}", S, d)
+            ref = oracle.somm_components((X0, X1), Wup, I, S, tri["A"][1:], tri["B"][1:], tri["C"][1:])
+            refd = oracle.simm_rowsets((H0, H1), W["W2"][1:], I, S, trd["A"][1:], trd["B"][1:], trd["C"][1:])
+            ctx.set_token_mask(tm)
+        for p, Xs in ((0, X0), (1, X1)):
+            ctx.load_shares(p, cb.X, cb.to_device(Xs))
+        hz.load_triple_up(ctx, tri)
+        hz.load_triple_down(ctx, trd)
+        ctx.ffn_up(T)
+        for p, Hs in ((0, H0), (1, H1)):
+            ctx.load_shares(p, cb.H, cb.to_device(Hs))
+        ctx.ffn_down(T)
+        for p in (0, 1):
+            bad += int((ctx.get(p, cb.Z_UP, (T, n)) != ref["Z"][p]).sum())
+            bad += int((ctx.get(p, cb.F_UP, (n, d)).T != ref["F"][p]).sum())
+            bad += int((ctx.get(p, cb.Y, (T, d)) != refd["Z"][p]).sum())
+            bad += int((ctx.get(p, cb.F_DN, (d, n)).T != refd["F"][p]).sum())
+            bad += int((ctx.get(p, cb.E_DN, (T, n)) != refd["E"][p]).sum())
+        return nab
+
+    m1 = wl.block_mask(cfg, seed, 0.5, 0)
+    nab = int(m1.sum())
+    both(0, m1, wl.token_block_masks_clustered(seed, "a", T, nab, 4, 0.5, 2, 1))     # grouped
+    assert ctx.stats().n_components >= 4
+    assert ctx.set_token_mask(None) == 0
+    both(1, m1, None)                                                                 # union, same block mask
+    both(2, m1, wl.token_block_masks(seed, "b", T, nab, 0.5))                         # one component: not grouped
+    m2 = wl.block_mask(cfg, seed, 0.75, 1)
+    both(3, m2, wl.token_block_masks_clustered(seed, "c", T, int(m2.sum()), 3, 0.6))  # new block mask, grouped again
+    both(4, m2, None)                                                                 # set_mask alone drops the token mask
+    ctx.close()
+    assert bad == 0
