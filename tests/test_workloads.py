@@ -65,3 +65,23 @@ def test_dealer_triple_is_a_product():
     assert np.array_equal(C, want)
     for key in "ABC":
         assert np.array_equal(t[key][1] + t[key][2], t[key][0])
+
+
+def test_clustered_token_masks_fall_into_the_requested_groups():
+    tm = wl.token_block_masks_clustered(3, "x", 200, 40, 5, 0.3, dead_tokens=3, dead_blocks=2)
+    assert tm.shape == (200, 40) and tm.dtype == np.uint8
+    rl, cl = wl.bipartite_components(tm)
+    assert len(set(rl[rl >= 0].tolist())) >= 5                      # at least one component per group
+    assert int((cl < 0).sum()) >= 2 and int((rl < 0).sum()) >= 3    # the blocks and tokens without any entry
+    # no edge joins two groups: every component's tokens use only that component's blocks
+    for r in range(200):
+        for b in np.nonzero(tm[r])[0]:
+            assert rl[r] == cl[b]
+    # same seed, same mask; another stream, another mask
+    assert np.array_equal(tm, wl.token_block_masks_clustered(3, "x", 200, 40, 5, 0.3, dead_tokens=3, dead_blocks=2))
+    assert not np.array_equal(tm, wl.token_block_masks_clustered(3, "y", 200, 40, 5, 0.3, dead_tokens=3, dead_blocks=2))
+
+
+def test_plain_token_masks_leave_no_token_and_no_block_empty():
+    tm = wl.token_block_masks(4, "t", 64, 26, 0.05)
+    assert tm.sum(axis=0).min() >= 1 and tm.sum(axis=1).min() >= 1
