@@ -8,6 +8,7 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+import oracle  # noqa: E402
 from paper_2505_07239_b200 import workloads as wl  # noqa: E402
 
 
@@ -270,3 +271,92 @@ def test_bound_inputs_give_the_same_bits_as_copied_ones(hz):
         ctx.close()
     for a, b in zip(*outs):
         assert np.array_equal(a, b)
+
+
+def test_four_problems_in_flight_at_full_size(hz):
+    """The benchmark's throughput configuration: four contexts on four streams, OPT-1.3B shape at 90 % sparsity,
+    inputs bound in place, two steps per context issued round-robin with nothing but each context's own mask
+    report between them.  Every context's last step is compared with the oracle: messages in full, products and
+    truncated products at sampled positions."""
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["opt1.3b"]
+    T, d, f, seed, C = cfg.tokens, cfg.d_model, cfg.frac_bits, 31, 4
+    W = wl.model_shares(cfg, seed, plain=False)
+    Wdev = [[cb.to_device(wl.lib_layout(W[k][1 + p])) for k in ("W1", "W2")] for p in (0, 1)]
+    n_cap = cfg.n_active_blocks(0.9) * cfg.block
+    ctxs, inputs = [], []
+    for k in range(C):
+        sk = torch.cuda.Stream()
+        cx = cb.Comet(T, d, cfg.d_ff, cfg.block, f, 0, 0, n_cap, cb.PATH_AUTO, sk)
+        for p in (0, 1):
+            cx.bind_shares(p, cb.W1, Wdev[p][0])
+            cx.bind_shares(p, cb.W2, Wdev[p][1])
+        ctxs.append((cx, sk))
+        steps = []
+        for j in range(2):
+            step = 10 * k + j
+            mask = wl.block_mask(cfg, seed, 0.9, step)
+            n = int(mask.sum()) * cfg.block
+            _, X0, X1 = wl.activation_shares(cfg, seed, step=step, tokens=T)
+            _, H0, H1 = wl.hidden_shares(cfg, seed, n, step=step, tokens=T)
+            tri = wl.dealer_triple(seed, f"fl/up/{step}", T, d, n, valid=False)
+            trd = wl.dealer_triple(seed, f"fl/dn/{step}", T, n, d, valid=False)
+            host = {"mask": mask, "n": n, "X": (X0, X1), "H": (H0, H1), "up": tri, "dn": trd}
+            dev = [{cb.X: cb.to_device((X0, X1)[p]), cb.H: cb.to_device((H0, H1)[p]),
+                    cb.A_UP: cb.to_device(tri["A"][1 + p]), cb.B_UP: cb.to_device(wl.lib_layout(tri["B"][1 + p])),
+                    cb.C_UP: cb.to_device(tri["C"][1 + p]), cb.A_DN: cb.to_device(trd["A"][1 + p]),
+                    cb.B_DN: cb.to_device(wl.lib_layout(trd["B"][1 + p])), cb.C_DN: cb.to_device(trd["C"][1 + p])}
+                   for p in (0, 1)]
+            steps.append((host, dev, torch.from_numpy(mask).cuda()))
+        inputs.append(steps)
+    torch.cuda.synchronize()
+    zup = {}
+    for j in range(2):
+        for k, (cx, sk) in enumerate(ctxs):
+            host, dev, mask_dev = inputs[k][j]
+            with torch.cuda.stream(sk):
+                assert cx.set_mask(mask_dev) == host["n"]
+                for p in (0, 1):
+                    for tid in (cb.X, cb.A_UP, cb.B_UP, cb.C_UP, cb.A_DN, cb.B_DN, cb.C_DN):
+                        cx.bind_shares(p, tid, dev[p][tid])
+                cx.ffn_up(T)
+                if j == 1:                              # keep the untruncated product of the step that is checked
+                    zup[k] = [torch.empty(T * host["n"], dtype=torch.int64, device="cuda") for _ in (0, 1)]
+                    for p in (0, 1):
+                        cx.get_into(p, cb.Z_UP, zup[k][p])
+                cx.truncate(cb.Z_UP)
+                for p in (0, 1):
+                    cx.bind_shares(p, cb.H, dev[p][cb.H])
+                cx.ffn_down(T)
+                cx.truncate(cb.Y)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(5)
+    bad = 0
+    for k, (cx, sk) in enumerate(ctxs):
+        host, _, _ = inputs[k][1]
+        n, tri, trd, mask = host["n"], host["up"], host["dn"], host["mask"]
+        I = oracle.index_set(mask, cfg.block, 1)
+        E = [oracle.mask_operand(host["X"][p], tri["A"][1 + p]) for p in (0, 1)]
+        F = [oracle.mask_operand(oracle.index_cols(W["W1"][1 + p], I), tri["B"][1 + p]) for p in (0, 1)]
+        Eo, Fo = oracle.reconstruct(*E), oracle.reconstruct(*F)
+        rows, cols = hz.sample_positions(rng, T, n, 256)
+        for p in (0, 1):
+            bad += int((cx.get(p, cb.E_UP, (T, d)) != E[p]).sum())
+            bad += int((cx.get(p, cb.F_UP, (n, d)).T != F[p]).sum())
+            want = oracle.beaver_combine_at(p, Eo, Fo, tri["A"][1 + p], tri["B"][1 + p], tri["C"][1 + p], rows, cols)
+            got = zup[k][p].cpu().numpy().view(np.uint64).reshape(T, n)
+            bad += int((got[rows, cols] != want).sum())
+            bad += int((cx.get(p, cb.Z_UP, (T, n))[rows, cols] != oracle.truncate(p, want, f)).sum())
+        E = [oracle.mask_operand(host["H"][p], trd["A"][1 + p]) for p in (0, 1)]
+        F = [oracle.mask_operand(oracle.index_rows(W["W2"][1 + p], I), trd["B"][1 + p]) for p in (0, 1)]
+        Eo, Fo = oracle.reconstruct(*E), oracle.reconstruct(*F)
+        rows, cols = hz.sample_positions(rng, T, d, 256)
+        for p in (0, 1):
+            bad += int((cx.get(p, cb.E_DN, (T, n)) != E[p]).sum())
+            bad += int((cx.get(p, cb.F_DN, (d, n)).T != F[p]).sum())
+            want = oracle.beaver_combine_at(p, Eo, Fo, trd["A"][1 + p], trd["B"][1 + p], trd["C"][1 + p], rows, cols)
+            bad += int((cx.get(p, cb.Y, (T, d))[rows, cols] != oracle.truncate(p, want, f)).sum())
+    for cx, _ in ctxs:
+        cx.close()
+    assert bad == 0
