@@ -423,9 +423,10 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 //
 // 1. The first step of Protocol 2: the connected components of the bipartite graph (token rows) x (active
 //    blocks) with the non-zero bytes as edges.  The paper uses depth-first search; here S becomes a bit matrix
-//    and minimum labels are propagated: every row takes the minimum over its blocks and pushes it to them, all
-//    rows in parallel, until nothing changes (at most T + nab + 1 sweeps).  Every node of a component ends up with
-//    the component's smallest token index as its label; nodes without an edge get -1.
+//    and minimum labels are propagated without atomics: every block takes the minimum over its rows (one warp per
+//    block), then every row the minimum over its blocks (one thread per row), until nothing changes (at most
+//    T + nab + 1 sweeps).  Every node of a component ends up with the component's smallest token index as its
+//    label; nodes without an edge get -1.
 //
 // 2. (plan != 0) Protocols 2 and 3 ask for one multiplication per component / per non-zero column entry, over the
 //    rows and columns that take part only (the multiplication counts of Theorems 1 and 2).  On the tensor cores
