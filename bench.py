@@ -195,7 +195,22 @@ def time_oracle(cfg, seed, sparsity, budget_s=15.0):
     if T > probe_T:
         dt, macs = run(T)
     return {"value": macs / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 3),
-            "sample": f"first {T} of {cfg.tokens} token rows of the same workload, whole path, both parties"}
+            "sample": f"first {T} of {cfg.tokens} token rows of the same workload, whole path, both parties",
+            "host": host_cpu()}
+
+
+def host_cpu() -> dict:
+    """The machine the oracle was timed on: model name and the number of cores it offers (the oracle uses one)."""
+    model = None
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for ln in fh:
+                if ln.lower().startswith("model name"):
+                    model = ln.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"model": model, "logical_cores": os.cpu_count()}
 
 
 def run_reference(args, cfg, sparsity):
@@ -217,7 +232,8 @@ def run_reference(args, cfg, sparsity):
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64", "data": "synthetic",
         "config": {"workload": workload_name(cfg, sparsity), "note": "CPU oracle, one thread, bounded sample per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": vals[-1]["sample"]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": vals[-1]["sample"],
+                         "host": host_cpu()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
