@@ -206,11 +206,12 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * per-component triples are passed stacked: row r of COMET_A_UP is the mask row
  * of r's component, row c of COMET_B_UP that of c's, COMET_C_UP holds a^t b^t
  * on the blocks (its other words are ignored).  Communication is Theorem 1's
- * minimum.  On the tensor-core path with more than 32 tokens the products of all
- * components are ONE launch over the component-sorted operands that computes
- * only the 128 x 64 output tiles which meet a component (a separate product for
- * every component, at tile granularity; comet_stats.ring_macs is then Theorem 1's count,
- * tensor_tile_macs what the tiles cover); otherwise one product over
+ * minimum.  On the tensor-core path with 33 to 32768 tokens, when there are
+ * several components or rows / blocks in none, the products of all components
+ * are ONE launch over the component-sorted operands that computes only the
+ * 128 x 64 output tiles which meet a component (a separate product for every
+ * component, at tile granularity; comet_stats.ring_macs is then Theorem 1's
+ * count, tensor_tile_macs what the tiles cover); otherwise one product over
  * [tokens, g*n], masked afterwards.  The shares are the same bits either way.
  *
  * Down-projection, Protocol 3 (its row sets R_j): the sparsity distribution of the hidden
@@ -227,14 +228,14 @@ int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
  * message; likewise the rows of F'_i that belong to an active block no token
  * uses) and ignores whatever COMET_H and COMET_A_DN hold off the support;
  * the dealer's C' is sum_j a_j b_j^T scattered to the rows R_j, i.e.
- * (mask * A') B'.  Communication is Theorem 2's minimum.  On the tensor-core
- * path with more than 32 tokens and several components, rows and contraction
- * index are taken in component order and every tile of 128 rows runs over the
- * blocks of its own components only; otherwise the product runs over
- * [tokens, n].  comet_stats.ring_macs is Theorem 2's count either way,
- * tensor_tile_macs what the tiles cover.  *masked_out (may be NULL) receives the number of
- * non-zero entries (neurons, summed over tokens); one 8-byte device-to-host
- * report and a stream synchronise.  Errors: STATE (no block mask yet), SHAPE
+ * (mask * A') B'.  Communication is Theorem 2's minimum.  Under the same
+ * conditions as for the up-projection, rows and contraction index are taken in
+ * component order and every tile of 128 rows runs over the blocks of its own
+ * components only; otherwise the product runs over [tokens, n].
+ * comet_stats.ring_macs is Theorem 2's count either way, tensor_tile_macs what
+ * the tiles cover.  *masked_out (may be NULL) receives the number of non-zero
+ * entries (neurons, summed over tokens); one kernel, one report of seven words
+ * through mapped host memory and a stream synchronise.  Errors: STATE (no block mask yet), SHAPE
  * (tokens out of range, n_active_blocks not the current count), INVALID_ARG. */
 int comet_set_token_mask(comet_ctx* ctx, const uint8_t* token_mask, int location, int32_t tokens,
                          int32_t n_active_blocks, int64_t* masked_out);
