@@ -45,6 +45,7 @@ struct comet_ctx {
     bool side_pending;                // ev_join not yet waited for on the main stream
     bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
     bool dn_right_few;                // ... and were laid out for the few-token kernel (128-row tiles)
+    bool f_as_planes[2];              // the messages F_i of the last up / down product exist as planes only
     uint8_t* d_mask;
     uint8_t* d_tmask;             // per-token mask over the active blocks, [cap_T, d_ff / block] capacity
     bool tmask_set;
@@ -218,7 +219,9 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
         a.B[p] = c->buf[p][pr.idB];
         a.F[p] = c->buf[p][pr.idF];
         a.Bpl[p] = planes[p][0];
+        a.Fpl[p] = planes[p][1];
     }
+    a.emit_f = limb_few(pr) ? 1 : 0;       // few-token products read the messages as planes (no plane of their sum)
     a.left_pairs = left ? (long long)pr.M * pr.K / 2 : 0;
     a.left_blocks = left ? ew_grid(c, a.left_pairs, 256) : 0;
     a.ids = c->d_ids;
@@ -238,7 +241,9 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.kmap = (pr.down && c->grouped) ? c->d_kmap : nullptr;
     const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
-    comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, 0, stream>>>(a);
+    if (right_tiles) c->f_as_planes[pr.down ? 1 : 0] = a.emit_f != 0;
+    const size_t smem = right_tiles ? (a.emit_f ? 2 : 1) * sizeof(comet::LimbTile) : 0;
+    comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, smem, stream>>>(a);
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
@@ -278,7 +283,8 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
     a.tmask_ld = c->n_active_blocks;
     a.bs = c->cfg.block;
     a.left_tiles = left ? kb * ceil_div(a.M, lb::PREP_ROWS) : 0;
-    a.right_tiles = right ? kb * ceil_div(a.N, lb::PREP_ROWS) : 0;
+    // few-token products take the planes of the two messages as limb_open_kernel wrote them
+    a.right_tiles = (right && !limb_few(pr)) ? kb * ceil_div(a.N, lb::PREP_ROWS) : 0;
     a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
     a.copy_blocks = copy ? ew_grid(c, a.copy_pairs, 256) : 0;
     const int blocks = a.left_tiles + a.right_tiles + a.copy_blocks;
@@ -327,7 +333,8 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
             a.group_units = c->group_units_up;
         }
     }
-    const long long total_units = grouped ? 2ll * a.group_units : 2ll * mt * nt * 2 * kb;
+    const long long total_units = grouped ? 2ll * a.group_units
+                                          : 2ll * mt * nt * (few ? comet::LIMB_FEW_PAIRS : 2) * kb;
     c->stats.tensor_tile_macs = total_units * lb::KC * (few ? lf::BW * lf::BT : lb::BM * lb::BN);
     const int grid = (int)(total_units < c->sm_count ? total_units : c->sm_count);
     {
@@ -961,6 +968,16 @@ int comet_get(comet_ctx* c, int party, int tensor_id, uint64_t* out, int locatio
                                     ? c->up_done : c->down_done))
         return COMET_ERR_STATE;
     if (capacity < words) return COMET_ERR_SHAPE;
+    if (words > 0 && (tensor_id == COMET_F_UP || tensor_id == COMET_F_DN) &&
+        c->f_as_planes[tensor_id == COMET_F_DN ? 1 : 0] && c->path == COMET_PATH_LIMB) {
+        // a few-token product wrote this message as limb planes only: rebuild the words
+        uint8_t* (*planes)[2] = tensor_id == COMET_F_DN ? c->planes_right_dn : c->planes_right_up;
+        comet::limb_planes_to_words_kernel<<<ew_grid(c, words, 256), 256, 0, c->stream>>>(
+            planes[party][1], c->buf[party][tensor_id], (int)rows, (int)cols, ceil_div((int)cols, comet::limb::KC),
+            comet::limb_few::BW);
+        c->stats.kernel_launches += 1;
+        COMET_CUDA(c, cudaGetLastError());
+    }
     if (words > 0)
         COMET_CUDA(c, cudaMemcpyAsync(out, c->buf[party][tensor_id], (size_t)words * sizeof(u64),
                                       copy_kind(location, false), c->stream));

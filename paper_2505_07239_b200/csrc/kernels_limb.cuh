@@ -105,7 +105,8 @@ __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows,
 //                 own B_i (it is in registers anyway, so it is not read a second time later).
 // gather: up   (down = 0): row c of the right operand is row neuron(c) of W (whole rows of `ldw` words);
 //         down (down = 1): contraction index c is column neuron(c) of W (strips of `bs` words in every row).
-// grid = (left_blocks + kblocks * ceil(rows / 64), party), 256 threads.
+// grid = (left_blocks + kblocks * ceil(rows / 64), party), 256 threads; dynamic shared memory: one LimbTile when
+// there are right tiles, two with emit_f.
 // ---------------------------------------------------------------------------
 struct LimbOpenArgs {
     const u64* X[2];
@@ -142,6 +143,11 @@ struct LimbOpenArgs {
     // With kmap (down only): contraction index k of the plane tiles is compact index kmap[k / bs] * bs + k % bs,
     // i.e. the planes run over the active blocks in component order while F_i keeps the compact order.
     const int32_t* kmap;
+    // Few-token products: the party's message F_i is written as blocked limb planes (same layout as Bpl) INSTEAD of
+    // as words: the product kernel reads both parties' messages in that form, so no plane of their sum has to be
+    // built and the words are never needed on the path (limb_planes_to_words_kernel rebuilds them when asked for).
+    uint8_t* Fpl[2];
+    int emit_f;
 };
 
 __global__ void __launch_bounds__(256)
@@ -171,7 +177,9 @@ limb_open_kernel(LimbOpenArgs a) {
         }
         return;
     }
-    __shared__ LimbTile sB;
+    extern __shared__ __align__(16) uint8_t open_smem[];
+    LimbTile& sB = *reinterpret_cast<LimbTile*>(open_smem);
+    LimbTile& sF = *reinterpret_cast<LimbTile*>(open_smem + sizeof(LimbTile));      // only with emit_f
     const int tile_id = blockIdx.x - a.left_blocks;
     const int kb = tile_id % a.kblocks;
     const int row0 = (tile_id / a.kblocks) * PREP_ROWS;
@@ -191,7 +199,7 @@ limb_open_kernel(LimbOpenArgs a) {
         for (int it = 0; it < PREP_ROWS / 16; ++it) {
             const int r = it * 16 + (tid >> 4);
             int row = row0 + r;
-            u64 b0 = 0, b1 = 0;
+            u64 b0 = 0, b1 = 0, f0 = 0, f1 = 0;
             if (row < a.rows && k < a.K) {
                 const u64* wsrc;
                 bool dead = false;
@@ -213,21 +221,44 @@ limb_open_kernel(LimbOpenArgs a) {
                 const size_t o = (size_t)row * a.K + ks;
                 const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2*>(wsrc));
                 const ulonglong2 b = __ldg(reinterpret_cast<const ulonglong2*>(Bi + o));
-                *reinterpret_cast<ulonglong2*>(Fi + o) = dead ? make_ulonglong2(0ull, 0ull)
-                                                              : make_ulonglong2(w.x - b.x, w.y - b.y);
+                f0 = dead ? 0ull : w.x - b.x;
+                f1 = dead ? 0ull : w.y - b.y;
+                if (!a.emit_f) *reinterpret_cast<ulonglong2*>(Fi + o) = make_ulonglong2(f0, f1);
                 b0 = b.x;
                 b1 = b.y;
             }
             sB[r][kk] = b0;
             sB[r][kk + 1] = b1;
+            if (a.emit_f) {
+                sF[r][kk] = f0;
+                sF[r][kk + 1] = f1;
+            }
         }
     }
     __syncthreads();
-    if (tid < 128) {
-        const int half = tid >> 6, r = tid & 63;
-        int rin;
-        uint8_t* blk = limb_block_ptr(party ? a.Bpl[1] : a.Bpl[0], a.right_tile_rows, row0 + r, a.kblocks, kb, &rin);
-        limb_emit_planes(sB, r, half, blk, a.right_tile_rows, rin);
+    const int which = tid >> 7;                       // 0: planes of B_i, 1: planes of F_i
+    if (which == 1 && !a.emit_f) return;
+    const int half = (tid >> 6) & 1, r = tid & 63;
+    int rin;
+    uint8_t* blk = limb_block_ptr(which ? (party ? a.Fpl[1] : a.Fpl[0]) : (party ? a.Bpl[1] : a.Bpl[0]),
+                                  a.right_tile_rows, row0 + r, a.kblocks, kb, &rin);
+    limb_emit_planes(which ? sF : sB, r, half, blk, a.right_tile_rows, rin);
+}
+
+// Blocked limb planes back to words: out[row, k] for a [rows, K] operand whose plane tiles have `tile_rows` rows.
+// Only used off the path, when a message that was written as planes is read back as words.
+__global__ void __launch_bounds__(256)
+limb_planes_to_words_kernel(const uint8_t* __restrict__ planes, u64* __restrict__ out, int rows, int K, int kblocks,
+                            int tile_rows) {
+    const long long total = (long long)rows * K, stride = (long long)gridDim.x * blockDim.x;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += stride) {
+        const int row = (int)(t / K), k = (int)(t - (long long)row * K);
+        const int tile = row / tile_rows, rin = row - tile * tile_rows, kb = k / limb::KC, kin = k - kb * limb::KC;
+        const uint8_t* blk = planes + ((size_t)tile * kblocks + kb) * (size_t)(limb::PLANES * tile_rows * limb::KC);
+        u64 v = 0;
+#pragma unroll
+        for (int p = 0; p < limb::PLANES; ++p) v |= (u64)blk[limb::block_offset(tile_rows, p, rin, kin)] << (8 * p);
+        out[t] = v;
     }
 }
 
@@ -1041,7 +1072,10 @@ combine_limb_grouped_kernel(LimbArgs a) {
 // left planes 0..7-q in one instruction of N = 32*(8-q) <= 256, 8 instructions per 32-deep step, and the eight
 // accumulators D_s (128 neurons x 32 tokens) take 256 TMEM columns.  A 128-row tile of the ordinary kernel would
 // spend three quarters of its tensor work on padding rows here.  Every weight plane is used by exactly one tile,
-// so the kernel streams them once; it is bound by that traffic, not by the tensor pipe.
+// so the kernel streams them once; it is bound by that traffic, not by the tensor pipe.  That leaves tensor time
+// to spare, which buys a pass over memory: the second product is taken as V_i*F_0 + V_i*F_1 over the planes of the
+// two messages as the parties wrote them, so no kernel has to read both messages back, add them and write planes
+// of the sum.  A tile thus runs over three operand pairs: (E, B_i), (V_i, F_0), (V_i, F_1).
 // Plane layouts: token side [k-block][8 planes x 32 rows x 32 B] (8 KiB blocks), weight side
 // [n-tile of 128][k-block][32 KiB].  The output tile Z^T (neurons x tokens) is transposed through shared memory
 // so that each bulk reduction adds 32 consecutive neurons of one token row.
@@ -1058,8 +1092,31 @@ constexpr int TMEM_COLS = PLANES * BT;            // 256
 constexpr size_t SMEM_BYTES = (size_t)STAGES * (W_BLOCK_BYTES + T_BLOCK_BYTES) + (size_t)EPI_WARPS * OUT_BYTES_PER_WARP + 128;
 }  // namespace limb_few
 
-// LimbArgs as for combine_limb_kernel with Epl/Vpl = token-side planes, Bpl/Fpl = weight-side planes, mt = 1,
+// LimbArgs as for combine_limb_kernel with Epl/Vpl = token-side planes, Bpl = weight-side planes of the party's
+// B_i, Fpl[0] / Fpl[1] = weight-side planes of the messages F_0 / F_1 (read by both parties), mt = 1,
 // nt = ceil(N / 128), M <= 32.
+constexpr int LIMB_FEW_PAIRS = 3;
+
+// One contiguous piece of a CTA's share: a run of k-blocks of one tile, kpos in [0, 3*kb).
+__device__ __forceinline__ LimbSegment limb_few_segment(const LimbArgs& a, long long u, long long u_end) {
+    const long long tile_units = (long long)LIMB_FEW_PAIRS * a.kb;
+    const long long tile = u / tile_units;
+    long long seg_end = (tile + 1) * tile_units;
+    if (seg_end > u_end) seg_end = u_end;
+    if (seg_end > u + limb::MAX_SEGMENT_UNITS) seg_end = u + limb::MAX_SEGMENT_UNITS;
+    const int per_party = a.mt * a.nt;
+    LimbSegment s;
+    s.party = (int)(tile / per_party);
+    const int t2 = (int)(tile - (long long)s.party * per_party);
+    s.tm = t2 / a.nt;
+    s.tn = t2 - s.tm * a.nt;
+    s.kpos = (int)(u - tile * tile_units);
+    s.count = (int)(seg_end - u);
+    s.kb = a.kb;
+    s.klo = 0;
+    return s;
+}
+
 __global__ void __launch_bounds__(limb_few::THREADS, 1)
 combine_limb_few_kernel(LimbArgs a) {
     using namespace limb_few;
@@ -1076,7 +1133,7 @@ combine_limb_few_kernel(LimbArgs a) {
     uint8_t* sOut = sT + (size_t)STAGES * T_BLOCK_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long total_units = 2ll * a.mt * a.nt * 2ll * a.kb;
+    const long long total_units = 2ll * a.mt * a.nt * LIMB_FEW_PAIRS * a.kb;
     const long long u_begin = total_units * blockIdx.x / gridDim.x;
     const long long u_end = total_units * (blockIdx.x + 1) / gridDim.x;
 
@@ -1109,15 +1166,17 @@ combine_limb_few_kernel(LimbArgs a) {
             const uint32_t full0 = ptx::smem_u32(&full_bar[0]), empty0 = ptx::smem_u32(&empty_bar[0]);
             const uint32_t sW0 = ptx::smem_u32(sW), sT0 = ptx::smem_u32(sT);
             for (long long u = u_begin; u < u_end && ok;) {
-                const LimbSegment sg = limb_segment(a, u, u_end);
+                const LimbSegment sg = limb_few_segment(a, u, u_end);
                 u += sg.count;
-                int kpos = sg.kpos;
-                bool second = kpos >= a.kb;
-                if (second) kpos -= a.kb;
-                const uint8_t* tok = (second ? (sg.party ? a.Vpl[1] : a.Vpl[0]) : (sg.party ? a.Epl[1] : a.Epl[0])) +
-                                     (size_t)kpos * T_BLOCK_BYTES;
-                const uint8_t* wgt = (second ? (sg.party ? a.Fpl[1] : a.Fpl[0]) : (sg.party ? a.Bpl[1] : a.Bpl[0])) +
-                                     ((size_t)sg.tn * a.kb + kpos) * W_BLOCK_BYTES;
+                int pair = sg.kpos / a.kb;                    // 0: (E, B_i), 1: (V_i, F_0), 2: (V_i, F_1)
+                int kpos = sg.kpos - pair * a.kb;
+                const uint8_t* tok_e = sg.party ? a.Epl[1] : a.Epl[0];
+                const uint8_t* tok_v = sg.party ? a.Vpl[1] : a.Vpl[0];
+                const size_t tile_off = (size_t)sg.tn * a.kb * W_BLOCK_BYTES;
+                const uint8_t* wgt_b = (sg.party ? a.Bpl[1] : a.Bpl[0]) + tile_off;
+                const uint8_t* tok = (pair == 0 ? tok_e : tok_v) + (size_t)kpos * T_BLOCK_BYTES;
+                const uint8_t* wgt = (pair == 0 ? wgt_b : (pair == 1 ? a.Fpl[0] : a.Fpl[1]) + tile_off) +
+                                     (size_t)kpos * W_BLOCK_BYTES;
                 for (int it = 0; it < sg.count; ++it) {
                     ok = limb_wait(empty0 + 8 * stage, phase ^ 1u, &abort_flag);
                     if (!ok) break;
@@ -1129,11 +1188,11 @@ combine_limb_few_kernel(LimbArgs a) {
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     tok += T_BLOCK_BYTES;
                     wgt += W_BLOCK_BYTES;
-                    if (++kpos == a.kb && !second) {
-                        second = true;
+                    if (++kpos == a.kb && pair < LIMB_FEW_PAIRS - 1) {
+                        ++pair;                               // on to V_i with the next message
                         kpos = 0;
-                        tok = (sg.party ? a.Vpl[1] : a.Vpl[0]);
-                        wgt = (sg.party ? a.Fpl[1] : a.Fpl[0]) + (size_t)sg.tn * a.kb * W_BLOCK_BYTES;
+                        tok = tok_v;
+                        wgt = (pair == 1 ? a.Fpl[0] : a.Fpl[1]) + tile_off;
                     }
                 }
             }
@@ -1159,7 +1218,7 @@ combine_limb_few_kernel(LimbArgs a) {
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (long long u = u_begin; u < u_end && ok;) {
-                const LimbSegment sg = limb_segment(a, u, u_end);
+                const LimbSegment sg = limb_few_segment(a, u, u_end);
                 u += sg.count;
                 ok = limb_wait(accum_empty, acc_phase ^ 1u, &abort_flag);
                 if (!ok) break;
@@ -1192,7 +1251,7 @@ combine_limb_few_kernel(LimbArgs a) {
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + thalf * 16;
         u64* stage_out = reinterpret_cast<u64*>(sOut + (size_t)warp * OUT_BYTES_PER_WARP);   // [16 tokens][32 neurons]
         for (long long u = u_begin; u < u_end && ok;) {
-            const LimbSegment sg = limb_segment(a, u, u_end);
+            const LimbSegment sg = limb_few_segment(a, u, u_end);
             u += sg.count;
             ok = limb_wait_warp(ptx::smem_u32(&accum_full_bar), acc_phase, &abort_flag);
             if (!ok) break;
