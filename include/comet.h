@@ -82,7 +82,9 @@ enum {
     COMET_B_DN = 9,   /* in : triple, masks W2[I, :]     [d_model, n]           */
     COMET_C_DN = 10,  /* in : triple                     [T, d_model]           */
     COMET_E_UP = 11,  /* out: message X_i - A_i          [T, d_model]           */
-    COMET_F_UP = 12,  /* out: message W_i[:, I] - B_i    [g*n, d_model]         */
+    COMET_F_UP = 12,  /* out: message W_i[:, I] - B_i    [g*n, d_model]  (after a product with at most 32
+                         tokens on the tensor-core path the messages F exist as limb planes; comet_get
+                         rebuilds the words)                                  */
     COMET_Z_UP = 13,  /* out: up-projection share        [T, g*n]               */
     COMET_E_DN = 14,  /* out: message H_i - A'_i         [T, n]                 */
     COMET_F_DN = 15,  /* out: message W2_i[I, :] - B'_i  [d_model, n]           */
