@@ -34,8 +34,9 @@ UNIT = "MAC64/s"
 L2_FLUSH_BYTES = 512 << 20
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the tensor-core combine kernel on the
-# default workload, from the ncu capture summarised in profiles/combine_limb__opt1.3b_s90.md (average of the
-# up- and the down-projection launch).  Valid only for the kernel source it was taken on: keyed by the SHA-256 of the kernel's part of kernels_limb.cuh.
+# default workload, from the committed ncu summary of that kernel (average of the up- and the down-projection
+# launch).  Valid only for the kernel source it was taken on: keyed by the SHA-256 of the kernel's part of
+# kernels_limb.cuh.
 COMBINE_LIMB_TRAFFIC = {
     "workload": ("opt1.3b", 0.9),
     "kernel_sha256": "2b11a0e9ac0c4abc86695f6910f87b457e3c798c2c32f2706a7a40a5865b64d4",
@@ -199,6 +200,11 @@ def time_oracle(cfg, seed, sparsity, budget_s=15.0):
             "host": host_cpu()}
 
 
+def bf16_sustained_derived(peaks: dict) -> float:
+    """Ring multiply-adds per second (in T) the sustained bf16 GEMM figure implies at the nominal int8 : bf16 ratio."""
+    return peaks.get("bf16_tflops_sustained", 1400.0) * 1e12 / 2 * 2 / 36 / 1e12
+
+
 def host_cpu() -> dict:
     """The machine the oracle was timed on: model name and the number of cores it offers (the oracle uses one)."""
     model = None
@@ -316,6 +322,57 @@ def run_shuffle(args, cfg):
                      "peak_source": "measured" if peaks else "fallback"}}))
 
 
+# --------------------------------------------------------------------------- measured peaks of the multiply pipes
+def measure_pipe_peaks(sampler, tensor_launches=24, alu_launches=12):
+    """The rate of the int8 tensor pipe (the instruction the limb kernel issues, operands resident in shared
+    memory) and of the 64-bit multiply-add loop on the integer ALUs, each as a run of back-to-back launches of
+    about 25 ms: `burst` is the best of the first three launches, `sustained` the median of the last third (the
+    part settles under its power limit within a few hundred milliseconds).  Rates in multiply-adds per second: 8-bit
+    ones for the tensor pipe (a ring multiply-add costs 36 of them), 64-bit ones for the ALUs."""
+    from paper_2505_07239_b200 import binding as cb
+
+    out = {}
+    for name, pipe, launches, work in (("tensor_i8", cb.PIPE_TENSOR_I8, tensor_launches, 10000),
+                                       ("alu_u64", cb.PIPE_ALU_U64, alu_launches, 40000)):
+        cb.pipe_probe(pipe, 2, max(1, work // 50))                         # load the module, touch the clocks
+        t0 = time.perf_counter()
+        ms, macs = cb.pipe_probe(pipe, launches, work)
+        t1 = time.perf_counter()
+        rates = [macs / (m * 1e-3) for m in ms]
+        tail = rates[-max(1, launches // 3):]
+        out[name] = {"burst": max(rates[:3]), "sustained": float(np.median(tail)), "unit": "MAC/s",
+                     "launches": launches, "ms_per_launch": [round(m, 3) for m in ms],
+                     "clocks": sampler.region(t0, t1) if sampler is not None else None}
+        time.sleep(0.5)                                                    # let the part cool before the next probe
+    t = out["tensor_i8"]
+    t["ring_mac_burst"], t["ring_mac_sustained"] = t["burst"] / 36, t["sustained"] / 36
+    if t["clocks"] and t["clocks"].get("sm_mhz"):
+        # 8-bit multiply-adds per SM and clock at the sampled median clock (the pipe's nominal figure is 8192)
+        t["macs_per_sm_clk_at_sampled_clock"] = t["sustained"] / 148 / (t["clocks"]["sm_mhz"] * 1e6)
+    return out
+
+
+def run_peak(args):
+    """`--op peak`: only the measured pipe peaks, one JSON line."""
+    import torch
+
+    rank, world, local = ranks.rank_world_local()
+    if rank != 0:
+        return
+    torch.cuda.set_device(local)
+    sampler = ClockSampler(local)
+    sampler.start()
+    sampler.wait_ready()
+    peaks = measure_pipe_peaks(sampler, tensor_launches=max(24, args.steps // 4), alu_launches=12)
+    sampler.stop()
+    print(json.dumps({"metric": "measured peak of the multiply pipes", "value": peaks["tensor_i8"]["ring_mac_burst"],
+                      "unit": UNIT, "n_gpus": 1, "steps": peaks["tensor_i8"]["launches"], "warmup": 2,
+                      "higher_is_better": True, "dtype": "u8 x u8 -> s32 (tensor), u64 (ALU)", "data": "synthetic",
+                      "config": {"workload": "tcgen05.mma kind::i8 M128 N256 K32 loop, 148 CTAs, operands in shared "
+                                             "memory; 64-bit multiply-add chains, 2 x 1024 threads per SM"},
+                      "peaks": peaks}))
+
+
 # --------------------------------------------------------------------------- GPU leg
 def main():
     ap = argparse.ArgumentParser()
@@ -327,6 +384,9 @@ def main():
     ap.add_argument("--sparsity", type=float, default=None)
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "limb"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-peak-probe", action="store_true",
+                    help="skip the measurement of the multiply pipes' peaks (the roofline then falls back to figures "
+                         "derived from the bf16 GEMM peak / the unit counts)")
     ap.add_argument("--token-masks", type=float, default=0.0, metavar="P",
                     help="give every token its own Bernoulli(P) mask over the active blocks (Protocols 2 and 3 in "
                          "general: connected components, per-column row sets); set_token_mask is timed with set_mask")
@@ -338,8 +398,12 @@ def main():
                     help="independent FFN problems in flight (contexts, one stream each, inputs bound in place); the "
                          "headline throughput is measured that way when C > 1, the one-problem-at-a-time figures are "
                          "reported beside it; 1 = only the latter")
-    ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle"],
-                    help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage")
+    ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle", "peak"],
+                    help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage; "
+                         "peak: the measured rates of the int8 tensor pipe and of the 64-bit ALU loop alone")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="the timed region of K steps is repeated until the device has been under load for this "
+                         "long; the first (burst), median and last (sustained) region are reported")
     ap.add_argument("--shuffle-rows", type=int, default=0, help="--op shuffle: rows instead of the workload's tokens")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
@@ -350,6 +414,8 @@ def main():
         return run_reference(args, cfg, sparsity)
     if args.op == "shuffle":
         return run_shuffle(args, cfg)
+    if args.op == "peak":
+        return run_peak(args)
     if args.warmup < 3:
         args.warmup = 3
 
@@ -476,6 +542,36 @@ def main():
         torch.cuda.synchronize(dev)
 
     # ---- device-resident timing (the headline): per-phase timers off, nothing but the path between the events
+    def repeat_regions(one_region):
+        """Runs `one_region(index)` (exactly K timed steps; returns its device milliseconds) again and again until
+        the device has been under load for --min-seconds, every rank the same number of times.  Returns the regions
+        as dicts {ms (max over ranks), t0, t1 (host times, for the clock samples)}."""
+        regions, busy = [], 0.0
+        while True:
+            t0 = time.perf_counter()
+            ms = one_region(len(regions))
+            t1 = time.perf_counter()
+            regions.append({"ms": ms, "t0": t0, "t1": t1})
+            busy += t1 - t0
+            (busy_max,) = ranks.max_over_ranks([busy], dev)
+            if busy_max >= args.min_seconds or len(regions) >= 5000:
+                break
+        for r, m in zip(regions, ranks.max_over_ranks([r["ms"] for r in regions], dev)):
+            r["ms"] = m
+        return regions
+
+    def summarise(regions):
+        """First (burst), median and last (sustained) region of a run, each with the clocks sampled while it ran."""
+        order = sorted(range(len(regions)), key=lambda k: regions[k]["ms"])
+        picks = {"first": regions[0], "median": regions[order[len(order) // 2]], "last": regions[-1]}
+        out = {"regions": len(regions), "steps_per_region": args.steps,
+               "seconds_under_load": round(regions[-1]["t1"] - regions[0]["t0"], 3)}
+        for name, r in picks.items():
+            out[name] = {"ms_per_step": r["ms"] / args.steps,
+                         "value": ranks.whole_job_throughput(macs, world, args.steps, r["ms"]),
+                         "clocks": sampler.region(r["t0"], r["t1"]) if rank == 0 else None}
+        return out
+
     for s in range(args.warmup):
         device_step(s, False)
     barrier()
@@ -483,14 +579,18 @@ def main():
     if rank == 0:
         sampler.wait_ready()
     barrier()
+
+    def single_region(index):
+        first = args.warmup + index * args.steps
+        events = [device_step(first + s, True) for s in range(args.steps)]
+        barrier()
+        return float(sum(e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) + e[4].elapsed_time(e[5]) for e in events))
+
     wall0 = time.perf_counter()
-    events = [device_step(args.warmup + s, True) for s in range(args.steps)]
-    barrier()
-    wall = time.perf_counter() - wall0
-    clocks_single = sampler.region(wall0, wall0 + wall) if rank == 0 else None
-    launches = ctx.stats().kernel_launches - launches0
-    step_ms = [e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) + e[4].elapsed_time(e[5]) for e in events]
-    total_ms = float(sum(step_ms))
+    single_regions = repeat_regions(single_region)
+    wall = (time.perf_counter() - wall0) / len(single_regions)
+    launches = (ctx.stats().kernel_launches - launches0) // len(single_regions)
+    single_sum = summarise(single_regions)
 
     # ---- the same steps again with the library's per-phase event timers on: kernel time of each phase
     #      (the timers add two event records per phase, so this pass is slower and is not the headline)
@@ -570,23 +670,27 @@ def main():
             piped_step(s)
         barrier()
         launched0 = sum(cx.stats().kernel_launches for cx, _ in pctx)
-        host0 = time.perf_counter()
-        p0, p1 = ev(), ev()
-        p0.record(tstream)
-        for s in range(args.steps):
-            piped_step(s)
-        for cx, sk in pctx:
-            done = torch.cuda.Event()
-            done.record(sk)
-            tstream.wait_event(done)
-        p1.record(tstream)
-        barrier()
-        clocks_piped = sampler.region(host0, time.perf_counter()) if rank == 0 else None
-        (piped_ms,) = ranks.max_over_ranks([p0.elapsed_time(p1)], dev)
-        piped = {"in_flight": C, "ms_per_step": piped_ms / args.steps,
-                 "launches": int(sum(cx.stats().kernel_launches for cx, _ in pctx) - launched0),
-                 "value": ranks.whole_job_throughput(macs, world, args.steps, piped_ms), "unit": UNIT,
-                 "note": "C independent problems on C streams, inputs bound in place, whole region timed on the device"}
+
+        def piped_region(index):
+            p0, p1 = ev(), ev()
+            p0.record(tstream)
+            for s in range(args.steps):
+                piped_step(index * args.steps + s)
+            for cx, sk in pctx:
+                done = torch.cuda.Event()
+                done.record(sk)
+                tstream.wait_event(done)
+            p1.record(tstream)
+            barrier()
+            return float(p0.elapsed_time(p1))
+
+        piped_regions = repeat_regions(piped_region)
+        piped_sum = summarise(piped_regions)
+        piped = {"in_flight": C, "ms_per_step": piped_sum["median"]["ms_per_step"],
+                 "launches": int(sum(cx.stats().kernel_launches for cx, _ in pctx) - launched0) // len(piped_regions),
+                 "value": piped_sum["median"]["value"], "unit": UNIT, "timed_regions": piped_sum,
+                 "note": "C independent problems on C streams, inputs bound in place, every region of K steps timed "
+                         "as a whole on the device; the median region is the figure"}
 
         # ---- the same C problems in flight end to end: every step copies its inputs from pinned host memory and
         #      its result back, on its context's stream, so one problem's copies run under another's kernels
@@ -634,29 +738,35 @@ def main():
     pairs = [e2e_step(3 + s) for s in range(args.steps)]
     barrier()
     e2e_ms = float(sum(a.elapsed_time(b) for a, b in pairs))
-    sampler.stop()
     h2d = sum(t.numel() * 8 for p in (0, 1) for t in sets[0]["pinned"][p].values()) + sets[0]["mask_host"].numel()
     d2h = 2 * T * d * 8 + 4
 
-    total_ms, e2e_ms = ranks.max_over_ranks([total_ms, e2e_ms], dev)
+    (e2e_ms,) = ranks.max_over_ranks([e2e_ms], dev)
     e2e_single_ms = e2e_ms
     e2e_in_flight = piped is not None and piped_e2e_ms < e2e_ms
     if e2e_in_flight:
         e2e_ms = piped_e2e_ms
 
+    # ---- measured peaks of the two multiply pipes, after the path's own timing (the probes heat the part)
+    pipe_peaks = None
+    if rank == 0 and not args.no_peak_probe:
+        torch.cuda.synchronize(dev)
+        time.sleep(1.0)
+        pipe_peaks = measure_pipe_peaks(sampler)
+    sampler.stop()
+
     if rank == 0:
-        single = {"ms_per_step": total_ms / args.steps,
-                  "value": ranks.whole_job_throughput(macs, world, args.steps, total_ms), "unit": UNIT,
+        single = {"ms_per_step": single_sum["median"]["ms_per_step"], "value": single_sum["median"]["value"],
+                  "unit": UNIT, "timed_regions": single_sum,
                   "note": "one problem at a time on one stream; sum over set_mask, ffn_up + truncate, ffn_down + "
-                          "truncate of CUDA-event pairs; 512 MiB written between steps to flush L2"}
+                          "truncate of CUDA-event pairs; 512 MiB written between steps to flush L2; the median "
+                          "region of K steps is the figure"}
         # Two issue policies are measured in this run; the headline is the faster one (large dense problems gain
         # nothing from sharing the GPU, small sparse ones hide their memory-side kernels under another problem's
         # tensor-core kernel), and both are reported.
         use_piped = piped is not None and piped["value"] > single["value"]
-        if use_piped:
-            ms_per_step, value = piped["ms_per_step"], piped["value"]
-        else:
-            ms_per_step, value = single["ms_per_step"], single["value"]
+        chosen = piped_sum if use_piped else single_sum
+        ms_per_step, value = chosen["median"]["ms_per_step"], chosen["median"]["value"]
         phase = {name: {"ms_per_step": stats.phase_ms[k] / prof_steps, "launches_per_step":
                         stats.phase_launches[k] / prof_steps} for k, name in enumerate(cb.PHASE_NAMES)}
         comb_launch_ms = stats.phase_ms[3] / max(1, stats.phase_launches[3])
@@ -675,8 +785,18 @@ def main():
         # up- and the down-projection launch)
         comb_bytes_per_launch = 8 * ((2 * T * d + 2 * d * g * n + 2 * T * g * n) + (2 * T * n + 2 * n * d + 2 * T * d))
         if used_path == "limb":
-            # int8 tensor peak = measured bf16 peak x nominal ratio 2, in MAC/s, over 36 limb products per ring MAC
-            peak = bf16 * 1e12 / 2 * 2 / 36 / 1e12
+            # The pipe's peak in ring multiply-adds: the measured rate of the tensor instruction the kernel issues,
+            # over 36 limb products.  Beside it, what the measured bf16 GEMM peak would imply at the nominal int8 :
+            # bf16 ratio of 2 (the figure used before the pipe itself was measured).
+            derived = bf16 * 1e12 / 2 * 2 / 36 / 1e12
+            if pipe_peaks is not None:
+                peak = pipe_peaks["tensor_i8"]["ring_mac_burst"] / 1e12
+                peak_sustained = pipe_peaks["tensor_i8"]["ring_mac_sustained"] / 1e12
+                peak_source = ("measured in this run: tcgen05.mma kind::i8 M128 N256 K32 loop on 148 SMs, operands in "
+                               "shared memory, best of the first three 25 ms launches, / 36 limb products")
+            else:
+                peak, peak_sustained = derived, bf16_sustained_derived(peaks)
+                peak_source = f"{src} bf16 GEMM peak x2 (int8 nominal ratio), as MAC/s, / 36 limb products"
             t_tensor = comb_macs_per_launch / (peak * 1e12)
             t_hbm = comb_bytes_per_launch / (hbm * 1e9)
             if t_hbm > t_tensor:
@@ -685,18 +805,46 @@ def main():
                         "unit": "GB/s", "peak_source": f"{src} HBM copy peak"}
             else:
                 roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
-                        "peak_source": f"{src} bf16 GEMM peak x2 (int8 nominal ratio), as MAC/s, / 36 limb products"}
+                        "peak_source": peak_source, "peak_sustained": peak_sustained,
+                        "frac_of_sustained_peak": achieved / peak_sustained,
+                        "peak_from_bf16_gemm": derived, "frac_of_peak_from_bf16_gemm": achieved / derived}
         else:
             # 148 SMs x 64 32-bit integer multiply-add lanes per clock x max SM clock / 4 issue slots per ring MAC
-            peak = 148 * 64 * 1.965e9 / 4 / 1e12
-            roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TMAC64/s",
-                    "peak_source": "148 SM x 64 int32 mul-add lanes/clk x 1.965 GHz / 4 issue slots per 64-bit MAC"}
+            derived = 148 * 64 * 1.965e9 / 4 / 1e12
+            if pipe_peaks is not None:
+                peak = pipe_peaks["alu_u64"]["burst"] / 1e12
+                peak_sustained = pipe_peaks["alu_u64"]["sustained"] / 1e12
+                peak_source = ("measured in this run: eight 64-bit multiply-add chains per thread, 2 x 1024 threads per "
+                               "SM, best of the first three 25 ms launches")
+            else:
+                peak = peak_sustained = derived
+                peak_source = "148 SM x 64 int32 mul-add lanes/clk x 1.965 GHz / 4 issue slots per 64-bit MAC"
+            roof = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TMAC64/s", "peak_source": peak_source,
+                    "peak_sustained": peak_sustained, "frac_of_sustained_peak": achieved / peak_sustained,
+                    "peak_from_unit_counts": derived}
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["kernel"] = "combine_" + used_path + ("_few" if used_path == "limb" and T <= 32 else "")
         roof["traffic"] = combine_traffic(args.workload, sparsity, used_path)
         roof["traffic_unit"] = "bytes per launch (ncu dram read+write); algorithmic: planes once + Z read-modify-write"
         roof["algorithmic_bytes_per_launch"] = comb_bytes_per_launch
-        t_roof = max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (peak * 1e12))     # peak: the multiply pipe's, T MAC64/s
+        roof["timed"] = "kernel time per launch from the per-phase CUDA-event pass, one problem at a time"
+
+        def t_roof_ms(pipe_peak):                 # slower of bytes at the HBM peak and MACs at the pipe's peak
+            return max(ffn_bytes(cfg, T, n) / (hbm * 1e9), macs / (pipe_peak * 1e12)) * 1e3
+
+        path_roof = {"algorithmic_bytes": ffn_bytes(cfg, T, n), "algorithmic_macs": macs, "hbm_gbs": hbm,
+                     "hbm_source": src, "pipe_peak": peak, "pipe_peak_sustained": peak_sustained,
+                     "roofline_ms": t_roof_ms(peak), "roofline_ms_sustained_peak": t_roof_ms(peak_sustained),
+                     "frac": t_roof_ms(peak) / ms_per_step,
+                     "note": "frac = roofline at the burst peak over the median region of the reported policy; below, "
+                             "first region against the burst peak and last region (after --min-seconds of load) "
+                             "against the sustained peak, for both policies"}
+        for name, summ in (("single_problem", single_sum), ("problems_in_flight", piped_sum if piped else None)):
+            if summ is not None:
+                path_roof[name] = {
+                    "frac_first_region_burst_peak": t_roof_ms(peak) / summ["first"]["ms_per_step"],
+                    "frac_median_region_burst_peak": t_roof_ms(peak) / summ["median"]["ms_per_step"],
+                    "frac_last_region_sustained_peak": t_roof_ms(peak_sustained) / summ["last"]["ms_per_step"]}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -707,9 +855,12 @@ def main():
                               "weight rows and intermediates of consecutive steps far exceed the L2); no flush"
                               if use_piped else
                               "512 MiB buffer written between steps, and 4 rotating input sets with different masks"),
-                       "timed": ("every step = set_mask + bind inputs + ffn_up + truncate + ffn_down + truncate; the whole "
-                                 "region of K steps between two CUDA events" if use_piped else
-                                 "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream"),
+                       "timed": ("every step = set_mask + bind inputs + ffn_up + truncate + ffn_down + truncate; a region "
+                                 "of exactly K steps between two CUDA events" if use_piped else
+                                 "set_mask + ffn_up + truncate + ffn_down + truncate, CUDA events on the library stream, "
+                                 "summed over a region of exactly K steps") +
+                                f"; the region is repeated for {args.min_seconds} s of load and the median region is "
+                                "the value (first and last regions under timed_regions)",
                        "token_masks": (f"per-token Bernoulli({args.token_masks}) masks over the active blocks, "
                                        f"{stats.n_components} component(s)"
                                        + (f", {args.clusters} groups of requests" if args.clusters > 1 else "")
@@ -717,7 +868,8 @@ def main():
                        "up_projection_under_token_mask": up_counts,
                        "parallelism": f"independent FFN per GPU x{world}"},
             "gpu_launches": int(piped["launches"] if use_piped else launches),
-            "clocks": clocks_piped if use_piped else clocks_single,
+            "clocks": chosen["median"]["clocks"],
+            "timed_regions": chosen,
             "e2e": {"value": ranks.whole_job_throughput(macs, world, args.steps, e2e_ms), "unit": UNIT,
                     "ms_per_step": e2e_ms / args.steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "in_flight": args.in_flight if e2e_in_flight else 1,
@@ -726,9 +878,8 @@ def main():
                     "note": "host buffers through the C ABI: H2D of every per-step input from pinned memory and D2H of "
                             "the result inside the timed region; the faster of one problem at a time and C in flight"},
             "roofline": roof,
-            "path_roofline": {"algorithmic_bytes": ffn_bytes(cfg, T, n), "algorithmic_macs": macs,
-                              "hbm_gbs": hbm, "hbm_source": src, "roofline_ms": t_roof * 1e3,
-                              "frac": t_roof * 1e3 / ms_per_step},
+            "path_roofline": path_roof,
+            "pipe_peaks": pipe_peaks,
             "single_problem": single,
             "problems_in_flight": piped,
             "phases": phase,

@@ -281,6 +281,25 @@ int comet_stats(comet_ctx* ctx, comet_stats_t* out);
  * bracketed by two events recorded on the context's stream. */
 int comet_set_profiling(comet_ctx* ctx, int on);
 
+/* Wait for everything this context has enqueued (its stream and its internal
+ * stream) and report whether any of its kernels gave up on a bounded wait.
+ * Every device-side wait of the tensor-core kernels (on a copy, on the tensor
+ * pipe, on the accumulators) ends after about two seconds; the kernel then lets
+ * its copies in flight land, frees its tensor memory, returns, and writes an
+ * error word that the host reads here.  COMET_ERR_TIMEOUT means that a result
+ * of this context holds only part of its sums.  The word is never cleared: a
+ * context that has timed out is to be destroyed.  comet_set_mask and comet_get
+ * report the same condition as soon as they see it (comet_get does not wait
+ * for the copy it enqueues, so only a comet_synchronize after it is a
+ * guarantee for that copy).  Errors: INVALID_ARG, CUDA, TIMEOUT. */
+int comet_synchronize(comet_ctx* ctx);
+
+/* Test hook: marks the context as if one of its kernels had given up on a
+ * bounded wait (it waits for the stream, then sets the error words such a
+ * kernel would have set).  Nothing is launched.  It lets a caller exercise its
+ * handling of COMET_ERR_TIMEOUT without any kernel actually waiting. */
+int comet_inject_timeout(comet_ctx* ctx);
+
 /* Text for an error code; never NULL. */
 const char* comet_strerror(int code);
 
@@ -404,12 +423,16 @@ int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], const uint64
  * All pointers are DEVICE pointers on the CURRENT device, owned by the caller:
  * X[i], A[i] are [T, K]; Y[i], B[i] are [N, K] (output-feature-major, like the
  * weights above); C[i], Z[i] are [T, N]; i = 0, 1 is the party.  K must be a
- * multiple of 8 and N a multiple of 4.  The work is enqueued on `cuda_stream`
+ * multiple of 8 and N a multiple of 4, and every one of the twelve pointers
+ * must be 16-byte aligned (the kernels move two words at a time; a pointer
+ * carved out of a pool at an odd word is refused with INVALID_ARG before
+ * anything is launched).  The work is enqueued on `cuda_stream`
  * (NULL = default stream) and the call returns without waiting for it.
  *
  * Limit: 2 * (T*K + N*K) <= COMET_STATIC_SCRATCH_WORDS, otherwise nothing is
  * launched and COMET_ERR_SCRATCH_LIMIT is returned.  Other errors: INVALID_ARG
- * (null pointer), SHAPE (non-positive size or the divisibility rule), CUDA.
+ * (null or unaligned pointer), SHAPE (non-positive size or the divisibility
+ * rule), CUDA.
  *
  * The first call on each device looks up the device address of the array
  * (once per device; no allocation).  Make that first call outside any stream
@@ -425,6 +448,32 @@ int comet_beaver_mul(void* cuda_stream, const uint64_t* const X[2], const uint64
 int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* const X[2], const uint64_t* const A[2],
                                const uint64_t* const Y[2], const uint64_t* const B[2], const uint64_t* const C[2],
                                uint64_t* const Z[2], int32_t T, int32_t K, int32_t N);
+
+/* ---------------------------------------------------------------------------
+ * Measured peak of a multiply pipe.  (Not an operation of the paper: it supports
+ * the roofline the benchmark reports, whose compute leg is "multiply-adds at the
+ * measured peak of the chosen multiply pipe".)
+ *
+ * COMET_PIPE_TENSOR_I8: one CTA per SM issues `work` batches of 32
+ *   tcgen05.mma kind::i8 instructions (M 128 x N 256 x K 32, u8 x u8 -> s32) on
+ *   operand tiles that stay in shared memory, accumulators in tensor memory --
+ *   the instruction the limb-plane kernel runs on, without any memory traffic.
+ * COMET_PIPE_ALU_U64: two CTAs of 1024 threads per SM run `work` rounds of eight
+ *   independent 64-bit multiply-add chains per thread -- the inner loop of the
+ *   CUDA-core kernel without its loads.
+ * `launches` such kernels are enqueued back to back on `cuda_stream` (NULL =
+ * default stream) of the current device, each bracketed by CUDA events, and the
+ * call waits for them.  ms_out[launches] (HOST) receives the duration of each
+ * launch in milliseconds, *macs_per_launch_out the 8-bit (tensor) or 64-bit
+ * (ALU) multiply-adds one launch performs; the first launches show the burst
+ * rate, later ones the rate the power limit sustains.  A ring multiply-add
+ * costs 36 of the 8-bit ones.  Allocates a small sink buffer and the events for
+ * the duration of the call.  Errors: INVALID_ARG, SHAPE (launches outside
+ * [1, 4096], work outside [1, 2^24]), OOM, CUDA, TIMEOUT (a bounded wait of the
+ * tensor probe ran out). */
+enum { COMET_PIPE_TENSOR_I8 = 0, COMET_PIPE_ALU_U64 = 1 };
+int comet_pipe_probe(void* cuda_stream, int pipe, int32_t launches, int32_t work, float* ms_out,
+                     double* macs_per_launch_out);
 
 #ifdef __cplusplus
 }

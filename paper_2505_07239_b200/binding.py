@@ -31,10 +31,12 @@ EXPORTS = (
     "comet_truncate", "comet_get", "comet_get_index", "comet_stats", "comet_strerror", "comet_last_cuda_error",
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
     "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
-    "comet_add_bias", "comet_bind_shares", "comet_truncate_pair",
+    "comet_add_bias", "comet_bind_shares", "comet_truncate_pair", "comet_synchronize", "comet_inject_timeout",
+    "comet_pipe_probe",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
+ERR_TIMEOUT = -6
 NUM_PHASES = 5
 PHASE_NAMES = ("compact", "open", "prep", "combine", "truncate")
 
@@ -87,6 +89,10 @@ def _load():
     lib.comet_strerror.restype = ctypes.c_char_p
     lib.comet_last_cuda_error.argtypes = [vp]
     lib.comet_set_profiling.argtypes = [vp, ctypes.c_int]
+    lib.comet_synchronize.argtypes = [vp]
+    lib.comet_inject_timeout.argtypes = [vp]
+    lib.comet_pipe_probe.argtypes = [vp, ctypes.c_int, i32, i32, ctypes.POINTER(ctypes.c_float),
+                                     ctypes.POINTER(ctypes.c_double)]
     pair = ctypes.c_void_p * 2
     lib.comet_beaver_matmul_static.argtypes = [vp, pair, pair, pair, pair, pair, pair, i32, i32, i32]
     lib.comet_shuffle.argtypes = [vp, pair, pair, pair, pair, pair, pair, pair, i64, i64, vp]
@@ -148,10 +154,8 @@ class Comet:
             pass
 
     def synchronize(self):
-        if self.stream is not None:
-            self.stream.synchronize()
-        else:
-            torch.cuda.default_stream(self.device).synchronize()
+        """Wait for the context's work; raises if one of its kernels gave up on a bounded wait."""
+        self._check(_lib.comet_synchronize(self._h), "comet_synchronize")
 
     # ------------------------------------------------------------------ the six calls
     def load_shares(self, party: int, tensor_id: int, t):
@@ -277,6 +281,21 @@ def beaver_matmul_static(X, A, Y, B, C, Z, stream: Optional[torch.cuda.Stream] =
     sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
     return _lib.comet_beaver_matmul_static(sp, ptrs(X, (T, K)), ptrs(A, (T, K)), ptrs(Y, (N, K)), ptrs(B, (N, K)),
                                            ptrs(C, (T, N)), ptrs(Z, (T, N)), T, K, N)
+
+
+PIPE_TENSOR_I8, PIPE_ALU_U64 = 0, 1
+
+
+def pipe_probe(pipe: int, launches: int, work: int, stream: Optional[torch.cuda.Stream] = None):
+    """Measured rate of a multiply pipe (comet_pipe_probe): returns (ms per launch [launches], multiply-adds per
+    launch): 8-bit ones for PIPE_TENSOR_I8, 64-bit ones for PIPE_ALU_U64."""
+    ms = (ctypes.c_float * launches)()
+    macs = ctypes.c_double(0.0)
+    sp = ctypes.c_void_p(stream.cuda_stream if stream is not None else 0)
+    code = _lib.comet_pipe_probe(sp, pipe, launches, work, ms, ctypes.byref(macs))
+    if code != OK:
+        raise CometError(code, "comet_pipe_probe")
+    return [float(v) for v in ms], macs.value
 
 
 def _pair(ts, shape=None, dtype=None):

@@ -16,6 +16,7 @@
 #include "kernels_limb.cuh"
 #include "kernels_mul.cuh"
 #include "kernels_open.cuh"
+#include "kernels_peak.cuh"
 #include "kernels_shuffle.cuh"
 #include "kernels_simt.cuh"
 
@@ -68,7 +69,8 @@ struct comet_ctx {
     int64_t component_pairs;      // sum over components of token rows x active blocks
     int32_t* d_ids;
     int32_t* d_count;             // {count, error flag of the bounded waits}
-    int32_t* h_count;             // pinned and mapped: {count, error flag} as the compaction kernel reports them
+    int32_t* h_count;             // pinned and mapped: {count, error flag as the compaction kernel saw it, ticket,
+                                  // error word written by a kernel whose bounded wait ran out}
     int32_t* h_count_dev;         // device-side address of h_count
     int top_priority;             // the device's highest stream / launch priority (numerically lowest)
     int32_t ticket;               // sequence number of the last compaction launch (echoed in h_count[2])
@@ -173,6 +175,13 @@ cudaMemcpyKind copy_kind(int location, bool to_library) {
 }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// True once a kernel of this context gave up on a bounded wait (the word is written by the kernel itself, in
+// mapped host memory, and never cleared: the context's results are not to be trusted from then on).
+inline bool timed_out(const comet_ctx* c) {
+    return *reinterpret_cast<volatile int32_t*>(c->h_count + 3) != 0 ||
+           *reinterpret_cast<volatile int32_t*>(c->h_count + 1) != 0;
+}
 
 // One Pi_MatMul of the path: sizes and tensor ids.
 struct Proj {
@@ -315,6 +324,7 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
     }
     a.M = pr.M; a.N = pr.N; a.mt = mt; a.nt = nt; a.kb = kb;
     a.error_flag = c->d_error;
+    a.error_host = c->h_count_dev + 3;
     a.ldz = pr.N; a.bs = c->cfg.block; a.group_units = 0;
     a.groups = nullptr; a.row_map = nullptr; a.col_map = nullptr;
     const bool grouped = c->grouped && !few;
@@ -548,7 +558,7 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     ok = ok && cudaMemset(c->d_count, 0, 2 * sizeof(int32_t)) == cudaSuccess;
     if (ok) c->d_error = c->d_count + 1;
     ok = ok && cudaHostAlloc((void**)&c->h_count, 4 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
-    if (ok) c->h_count[2] = 0;
+    if (ok) c->h_count[2] = c->h_count[3] = 0;
     ok = ok && cudaHostGetDevicePointer((void**)&c->h_count_dev, c->h_count, 0) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -682,7 +692,7 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
         if (!arrived) COMET_CUDA(c, cudaStreamSynchronize(c->stream));
         std::atomic_thread_fence(std::memory_order_acquire);
     }
-    if (c->h_count[1] != 0) return COMET_ERR_TIMEOUT;     // an earlier kernel gave up on a bounded wait
+    if (timed_out(c)) return COMET_ERR_TIMEOUT;           // an earlier kernel gave up on a bounded wait
     const int32_t blocks = *c->h_count;
     const int64_t n = (int64_t)blocks * c->cfg.block;
     if (n > c->cap_n) {            // more active neurons than the context was sized for
@@ -712,8 +722,10 @@ int comet_set_token_mask(comet_ctx* c, const uint8_t* token_mask, int location, 
     if (!c->mask_set) return COMET_ERR_STATE;
     if (!token_mask) {                         // back to "every token uses every active neuron"
         if (tokens != 0 || n_active_blocks != 0) return COMET_ERR_INVALID_ARG;
+        // the weight side of the down-projection may have been opened early under the mask that is going away
+        // (its unused blocks zeroed, its contraction index in component order): it is opened again
+        if (c->tmask_set) c->dn_right_ready = false;
         c->tmask_set = false;
-        if (c->grouped) c->dn_right_ready = false;
         c->grouped = false;
         if (masked_out) *masked_out = 0;
         return COMET_OK;
@@ -982,6 +994,24 @@ int comet_get(comet_ctx* c, int party, int tensor_id, uint64_t* out, int locatio
         COMET_CUDA(c, cudaMemcpyAsync(out, c->buf[party][tensor_id], (size_t)words * sizeof(u64),
                                       copy_kind(location, false), c->stream));
     if (written) *written = words;
+    if (timed_out(c)) return COMET_ERR_TIMEOUT;    // what has been handed out is not the result
+    return COMET_OK;
+}
+
+int comet_synchronize(comet_ctx* c) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (c->side) COMET_CUDA(c, cudaStreamSynchronize(c->side));
+    std::atomic_thread_fence(std::memory_order_acquire);
+    return timed_out(c) ? COMET_ERR_TIMEOUT : COMET_OK;
+}
+
+int comet_inject_timeout(comet_ctx* c) {
+    if (!c) return COMET_ERR_INVALID_ARG;
+    COMET_CUDA(c, cudaStreamSynchronize(c->stream));
+    const int32_t one = 1;
+    COMET_CUDA(c, cudaMemcpy(c->d_error, &one, sizeof(one), cudaMemcpyHostToDevice));
+    c->h_count[3] = 1;
     return COMET_OK;
 }
 
@@ -1086,6 +1116,12 @@ extern "C" int comet_beaver_matmul_static(void* cuda_stream, const uint64_t* con
     if (!X || !A || !Y || !B || !C || !Z) return COMET_ERR_INVALID_ARG;
     for (int p = 0; p < 2; ++p)
         if (!X[p] || !A[p] || !Y[p] || !B[p] || !C[p] || !Z[p]) return COMET_ERR_INVALID_ARG;
+    // the kernels below read and write every operand 16 bytes at a time
+    for (int p = 0; p < 2; ++p) {
+        const void* ptrs[6] = {X[p], A[p], Y[p], B[p], C[p], Z[p]};
+        for (const void* q : ptrs)
+            if ((reinterpret_cast<uintptr_t>(q) & 15u) != 0) return COMET_ERR_INVALID_ARG;
+    }
     if (T < 1 || K < 8 || N < 4 || K % 8 || N % 4) return COMET_ERR_SHAPE;
     const int64_t left = (int64_t)T * K, right = (int64_t)N * K;
     if (2 * (left + right) > (int64_t)COMET_STATIC_SCRATCH_WORDS) return COMET_ERR_SCRATCH_LIMIT;
@@ -1312,4 +1348,66 @@ extern "C" int comet_add_bias(void* cuda_stream, uint64_t* const Z[2], const uin
     g.cols = (int)cols;
     comet::add_bias_kernel<<<dim3(shuffle_grid(rows * cols), 2), 256, 0, (cudaStream_t)cuda_stream>>>(g);
     return cudaGetLastError() == cudaSuccess ? COMET_OK : COMET_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
+// Measured peak of a multiply pipe (support for the roofline; not a step of the path).
+// ---------------------------------------------------------------------------
+extern "C" int comet_pipe_probe(void* cuda_stream, int pipe, int32_t launches, int32_t work, float* ms_out,
+                                double* macs_per_launch_out) {
+    namespace pk = comet::peak;
+    if (!ms_out || !macs_per_launch_out) return COMET_ERR_INVALID_ARG;
+    if (pipe != COMET_PIPE_TENSOR_I8 && pipe != COMET_PIPE_ALU_U64) return COMET_ERR_INVALID_ARG;
+    if (launches < 1 || launches > 4096 || work < 1 || work > (1 << 24)) return COMET_ERR_SHAPE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return COMET_ERR_CUDA;
+    }
+    const int alu_blocks = sms * 2;
+    const size_t sink_bytes = pipe == COMET_PIPE_TENSOR_I8 ? (size_t)sms * 32 * sizeof(unsigned) + sizeof(int)
+                                                           : (size_t)alu_blocks * pk::ALU_THREADS * sizeof(u64);
+    void* sink = nullptr;
+    if (cudaMalloc(&sink, sink_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return COMET_ERR_OOM;
+    }
+    std::vector<cudaEvent_t> ev((size_t)launches + 1, nullptr);
+    int rc = COMET_OK;
+    for (auto& e : ev)
+        if (cudaEventCreate(&e) != cudaSuccess) rc = COMET_ERR_CUDA;
+    int* flag = reinterpret_cast<int*>(static_cast<char*>(sink) + (size_t)sms * 32 * sizeof(unsigned));
+    if (rc == COMET_OK && cudaMemsetAsync(sink, 0, sink_bytes, stream) != cudaSuccess) rc = COMET_ERR_CUDA;
+    if (rc == COMET_OK) {
+        for (int i = 0; i < launches; ++i) {
+            cudaEventRecord(ev[i], stream);
+            if (pipe == COMET_PIPE_TENSOR_I8)
+                comet::tensor_i8_probe_kernel<<<sms, pk::THREADS, 0, stream>>>(work, 0x9E3779B9u + i, flag,
+                                                                                static_cast<unsigned*>(sink));
+            else
+                comet::alu_u64_probe_kernel<<<alu_blocks, pk::ALU_THREADS, 0, stream>>>(work, 0x9E3779B97F4A7C15ull + i,
+                                                                                         static_cast<u64*>(sink));
+        }
+        cudaEventRecord(ev[launches], stream);
+        if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess) rc = COMET_ERR_CUDA;
+    }
+    if (rc == COMET_OK) {
+        for (int i = 0; i < launches; ++i)
+            if (cudaEventElapsedTime(&ms_out[i], ev[i], ev[i + 1]) != cudaSuccess) rc = COMET_ERR_CUDA;
+        if (pipe == COMET_PIPE_TENSOR_I8) {
+            int h_flag = 0;
+            if (cudaMemcpy(&h_flag, flag, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) rc = COMET_ERR_CUDA;
+            else if (h_flag) rc = COMET_ERR_TIMEOUT;
+            *macs_per_launch_out = (double)sms * work * pk::BATCH * ((double)pk::M * pk::N * pk::KC);
+        } else {
+            *macs_per_launch_out = (double)alu_blocks * pk::ALU_THREADS * pk::ALU_CHAINS * (double)work;
+        }
+    }
+    for (auto e : ev)
+        if (e) cudaEventDestroy(e);
+    cudaFree(sink);
+    if (rc == COMET_ERR_CUDA) cudaGetLastError();
+    return rc;
 }

@@ -723,6 +723,7 @@ struct LimbArgs {
     int M, N;                // N a multiple of 16
     int mt, nt, kb;          // tiles and k-blocks per operand pair; one tile runs over 2*kb blocks
     int* error_flag;         // set to 1 if a bounded wait ran out
+    int* error_host;         // the same report in mapped host memory, so that the host sees it without a copy
     // Only read by the grouped kernel (one multiplication per connected component): the planes hold the operands
     // in component-sorted order, M counts the rows that lie in a component (and N the columns, when col_map is
     // given), and every row tile runs over the column tiles and k-blocks its LimbGroupRow names.  kb stays the
@@ -1046,7 +1047,11 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
 
     ptx::fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0 && abort_flag) *a.error_flag = 1;
+    if (threadIdx.x == 0 && abort_flag) {
+        *a.error_flag = 1;
+        *reinterpret_cast<volatile int*>(a.error_host) = 1;
+        __threadfence_system();
+    }
     if (warp == 0) {
         ptx::fence_after_sync();
         ptx::tmem_dealloc(tmem_base, 512);
@@ -1296,7 +1301,11 @@ combine_limb_few_kernel(LimbArgs a) {
 
     ptx::fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0 && abort_flag) *a.error_flag = 1;
+    if (threadIdx.x == 0 && abort_flag) {
+        *a.error_flag = 1;
+        *reinterpret_cast<volatile int*>(a.error_host) = 1;
+        __threadfence_system();
+    }
     if (warp == 0) {
         ptx::fence_after_sync();
         ptx::tmem_dealloc(tmem_base, limb_few::TMEM_COLS);

@@ -230,3 +230,66 @@ def run_and_compare_sampled(cfg, seed, sparsity=None, tokens=None, step=0, matmu
     if own_ctx:
         ctx.close()
     return report
+
+
+def run_and_compare_products(cfg, seed, sparsity=None, tokens=None, step=0, matmul_path=cb.PATH_AUTO, ctx=None,
+                             weights=None, early_down=True):
+    """Full-size check, element by element: both projections under the configuration's mask on uniformly random
+    shares (what the kernels see whatever the plaintext distribution), with the messages, the products and the
+    truncated products of both parties compared in full with `oracle.somm` / `oracle.simm` / `oracle.truncate`.
+    The two projections are exercised independently (the hidden state is synthetic), so no reconstruction or
+    float64 report is made here; `run_and_compare_full` does that on real plaintexts."""
+    T = cfg.tokens if tokens is None else tokens
+    d, f, g = cfg.d_model, cfg.frac_bits, cfg.groups
+    report = {"config": cfg.name, "tokens": T, "compared": [], "mismatches": 0}
+    W = weights if weights is not None else wl.model_shares(cfg, seed, plain=False)
+    _, X0, X1 = wl.activation_shares(cfg, seed, step=step, tokens=T)
+    mask = wl.block_mask(cfg, seed, sparsity, step)
+    own_ctx = ctx is None
+    if own_ctx:
+        ctx = make_context(cfg, T, matmul_path)
+        load_weights(ctx, cfg, W)
+    for party, Xs in ((0, X0), (1, X1)):
+        ctx.load_shares(party, cb.X, cb.to_device(Xs))
+    n = ctx.set_mask(mask)
+    I1 = oracle.index_set(mask, cfg.block, 1)
+    Ig = oracle.index_set(mask, cfg.block, g)
+    report["n_active"] = n
+    assert n == I1.size
+
+    tri = wl.dealer_triple(seed, f"{cfg.name}/up/step{step}", T, d, g * n, valid=False)
+    load_triple_up(ctx, tri)
+    trd = wl.dealer_triple(seed, f"{cfg.name}/down/step{step}", T, n, d, valid=False)
+    if early_down:
+        load_triple_down(ctx, trd)
+    ctx.ffn_up(T)
+    report["path"] = ctx.stats().matmul_path
+    Zg = [ctx.get(party, cb.Z_UP, (T, g * n)) for party in (0, 1)]
+    ctx.truncate(cb.Z_UP)
+    ref = oracle.somm((X0, X1), (oracle_up_operand(cfg, W, 1), oracle_up_operand(cfg, W, 2)), Ig,
+                      tri["A"][1:], tri["B"][1:], tri["C"][1:])
+    for party in (0, 1):
+        _mismatch(f"E_up[{party}]", ctx.get(party, cb.E_UP, (T, d)), ref["E"][party], report)
+        _mismatch(f"F_up[{party}]", ctx.get(party, cb.F_UP, (g * n, d)).T, ref["F"][party], report)
+        _mismatch(f"Z_up[{party}]", Zg[party], ref["Z"][party], report)
+        _mismatch(f"trunc(Z_up)[{party}]", ctx.get(party, cb.Z_UP, (T, g * n)),
+                  oracle.truncate(party, ref["Z"][party], f), report)
+
+    _, H0, H1 = wl.hidden_shares(cfg, seed, n, step=step, tokens=T)
+    for party, Hs in ((0, H0), (1, H1)):
+        ctx.load_shares(party, cb.H, cb.to_device(Hs))
+    if not early_down:
+        load_triple_down(ctx, trd)
+    ctx.ffn_down(T)
+    Yg = [ctx.get(party, cb.Y, (T, d)) for party in (0, 1)]
+    ctx.truncate(cb.Y)
+    refd = oracle.simm((H0, H1), W["W2"][1:], I1, trd["A"][1:], trd["B"][1:], trd["C"][1:])
+    for party in (0, 1):
+        _mismatch(f"E_dn[{party}]", ctx.get(party, cb.E_DN, (T, n)), refd["E"][party], report)
+        _mismatch(f"F_dn[{party}]", ctx.get(party, cb.F_DN, (d, n)).T, refd["F"][party], report)
+        _mismatch(f"Y[{party}]", Yg[party], refd["Z"][party], report)
+        _mismatch(f"trunc(Y)[{party}]", ctx.get(party, cb.Y, (T, d)), oracle.truncate(party, refd["Z"][party], f),
+                  report)
+    if own_ctx:
+        ctx.close()
+    return report

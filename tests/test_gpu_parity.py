@@ -109,6 +109,64 @@ def test_opt67b_decode_steps_sampled(hz, path):
     ctx.close()
 
 
+# ---- every benchmark configuration at full size, products compared element by element (not at samples)
+
+@pytest.mark.parametrize("path", PATHS)
+def test_opt13b_90_products_in_full(hz, path):
+    """The headline configuration: OPT-1.3B shape at 90 % block sparsity."""
+    r = _ok(hz.run_and_compare_products(wl.CONFIGS["opt1.3b"], seed=21, sparsity=0.9, matmul_path=path), path)
+    assert r["n_active"] == 832
+
+
+@pytest.mark.parametrize("sparsity,n", [(0.8, 1632), (0.5, 4096), (0.0, 8192)])
+def test_opt13b_sweep_products_in_full(hz, sparsity, n):
+    """The rest of the sparsity sweep on the default (tensor-core) path; n = 1632 leaves a ragged column tile."""
+    r = _ok(hz.run_and_compare_products(wl.CONFIGS["opt1.3b"], seed=22, sparsity=sparsity), 2)
+    assert r["n_active"] == n
+
+
+def test_llama7b_products_in_full(hz):
+    r = _ok(hz.run_and_compare_products(wl.CONFIGS["llama7b"], seed=23), 2)
+    assert 23 * 64 <= r["n_active"] <= 26 * 64
+
+
+def test_opt67b_decode_steps_products_in_full(hz):
+    cfg = wl.CONFIGS["opt6.7b-decode"]
+    W = wl.model_shares(cfg, 24, plain=False)
+    ctx = hz.make_context(cfg, cfg.tokens, 2, max_active=2048)
+    hz.load_weights(ctx, cfg, W)
+    for step in (0, 1, 63):       # fresh mask, X and triples per step, weights loaded once
+        r = _ok(hz.run_and_compare_products(cfg, seed=24, step=step, ctx=ctx, weights=W), 2)
+        assert r["n_active"] == 1312
+    ctx.close()
+
+
+def test_timeout_status_reaches_the_caller(hz):
+    """COMET_ERR_TIMEOUT is handed out by the calls that hand results out.  No kernel waits here: the error
+    words a timed-out kernel would write are set through the library's test hook."""
+    from paper_2505_07239_b200 import binding as cb
+
+    cfg = wl.CONFIGS["tiny"]
+    r = hz.run_and_compare_full(cfg, seed=25, float_report=False)
+    assert r["mismatches"] == 0
+    ctx = hz.make_context(cfg, cfg.tokens)
+    lib, h = cb.library(), ctx._h
+    W = wl.model_shares(cfg, 25, plain=False)
+    hz.load_weights(ctx, cfg, W)
+    assert lib.comet_synchronize(h) == cb.OK
+    assert lib.comet_inject_timeout(h) == cb.OK
+    assert lib.comet_synchronize(h) == cb.ERR_TIMEOUT
+    out = torch.zeros(cfg.d_ff * cfg.d_model, dtype=torch.int64, device="cuda")
+    assert lib.comet_get(h, 0, cb.W1, out.data_ptr(), 0, out.numel(), None) == cb.ERR_TIMEOUT
+    n = ctypes.c_int32(0)
+    m = torch.ones(cfg.n_blocks, dtype=torch.uint8, device="cuda")
+    assert lib.comet_set_mask(h, m.data_ptr(), 0, cfg.n_blocks, ctypes.byref(n)) == cb.ERR_TIMEOUT
+    assert b"bounded" in lib.comet_strerror(cb.ERR_TIMEOUT)
+    ctx.close()
+    # another context is unaffected
+    assert hz.run_and_compare_full(cfg, seed=26, float_report=False)["mismatches"] == 0
+
+
 def test_masked_neurons_contribute_exactly_zero(hz):
     """Garbage in the weight shares of inactive neurons leaves every output bit unchanged."""
     from paper_2505_07239_b200 import binding as cb

@@ -176,3 +176,50 @@ def test_token_mask_errors():
     assert lib.comet_set_token_mask(h, m.data_ptr(), 0, cfg.tokens, 3, ctypes.byref(out)) == 0
     assert out.value == cfg.tokens * 96
     ctx.close()
+
+
+@pytest.mark.parametrize("tokens", [16, 70])
+def test_token_mask_cleared_between_the_projections(tokens):
+    """The up-projection runs under a token mask in which one active block is used by no token and, since W2 and
+    B' are already loaded, opens the down-projection's weight side early with that block's rows zeroed; the mask
+    is then cleared, so the down-projection is the token-shared one and must open those rows after all."""
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2505_07239_b200 import binding as cb
+    from tests import harness as hz
+
+    cfg = wl.FFNConfig("rowsets-clear", tokens, 128, 512, 32, 16, False, 0.5, "uniform", "normal", "normal0.02")
+    seed, T, d = 910 + tokens, tokens, cfg.d_model
+    W = wl.model_shares(cfg, seed, plain=False)
+    mask = wl.block_mask(cfg, seed, 0.5)
+    I = oracle.index_set(mask, cfg.block, 1)
+    n, nab = I.size, int(mask.sum())
+    tm = wl.token_block_masks(seed, "tm", T, nab, 0.4)
+    tm[:, 1] = 0
+    S = np.repeat(tm, cfg.block, axis=1)
+    _, X0, X1 = wl.activation_shares(cfg, seed, tokens=T)
+    _, H0, H1 = wl.hidden_shares(cfg, seed, n, tokens=T)
+    tri = wl.dealer_triple_components(seed, "up", S, d)
+    full = wl.dealer_triple(seed, "down/full", T, n, d, valid=False)
+
+    ctx = hz.make_context(cfg, T, cb.PATH_LIMB)
+    hz.load_weights(ctx, cfg, W)
+    assert ctx.set_mask(mask) == n
+    ctx.set_token_mask(tm)
+    for p, Xs in ((0, X0), (1, X1)):
+        ctx.load_shares(p, cb.X, cb.to_device(Xs))
+    hz.load_triple_up(ctx, tri)
+    hz.load_triple_down(ctx, full)                  # W2 and B' are there: the weight side is opened during ffn_up
+    ctx.ffn_up(T)
+    assert ctx.set_token_mask(None) == 0
+    for p, Hs in ((0, H0), (1, H1)):
+        ctx.load_shares(p, cb.H, cb.to_device(Hs))
+    ctx.ffn_down(T)
+    ref = oracle.simm((H0, H1), W["W2"][1:], I, full["A"][1:], full["B"][1:], full["C"][1:])
+    bad = 0
+    for p in (0, 1):
+        bad += int((ctx.get(p, cb.E_DN, (T, n)) != ref["E"][p]).sum())
+        bad += int((ctx.get(p, cb.F_DN, (d, n)).T != ref["F"][p]).sum())
+        bad += int((ctx.get(p, cb.Y, (T, d)) != ref["Z"][p]).sum())
+    ctx.close()
+    assert bad == 0
