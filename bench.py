@@ -322,6 +322,125 @@ def run_shuffle(args, cfg):
                      "peak_source": "measured" if peaks else "fallback"}}))
 
 
+# --------------------------------------------------------------------------- one layer sharded over the neurons
+def run_sharded(args, cfg, sparsity):
+    """`--shard neurons`: ONE FFN problem per step for the whole job, its neurons dealt to the ranks block by block
+    (rank r owns blocks r, r + N, ...; it stores only its slice of the weights).  The up-projection needs no
+    exchange; every rank's down-projection is a partial sum of Eq. 1, the partial shares are added over the ranks
+    with one integer all-reduce per party, and the sum is truncated.  Strong scaling: the work per step is fixed."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_07239_b200 import binding as cb
+    from paper_2505_07239_b200 import shard
+
+    rank, world, local = ranks.rank_world_local()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    assert cfg.n_blocks % world == 0, "the block count must be a multiple of the number of ranks"
+    if args.warmup < 3:
+        args.warmup = 3
+    T, d, g, f = cfg.tokens, cfg.d_model, cfg.groups, cfg.frac_bits
+    seed = 1000                                       # the same layer on every rank
+    stream = torch.cuda.Stream(device=dev)
+    n_glob = cfg.n_active_blocks(sparsity) * cfg.block
+    ctx = cb.Comet(T, d, cfg.d_ff // world, cfg.block, f, cfg.groups - 1, local, 0, cb.PATH_AUTO, stream)
+    W = wl.model_shares(cfg, seed, plain=False)
+    with torch.cuda.stream(stream):
+        for p in (0, 1):
+            w1, w2 = shard.slice_stored_weights(wl.lib_layout(W["W1"][1 + p]), wl.lib_layout(W["W2"][1 + p]),
+                                                cfg.block, rank, world)
+            ctx.load_shares(p, cb.W1, cb.to_device(w1, dev))
+            ctx.load_shares(p, cb.W2, cb.to_device(w2, dev))
+            if cfg.gated:
+                wg, _ = shard.slice_stored_weights(wl.lib_layout(W["WG"][1 + p]), wl.lib_layout(W["W2"][1 + p]),
+                                                   cfg.block, rank, world)
+                ctx.load_shares(p, cb.WG, cb.to_device(wg, dev))
+    ctx.synchronize()
+    del W
+    sets = []
+    for s_ in range(4):
+        inp = make_inputs(cfg, seed, sparsity, s_, T)
+        cols = shard.local_columns(inp["mask"], cfg.block, rank, world)
+        gcols = np.concatenate([cols + k * inp["n"] for k in range(g)])          # [gate(I_r) || up(I_r)]
+        zero = np.zeros((T, d), np.uint64)
+        per = []
+        for p in (0, 1):
+            per.append({k: cb.to_device(np.ascontiguousarray(v), dev) for k, v in {
+                cb.X: inp["X"][p], cb.A_UP: inp["up"]["A"][1 + p],
+                cb.B_UP: wl.lib_layout(inp["up"]["B"][1 + p][:, gcols]), cb.C_UP: inp["up"]["C"][1 + p][:, gcols],
+                cb.H: inp["H"][p][:, cols], cb.A_DN: inp["dn"]["A"][1 + p][:, cols],
+                cb.B_DN: wl.lib_layout(inp["dn"]["B"][1 + p][cols, :]),
+                cb.C_DN: inp["dn"]["C"][1 + p] if rank == 0 else zero}.items()})    # C' enters the sum once
+        sets.append({"mask": torch.from_numpy(shard.local_mask(inp["mask"], rank, world)).to(dev), "dev": per,
+                     "n_local": cols.size})
+    torch.cuda.synchronize(dev)
+    macs = ffn_macs(cfg, T, n_glob)
+    y_view = [ctx.result_view(p, cb.Y, (T, d)) for p in (0, 1)]
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def step(k):
+        st = sets[k % 4]
+        with torch.cuda.stream(stream):
+            ctx.set_mask(st["mask"])
+            for p in (0, 1):
+                for tid, t in st["dev"][p].items():
+                    if t.numel() and tid != cb.H:
+                        ctx.bind_shares(p, tid, t)
+            if st["n_local"]:
+                ctx.ffn_up(T)
+                ctx.truncate(cb.Z_UP)
+                for p in (0, 1):
+                    ctx.bind_shares(p, cb.H, st["dev"][p][cb.H])
+            ctx.ffn_down(T)
+            for p in (0, 1):
+                shard.add_over_ranks(y_view[p])            # the exchange: partial shares added over the ranks
+            ctx.truncate(cb.Y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for k in range(args.warmup):
+        step(k)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        sampler.wait_ready()
+    launches0 = ctx.stats().kernel_launches
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    host0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        flush.zero_()
+        e0.record(stream)
+    for k in range(args.steps):
+        step(args.warmup + k)
+    with torch.cuda.stream(stream):
+        e1.record(stream)
+    barrier()
+    clocks = sampler.region(host0, time.perf_counter()) if rank == 0 else None
+    sampler.stop()
+    (ms,) = ranks.max_over_ranks([e0.elapsed_time(e1)], dev)
+    launches = ctx.stats().kernel_launches - launches0
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": macs * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": workload_name(cfg, sparsity), "parallelism": f"neurons sharded over {world} rank(s), "
+                       "one int64 all-reduce of Y_i per party per step", "l2": "4 rotating input sets with different "
+                       "masks; 512 MiB flushed before the region", "timed": "region of exactly K steps between two "
+                       "CUDA events on the library stream, collectives included, max over ranks"},
+            "gpu_launches": int(launches), "clocks": clocks}))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # --------------------------------------------------------------------------- measured peaks of the multiply pipes
 def measure_pipe_peaks(sampler, tensor_launches=24, alu_launches=12):
     """The rate of the int8 tensor pipe (the instruction the limb kernel issues, operands resident in shared
@@ -401,6 +520,15 @@ def main():
     ap.add_argument("--op", default="ffn", choices=["ffn", "shuffle", "peak"],
                     help="ffn: the sparse FFN path (the headline); shuffle: the oblivious shuffle's online stage; "
                          "peak: the measured rates of the int8 tensor pipe and of the 64-bit ALU loop alone")
+    ap.add_argument("--mask-location", default="host", choices=["host", "device"],
+                    help="where the block mask (public, one byte per block) is when set_mask is called in the "
+                         "device-resident timing: host memory (counted on the host, no round trip) or device memory "
+                         "(the count comes back from the compaction kernel)")
+    ap.add_argument("--shard", default="problems", choices=["problems", "neurons"],
+                    help="how --gpus N > 1 divides the work: problems = every rank runs its own independent FFN "
+                         "problems (no collective, weak scaling; the default); neurons = one problem per step, its "
+                         "neurons dealt to the ranks, the down-projection's partial shares summed by an all-reduce "
+                         "(strong scaling)")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="the timed region of K steps is repeated until the device has been under load for this "
                          "long; the first (burst), median and last (sustained) region are reported")
@@ -416,6 +544,8 @@ def main():
         return run_shuffle(args, cfg)
     if args.op == "peak":
         return run_peak(args)
+    if args.shard == "neurons":
+        return run_sharded(args, cfg, sparsity)
     if args.warmup < 3:
         args.warmup = 3
 
@@ -481,6 +611,11 @@ def main():
     UP_IDS = (cb.X, cb.A_UP, cb.B_UP, cb.C_UP, cb.A_DN, cb.B_DN, cb.C_DN)
     DN_IDS = (cb.H,)
 
+    # The block mask is the public sparsity distribution (one byte per block): by default it is handed over in host
+    # memory, where the library counts it without a device round trip (its copy to the device and the compaction
+    # kernel are inside the timed region); every share, triple and weight is resident in HBM.
+    mask_key = "mask_host" if args.mask_location == "host" else "mask_dev"
+
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
@@ -491,7 +626,7 @@ def main():
             flush.zero_()                                  # evict L2 between steps
             e = [ev() for _ in range(6)]
             e[0].record(stream)
-            ctx.set_mask(st["mask_dev"])
+            ctx.set_mask(st[mask_key])
             if st["tm_dev"] is not None:
                 ctx.set_token_mask(st["tm_dev"])
             e[1].record(stream)
@@ -653,7 +788,7 @@ def main():
             cx, sk = pctx[s % C]
             st = psets[s % C][(s // C) % 2]
             with torch.cuda.stream(sk):
-                cx.set_mask(st["mask_dev"])
+                cx.set_mask(st[mask_key])
                 if st["tm_dev"] is not None:
                     cx.set_token_mask(st["tm_dev"])
                 for p in (0, 1):
@@ -851,6 +986,8 @@ def main():
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {"workload": workload_name(cfg, sparsity), "matmul_path": used_path,
                        "in_flight": args.in_flight if use_piped else 1,
+                       "block_mask": f"{cfg.n_blocks} bytes, passed from {args.mask_location} memory; all shares, "
+                                     "triples and weights resident in HBM",
                        "l2": (f"{args.in_flight} contexts x 2 input sets with different masks rotate (inputs, gathered "
                               "weight rows and intermediates of consecutive steps far exceed the L2); no flush"
                               if use_piped else

@@ -30,9 +30,10 @@
  *     exception is comet_bind_shares, which reads the caller's device memory in
  *     place).
  *   - All work is enqueued on the CUDA stream given to comet_init.  Calls are
- *     asynchronous with respect to the host except comet_set_mask (it returns
- *     the public count n), comet_get/comet_load_shares with host pointers to
- *     pageable memory, comet_stats and comet_destroy.
+ *     asynchronous with respect to the host except comet_set_mask with a DEVICE
+ *     mask and comet_set_token_mask (they return public counts computed on the
+ *     device), comet_get/comet_load_shares with host pointers to pageable
+ *     memory, comet_synchronize, comet_stats and comet_destroy.
  */
 #ifndef COMET_H_
 #define COMET_H_
@@ -181,8 +182,14 @@ int comet_bind_shares(comet_ctx* ctx, int party, int tensor_id, const uint64_t* 
  * = active) into the ascending list of active blocks, i.e. the index set I.
  * `n_blocks` must equal d_ff / block.  Returns the number of active NEURONS in
  * *n_active_out (the sparsity level is public in the threat model of Section
- * 3.2), which costs one 4-byte device-to-host copy and a stream synchronise.
- * Zero active blocks is legal.  Invalidates previously loaded triples and H. */
+ * 3.2).  With a HOST mask the library counts the active blocks itself, copies
+ * the bytes out of a pinned slot of its own (the caller's buffer may be reused
+ * at once) and returns without waiting for the device; with a DEVICE mask the
+ * count comes back from the compaction kernel through mapped host memory,
+ * which the call waits for.  Zero active blocks is legal.  Invalidates
+ * previously loaded triples and H.  Errors: INVALID_ARG, SHAPE (n_blocks; more
+ * active neurons than max_active), CUDA, TIMEOUT (an earlier kernel of the
+ * context gave up on a bounded wait). */
 int comet_set_mask(comet_ctx* ctx, const uint8_t* block_mask, int location, int32_t n_blocks,
                    int32_t* n_active_out);
 
@@ -266,6 +273,18 @@ int comet_truncate(comet_ctx* ctx, int tensor_id);
  * is returned in *written (may be NULL). */
 int comet_get(comet_ctx* ctx, int party, int tensor_id, uint64_t* out, int location, int64_t capacity,
               int64_t* written);
+
+/* Device address of the library's own buffer of a RESULT tensor (COMET_Z_UP or
+ * COMET_Y) of party `party`, valid until comet_destroy; the tensor's current
+ * contents are its first rows*cols words.  For steps that combine results in
+ * place between two calls of the path -- when the active neurons are sharded
+ * over several GPUs, every GPU's comet_ffn_down leaves a partial sum of Eq. 1
+ * in COMET_Y, the partial sums are added over the GPUs (addition of shares is
+ * local, Section 2.1 "Addition"; an integer all-reduce, which wraps mod 2^64),
+ * and comet_truncate then runs on the sum.  Whatever touches the buffer must be
+ * ordered after the producing call and before the next consuming call on the
+ * context's stream.  Errors: INVALID_ARG. */
+int comet_device_pointer(comet_ctx* ctx, int party, int tensor_id, uint64_t** out);
 
 /* The compacted index list: ascending ids of the active blocks (int32).
  * `capacity` in entries; the count goes to *n_active_blocks_out. */

@@ -32,7 +32,7 @@ EXPORTS = (
     "comet_set_profiling", "comet_beaver_matmul_static", "comet_shuffle", "comet_invert_permutation",
     "comet_beaver_mul", "comet_set_token_mask", "comet_get_components", "comet_kv_plan",
     "comet_add_bias", "comet_bind_shares", "comet_truncate_pair", "comet_synchronize", "comet_inject_timeout",
-    "comet_pipe_probe",
+    "comet_pipe_probe", "comet_device_pointer",
 )
 STATIC_SCRATCH_WORDS = 1 << 20
 ERR_SCRATCH_LIMIT = -7
@@ -91,6 +91,7 @@ def _load():
     lib.comet_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.comet_synchronize.argtypes = [vp]
     lib.comet_inject_timeout.argtypes = [vp]
+    lib.comet_device_pointer.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.comet_pipe_probe.argtypes = [vp, ctypes.c_int, i32, i32, ctypes.POINTER(ctypes.c_float),
                                      ctypes.POINTER(ctypes.c_double)]
     pair = ctypes.c_void_p * 2
@@ -234,6 +235,18 @@ class Comet:
         self.synchronize()
         assert n == out.numel(), (n, shape)
         return out.cpu().numpy().view(np.uint64).reshape(shape)
+
+    def result_view(self, party: int, tensor_id: int, shape) -> torch.Tensor:
+        """The library's own buffer of a result tensor (Z_UP or Y) as a torch int64 tensor of the given stored
+        shape, sharing memory with the library (no copy): for in-place collectives between two calls of the path."""
+        addr = ctypes.c_void_p()
+        self._check(_lib.comet_device_pointer(self._h, party, tensor_id, ctypes.byref(addr)), "comet_device_pointer")
+
+        class _View:                             # the CUDA array interface: address, shape and element type
+            __cuda_array_interface__ = {"shape": tuple(int(v) for v in shape), "typestr": "<i8",
+                                        "data": (addr.value, False), "version": 2, "strides": None}
+
+        return torch.as_tensor(_View(), device=self.device)
 
     def get_index(self) -> np.ndarray:
         nb = self.cfg.d_ff // self.cfg.block

@@ -9,6 +9,7 @@
 #include <atomic>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -48,6 +49,12 @@ struct comet_ctx {
     bool dn_right_few;                // ... and were laid out for the few-token kernel (128-row tiles)
     bool f_as_planes[2];              // the messages F_i of the last up / down product exist as planes only
     uint8_t* d_mask;
+    // a block mask given in host memory is counted on the host and copied from a pinned staging slot of the
+    // library's own, so that comet_set_mask need not wait for the device
+    uint8_t* h_mask_stage;            // pinned: kMaskSlots x n_blocks bytes
+    cudaEvent_t stage_done[4];        // recorded after the copy out of each slot
+    bool stage_used[4];
+    int stage_next;
     uint8_t* d_tmask;             // per-token mask over the active blocks, [cap_T, d_ff / block] capacity
     bool tmask_set;
     int32_t tmask_tokens;
@@ -176,6 +183,31 @@ cudaMemcpyKind copy_kind(int location, bool to_library) {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Launch of a kernel of the step's chain: programmatic stream serialisation (the kernel may begin while its
+// predecessor on the stream is finishing; it calls pdl_wait() before it touches global memory) and, for the
+// tensor-core kernels, the device's highest scheduling priority.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                           const int* priority, Args&&... args) {
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof(lc));
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.numAttrs = 1;
+    if (priority) {
+        attr[1].id = cudaLaunchAttributePriority;
+        attr[1].val.priority = *priority;
+        lc.numAttrs = 2;
+    }
+    lc.attrs = attr;
+    return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
+
 // True once a kernel of this context gave up on a bounded wait (the word is written by the kernel itself, in
 // mapped host memory, and never cleared: the context's results are not to be trusted from then on).
 inline bool timed_out(const comet_ctx* c) {
@@ -252,7 +284,8 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     if (right_tiles) c->f_as_planes[pr.down ? 1 : 0] = a.emit_f != 0;
     const size_t smem = right_tiles ? (a.emit_f ? 2 : 1) * sizeof(comet::LimbTile) : 0;
-    comet::limb_open_kernel<<<dim3(a.left_blocks + right_tiles, 2), 256, smem, stream>>>(a);
+    COMET_CUDA(c, launch_chained(comet::limb_open_kernel, dim3(2 * (a.left_blocks + right_tiles)), dim3(256), smem,
+                                 stream, nullptr, a));
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
@@ -299,7 +332,7 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
     const int blocks = a.left_tiles + a.right_tiles + a.copy_blocks;
     if (blocks == 0) return COMET_OK;
     const size_t smem = (left ? 2 : 1) * sizeof(comet::LimbTile);
-    comet::limb_prep_kernel<<<dim3(blocks, 2), 256, smem, stream>>>(a);
+    COMET_CUDA(c, launch_chained(comet::limb_prep_kernel, dim3(2 * blocks), dim3(256), smem, stream, nullptr, a));
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
@@ -352,20 +385,11 @@ int limb_combine(comet_ctx* c, const Proj& pr) {
         // The persistent kernel needs a slot on every SM.  With the device's highest scheduling priority its CTAs
         // get the slots that free up before the memory-side CTAs of other contexts queued beside it do, so the
         // tensor cores do not wait behind work that could as well run under them.
-        cudaLaunchConfig_t lc;
-        std::memset(&lc, 0, sizeof(lc));
-        lc.gridDim = dim3(grid);
-        lc.blockDim = dim3(few ? lf::THREADS : lb::THREADS);
-        lc.dynamicSmemBytes = few ? lf::SMEM_BYTES : lb::SMEM_BYTES;
-        lc.stream = c->stream;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributePriority;
-        attr.val.priority = c->top_priority;
-        lc.attrs = &attr;
-        lc.numAttrs = 1;
-        if (few) COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_few_kernel, a));
-        else if (grouped) COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_grouped_kernel, a));
-        else COMET_CUDA(c, cudaLaunchKernelEx(&lc, comet::combine_limb_kernel, a));
+        const dim3 block(few ? lf::THREADS : lb::THREADS);
+        const size_t smem = few ? lf::SMEM_BYTES : lb::SMEM_BYTES;
+        auto* kernel = few ? comet::combine_limb_few_kernel
+                           : grouped ? comet::combine_limb_grouped_kernel : comet::combine_limb_kernel;
+        COMET_CUDA(c, launch_chained(kernel, dim3(grid), block, smem, c->stream, &c->top_priority, a));
     }
     c->stats.kernel_launches += 1;
     c->stats.matmul_path = COMET_PATH_LIMB;
@@ -413,8 +437,9 @@ int somm_merge(comet_ctx* c, int tokens) {
     if (pairs == 0) return COMET_OK;
     comet::PartyOut Z;
     for (int p = 0; p < 2; ++p) Z.p[p] = c->buf[p][COMET_Z_UP];
-    comet::somm_merge_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(
-        Z, pairs, cols, c->n_active, c->cfg.block, c->d_row_label, c->d_blk_label);
+    COMET_CUDA(c, launch_chained(comet::somm_merge_kernel, dim3(ew_grid(c, pairs, 256), 2), dim3(256), 0, c->stream,
+                                 nullptr, Z, pairs, cols, (int)c->n_active, (int)c->cfg.block,
+                                 (const int32_t*)c->d_row_label, (const int32_t*)c->d_blk_label));
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
@@ -539,6 +564,9 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     const int nb = cfg->d_ff / cfg->block;
     ok = ok && cudaMalloc((void**)&c->d_mask, (size_t)nb) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_tmask, (size_t)nb * (size_t)c->cap_T) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->h_mask_stage, (size_t)nb * 4, cudaHostAllocDefault) == cudaSuccess;
+    for (int k = 0; k < 4 && ok; ++k)
+        ok = cudaEventCreateWithFlags(&c->stage_done[k], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc((void**)&c->h_masked, 7 * sizeof(long long), cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_row_map, (size_t)c->cap_T * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->d_col_map, (size_t)c->groups * nb * sizeof(int32_t)) == cudaSuccess;
@@ -588,6 +616,9 @@ void comet_destroy(comet_ctx* c) {
     if (c->side) cudaStreamDestroy(c->side);
     if (c->d_mask) cudaFree(c->d_mask);
     if (c->d_tmask) cudaFree(c->d_tmask);
+    if (c->h_mask_stage) cudaFreeHost(c->h_mask_stage);
+    for (int k = 0; k < 4; ++k)
+        if (c->stage_done[k]) cudaEventDestroy(c->stage_done[k]);
     if (c->h_masked) cudaFreeHost(c->h_masked);
     if (c->d_row_label) cudaFree(c->d_row_label);
     if (c->d_row_map) cudaFree(c->d_row_map);
@@ -667,8 +698,20 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     }
     c->dn_right_ready = false;
     const uint8_t* dmask = block_mask;         // a device mask is read in place
+    int32_t host_count = -1;                   // number of active blocks when the host could count them itself
     if (location == COMET_HOST) {
-        COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, block_mask, (size_t)n_blocks, cudaMemcpyHostToDevice, c->stream));
+        // The count is public (Section 3.2) and the mask is in host memory: count here, hand the bytes to the copy
+        // engine from a pinned slot of our own (the caller's buffer is free again on return) and do not wait.
+        const int slot = c->stage_next;
+        c->stage_next = (slot + 1) % 4;
+        if (c->stage_used[slot]) COMET_CUDA(c, cudaEventSynchronize(c->stage_done[slot]));
+        uint8_t* stage = c->h_mask_stage + (size_t)slot * n_blocks;
+        std::memcpy(stage, block_mask, (size_t)n_blocks);
+        host_count = 0;
+        for (int32_t b = 0; b < n_blocks; ++b) host_count += stage[b] != 0;
+        COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, stage, (size_t)n_blocks, cudaMemcpyHostToDevice, c->stream));
+        COMET_CUDA(c, cudaEventRecord(c->stage_done[slot], c->stream));
+        c->stage_used[slot] = true;
         dmask = c->d_mask;
     }
     {
@@ -680,7 +723,7 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     }
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
-    {
+    if (host_count < 0) {
         // The kernel is the last thing on the stream and reports through mapped memory: watching its ticket for
         // a short while is quicker than a stream synchronise; after that, synchronise as usual.
         volatile int32_t* seen = c->h_count + 2;
@@ -693,7 +736,7 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
         std::atomic_thread_fence(std::memory_order_acquire);
     }
     if (timed_out(c)) return COMET_ERR_TIMEOUT;           // an earlier kernel gave up on a bounded wait
-    const int32_t blocks = *c->h_count;
+    const int32_t blocks = host_count >= 0 ? host_count : *c->h_count;
     const int64_t n = (int64_t)blocks * c->cfg.block;
     if (n > c->cap_n) {            // more active neurons than the context was sized for
         c->mask_set = false;
@@ -816,13 +859,10 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
             rc = limb_open(c, up, true, true, c->stream);
         }
         if (rc != COMET_OK) return rc;
-        {
-            PhaseTimer timer(c, COMET_PHASE_PREP, 1);
-            rc = limb_prep(c, up, true, true, true, c->stream);
-        }
-        if (rc != COMET_OK) return rc;
         // The weight side of the down-projection depends only on the mask, W2 and B'_i: if those are loaded
-        // already, open it now on the side stream, under the tensor-core kernel that follows.
+        // already, open it now on the side stream, beside the preparation and the tensor-core kernel that follow.
+        // (The fork sits before the preparation kernel so that nothing separates that kernel from the tensor-core
+        // kernel on the main stream: the latter is launched as the former's programmatic dependent.)
         const bool early = !c->dn_right_ready && limb_fits(c, dn) && c->loaded[0][COMET_W2] &&
                            c->loaded[1][COMET_W2] && c->loaded[0][COMET_B_DN] && c->loaded[1][COMET_B_DN];
         if (early) {
@@ -836,6 +876,11 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
             c->dn_right_ready = true;
             c->dn_right_few = limb_few(dn);
         }
+        {
+            PhaseTimer timer(c, COMET_PHASE_PREP, 1);
+            rc = limb_prep(c, up, true, true, true, c->stream);
+        }
+        if (rc != COMET_OK) return rc;
         rc = limb_combine(c, up);
         if (rc != COMET_OK) return rc;
         return somm_merge(c, tokens);
@@ -955,7 +1000,8 @@ int comet_truncate(comet_ctx* c, int tensor_id) {
     for (int p = 0; p < 2; ++p) Z.p[p] = c->buf[p][tensor_id];
     {
         PhaseTimer timer(c, COMET_PHASE_TRUNCATE, 1);
-        comet::truncate_kernel<<<dim3(ew_grid(c, pairs, 256), 2), 256, 0, c->stream>>>(Z, pairs, c->cfg.frac_bits);
+        COMET_CUDA(c, launch_chained(comet::truncate_kernel, dim3(ew_grid(c, pairs, 256), 2), dim3(256), 0, c->stream,
+                                     nullptr, Z, pairs, (int)c->cfg.frac_bits));
     }
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
@@ -1012,6 +1058,13 @@ int comet_inject_timeout(comet_ctx* c) {
     const int32_t one = 1;
     COMET_CUDA(c, cudaMemcpy(c->d_error, &one, sizeof(one), cudaMemcpyHostToDevice));
     c->h_count[3] = 1;
+    return COMET_OK;
+}
+
+int comet_device_pointer(comet_ctx* c, int party, int tensor_id, uint64_t** out) {
+    if (!c || !out || (party != 0 && party != 1)) return COMET_ERR_INVALID_ARG;
+    if (tensor_id != COMET_Z_UP && tensor_id != COMET_Y) return COMET_ERR_INVALID_ARG;
+    *out = reinterpret_cast<uint64_t*>(c->own[party][tensor_id]);
     return COMET_OK;
 }
 

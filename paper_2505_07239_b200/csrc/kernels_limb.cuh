@@ -23,6 +23,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "pdl.cuh"
+
 namespace comet {
 
 typedef unsigned long long u64;
@@ -105,8 +107,9 @@ __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows,
 //                 own B_i (it is in registers anyway, so it is not read a second time later).
 // gather: up   (down = 0): row c of the right operand is row neuron(c) of W (whole rows of `ldw` words);
 //         down (down = 1): contraction index c is column neuron(c) of W (strips of `bs` words in every row).
-// grid = (left_blocks + kblocks * ceil(rows / 64), party), 256 threads; dynamic shared memory: one LimbTile when
-// there are right tiles, two with emit_f.
+// grid = 2 * (left_blocks + kblocks * ceil(rows / 64)), 256 threads, the party being the lowest bit of the block
+// index (both parties' messages are then written in the same order, which the next kernel reads backwards);
+// dynamic shared memory: one LimbTile when there are right tiles, two with emit_f.
 // ---------------------------------------------------------------------------
 struct LimbOpenArgs {
     const u64* X[2];
@@ -153,14 +156,17 @@ struct LimbOpenArgs {
 __global__ void __launch_bounds__(256)
 limb_open_kernel(LimbOpenArgs a) {
     using namespace limb;
-    const int party = blockIdx.y;
+    pdl_wait();
+    pdl_launch_dependents();
+    const int party = blockIdx.x & 1;
+    const int bid = blockIdx.x >> 1;
     const int tid = threadIdx.x;
-    if ((int)blockIdx.x < a.left_blocks) {
+    if (bid < a.left_blocks) {
         const ulonglong2* __restrict__ x = reinterpret_cast<const ulonglong2*>(party ? a.X[1] : a.X[0]);
         const ulonglong2* __restrict__ m = reinterpret_cast<const ulonglong2*>(party ? a.A[1] : a.A[0]);
         ulonglong2* __restrict__ e = reinterpret_cast<ulonglong2*>(party ? a.E[1] : a.E[0]);
         const long long stride = (long long)a.left_blocks * 256;
-        for (long long t = (long long)blockIdx.x * 256 + tid; t < a.left_pairs; t += stride) {
+        for (long long t = (long long)bid * 256 + tid; t < a.left_pairs; t += stride) {
             if (a.tmask) {
                 const unsigned word = (unsigned)(2 * t), row = word / (unsigned)a.K, col = word - row * (unsigned)a.K;
                 if (a.tmask[(size_t)row * a.tmask_ld + col / (unsigned)a.bs] == 0) {
@@ -172,7 +178,7 @@ limb_open_kernel(LimbOpenArgs a) {
                 e[t] = make_ulonglong2(0ull, 0ull);
                 continue;
             }
-            const ulonglong2 xv = __ldg(x + t), av = __ldg(m + t);
+            const ulonglong2 xv = __ldcs(x + t), av = __ldcs(m + t);      // read once: leave L2 to what is written
             e[t] = make_ulonglong2(xv.x - av.x, xv.y - av.y);
         }
         return;
@@ -180,7 +186,7 @@ limb_open_kernel(LimbOpenArgs a) {
     extern __shared__ __align__(16) uint8_t open_smem[];
     LimbTile& sB = *reinterpret_cast<LimbTile*>(open_smem);
     LimbTile& sF = *reinterpret_cast<LimbTile*>(open_smem + sizeof(LimbTile));      // only with emit_f
-    const int tile_id = blockIdx.x - a.left_blocks;
+    const int tile_id = bid - a.left_blocks;
     const int kb = tile_id % a.kblocks;
     const int row0 = (tile_id / a.kblocks) * PREP_ROWS;
     const u64* __restrict__ Bi = party ? a.B[1] : a.B[0];
@@ -219,8 +225,10 @@ limb_open_kernel(LimbOpenArgs a) {
                            (size_t)neuron * a.ldw + k;
                 }
                 const size_t o = (size_t)row * a.K + ks;
-                const ulonglong2 w = __ldg(reinterpret_cast<const ulonglong2*>(wsrc));
-                const ulonglong2 b = __ldg(reinterpret_cast<const ulonglong2*>(Bi + o));
+                // shares and triples are read once per product: streaming loads, so that the messages and planes
+                // written here are still in L2 when the next kernel reads them
+                const ulonglong2 w = __ldcs(reinterpret_cast<const ulonglong2*>(wsrc));
+                const ulonglong2 b = __ldcs(reinterpret_cast<const ulonglong2*>(Bi + o));
                 f0 = dead ? 0ull : w.x - b.x;
                 f1 = dead ? 0ull : w.y - b.y;
                 if (!a.emit_f) *reinterpret_cast<ulonglong2*>(Fi + o) = make_ulonglong2(f0, f1);
@@ -267,7 +275,10 @@ limb_planes_to_words_kernel(const uint8_t* __restrict__ planes, u64* __restrict_
 //   left tiles : E = E_0 + E_1 -> planes(E);  V_i = A_i + i*E -> planes(V_i)      [M, K], 128-row blocks
 //   right tiles: F = F_0 + F_1 -> planes(F)                                      [N, K],  64-row blocks
 //   copy blocks: Z_i <- C_i (the accumulation target starts from the triple's C share)
-// grid = (kblocks * (ceil(M/64) + ceil(N/64)) + copy_blocks, party), 256 threads.  Any part may be empty.
+// grid = 2 * (kblocks * (ceil(M/64) + ceil(N/64)) + copy_blocks), 256 threads.  Any part may be empty.
+// The party is the lowest bit of the block index: the two parties' CTAs of one tile read the same two messages and
+// run side by side, so the second read comes from L2.  Tiles are taken from the last to the first: the kernel before
+// this one wrote the messages in ascending order, and its last tiles are the ones most likely still in L2.
 // ---------------------------------------------------------------------------
 struct LimbPrepArgs {
     const u64* E0; const u64* E1;
@@ -298,15 +309,19 @@ struct LimbPrepArgs {
 __global__ void __launch_bounds__(256)
 limb_prep_kernel(LimbPrepArgs a) {
     using namespace limb;
-    const int party = blockIdx.y;
+    pdl_wait();
+    pdl_launch_dependents();
+    const int party = blockIdx.x & 1;
     const int tid = threadIdx.x;
-    int id = blockIdx.x;
-    if (id >= a.left_tiles + a.right_tiles) {
+    int id = blockIdx.x >> 1;
+    if (id < a.left_tiles + a.right_tiles) {
+        id = a.left_tiles + a.right_tiles - 1 - id;
+    } else {
         id -= a.left_tiles + a.right_tiles;
         const ulonglong2* __restrict__ s = reinterpret_cast<const ulonglong2*>(party ? a.C[1] : a.C[0]);
         ulonglong2* __restrict__ d = reinterpret_cast<ulonglong2*>(party ? a.Z[1] : a.Z[0]);
         const long long stride = (long long)a.copy_blocks * 256;
-        for (long long t = (long long)id * 256 + tid; t < a.copy_pairs; t += stride) d[t] = __ldg(s + t);
+        for (long long t = (long long)id * 256 + tid; t < a.copy_pairs; t += stride) d[t] = __ldcs(s + t);
         return;
     }
     extern __shared__ __align__(16) uint8_t prep_smem[];     // one tile (right/copy only) or two (left present)
@@ -341,12 +356,13 @@ limb_prep_kernel(LimbPrepArgs a) {
                     row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
                 }
                 const size_t o = (size_t)row * a.K + ks;
-                const ulonglong2 x = __ldg(reinterpret_cast<const ulonglong2*>(in0 + o));
-                const ulonglong2 y = __ldg(reinterpret_cast<const ulonglong2*>(in1 + o));
+                // the messages were written by the kernel before this one and are not read again on the path
+                const ulonglong2 x = __ldcs(reinterpret_cast<const ulonglong2*>(in0 + o));
+                const ulonglong2 y = __ldcs(reinterpret_cast<const ulonglong2*>(in1 + o));
                 s0 = x.x + y.x;                       // the exchange: both messages summed
                 s1 = x.y + y.y;
                 if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + ks / a.bs] != 0)) {
-                    const ulonglong2 z = __ldg(reinterpret_cast<const ulonglong2*>(own + o));
+                    const ulonglong2 z = __ldcs(reinterpret_cast<const ulonglong2*>(own + o));
                     w0 = z.x + (party ? s0 : 0ull);   // V_i = A_i + i*E
                     w1 = z.y + (party ? s1 : 0ull);
                 }
@@ -782,6 +798,18 @@ __device__ __forceinline__ bool limb_wait_warp(uint32_t bar, uint32_t parity, vo
     return __all_sync(0xffffffffu, ok);
 }
 
+// Z = sum_s 2^(8s) D_s mod 2^64 from the eight 32-bit accumulators of one output element: the terms with s <= 3 are
+// 32 x 32 -> 64-bit multiply-adds by 2^(8s), the terms with s >= 4 only reach the high word (32-bit shifts and adds).
+__device__ __forceinline__ u64 limb_recombine(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t d3, uint32_t d4,
+                                              uint32_t d5, uint32_t d6, uint32_t d7) {
+    u64 v = (u64)d0;
+    v += (u64)d1 * (u64)(1u << 8);
+    v += (u64)d2 * (u64)(1u << 16);
+    v += (u64)d3 * (u64)(1u << 24);
+    const uint32_t hi = (uint32_t)(v >> 32) + d4 + (d5 << 8) + (d6 << 16) + (d7 << 24);
+    return ((u64)hi << 32) | (u64)(uint32_t)v;
+}
+
 // One contiguous piece of a CTA's share of the (party, tile, k-block) space: a run of k-blocks of one tile.
 struct LimbSegment {
     int party, tm, tn;
@@ -872,6 +900,8 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
     __syncthreads();
     ptx::fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
+    // barriers and tensor memory are set up; from here on the kernel touches what its predecessors wrote
+    pdl_wait();
 
     if (warp == EPI_WARPS) {
         // ---------------- producer: one bulk copy per operand block ----------------
@@ -977,6 +1007,8 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                 ptx::mma_commit(accum_full);
                 acc_phase ^= 1u;
             }
+            // the main loop is over: the next kernel of the stream may be brought in beside the last drain
+            pdl_launch_dependents();
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> recombine mod 2^64 -> release TMEM ->
@@ -1011,12 +1043,10 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                     ptx::tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 8; j += 2) {
-                        u64 v0 = (u64)d[0][j], v1 = (u64)d[0][j + 1];
-#pragma unroll
-                        for (int s = 1; s < PLANES; ++s) {
-                            v0 += (u64)d[s][j] << (8 * s);
-                            v1 += (u64)d[s][j + 1] << (8 * s);
-                        }
+                        const u64 v0 = limb_recombine(d[0][j], d[1][j], d[2][j], d[3][j], d[4][j], d[5][j], d[6][j],
+                                                      d[7][j]);
+                        const u64 v1 = limb_recombine(d[0][j + 1], d[1][j + 1], d[2][j + 1], d[3][j + 1], d[4][j + 1],
+                                                      d[5][j + 1], d[6][j + 1], d[7][j + 1]);
                         *reinterpret_cast<ulonglong2*>(my_row + (c * 8 + j) * 8) = make_ulonglong2(v0, v1);
                     }
                 }
@@ -1160,6 +1190,8 @@ combine_limb_few_kernel(LimbArgs a) {
     __syncthreads();
     ptx::fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
+    // barriers and tensor memory are set up; from here on the kernel touches what its predecessors wrote
+    pdl_wait();
 
     if (warp == EPI_WARPS) {
         // ---------------- producer: one bulk copy per operand block ----------------
@@ -1247,6 +1279,8 @@ combine_limb_few_kernel(LimbArgs a) {
                 ptx::mma_commit(accum_full);
                 acc_phase ^= 1u;
             }
+            // the main loop is over: the next kernel of the stream may be brought in beside the last drain
+            pdl_launch_dependents();
         }
     } else {
         // ---------------- epilogue: lane = neuron, registers = tokens; transpose through shared memory ----------------
@@ -1269,12 +1303,8 @@ combine_limb_few_kernel(LimbArgs a) {
                 for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BT * s + c * 8, d[s]);
                 ptx::tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    u64 v = (u64)d[0][j];
-#pragma unroll
-                    for (int s = 1; s < PLANES; ++s) v += (u64)d[s][j] << (8 * s);
-                    z[c * 8 + j] = v;
-                }
+                for (int j = 0; j < 8; ++j)
+                    z[c * 8 + j] = limb_recombine(d[0][j], d[1][j], d[2][j], d[3][j], d[4][j], d[5][j], d[6][j], d[7][j]);
             }
             ptx::fence_before_sync();
             ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));

@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "pdl.cuh"
+
 namespace comet {
 
 typedef unsigned long long u64;
@@ -105,6 +107,8 @@ open_activation_kernel(PartyPtrs X, PartyPtrs A, PartyOut E, int64_t pairs, cons
 __global__ void __launch_bounds__(256)
 somm_merge_kernel(PartyOut Z, int64_t pairs, int cols, int n, int bs, const int32_t* __restrict__ row_label,
                   const int32_t* __restrict__ blk_label) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int party = blockIdx.y;
     ulonglong2* __restrict__ z = reinterpret_cast<ulonglong2*>((party ? Z.p[1] : Z.p[0]));
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -190,6 +194,8 @@ __device__ __forceinline__ u64 trunc_word(u64 s, int f, int party) {
 
 __global__ void __launch_bounds__(256)
 truncate_kernel(PartyOut Z, int64_t pairs, int f) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int party = blockIdx.y;
     ulonglong2* __restrict__ z = reinterpret_cast<ulonglong2*>((party ? Z.p[1] : Z.p[0]));
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
