@@ -201,42 +201,51 @@ limb_open_kernel(LimbOpenArgs a) {
         }
         // down: the strip of W that holds compact contraction indices ks, ks+1
         const int kcol = a.down && k < a.K ? a.ids[ks / a.bs] * a.bs + (ks % a.bs) : 0;
+        // First every load of this thread's four rows is issued (eight 16-byte requests in flight per thread), then
+        // the words are used: the kernel is bound by memory latency otherwise.  Shares and triples are read once per
+        // product: streaming loads, so that the messages and planes written here are still in L2 when the next
+        // kernel reads them.
+        constexpr int ITERS = PREP_ROWS / 16;
+        ulonglong2 w[ITERS], b[ITERS];
+        size_t off[ITERS];
+        bool live[ITERS], dead[ITERS];
 #pragma unroll
-        for (int it = 0; it < PREP_ROWS / 16; ++it) {
-            const int r = it * 16 + (tid >> 4);
-            int row = row0 + r;
-            u64 b0 = 0, b1 = 0, f0 = 0, f1 = 0;
-            if (row < a.rows && k < a.K) {
+        for (int it = 0; it < ITERS; ++it) {
+            int row = row0 + it * 16 + (tid >> 4);
+            live[it] = row < a.rows && k < a.K;
+            dead[it] = false;
+            w[it] = b[it] = make_ulonglong2(0ull, 0ull);
+            off[it] = 0;
+            if (live[it]) {
                 const u64* wsrc;
-                bool dead = false;
                 if (a.col_map) {
                     const int sb = row / a.bs;
                     row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
                 }
                 if (a.down) {
-                    dead = a.blk_label && a.blk_label[ks / a.bs] < 0;     // a block without a non-zero column of X
+                    dead[it] = a.blk_label && a.blk_label[ks / a.bs] < 0;     // a block without a non-zero column of X
                     wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
                 } else {
                     const int grp = row / a.n, j = row - grp * a.n;
                     const int neuron = a.ids[j / a.bs] * a.bs + (j % a.bs);
-                    dead = a.blk_label && a.blk_label[j / a.bs] < 0;
+                    dead[it] = a.blk_label && a.blk_label[j / a.bs] < 0;
                     wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0])
                                      : grp == 1 ? (party ? a.W1[1] : a.W1[0]) : (party ? a.W2g[1] : a.W2g[0])) +
                            (size_t)neuron * a.ldw + k;
                 }
-                const size_t o = (size_t)row * a.K + ks;
-                // shares and triples are read once per product: streaming loads, so that the messages and planes
-                // written here are still in L2 when the next kernel reads them
-                const ulonglong2 w = __ldcs(reinterpret_cast<const ulonglong2*>(wsrc));
-                const ulonglong2 b = __ldcs(reinterpret_cast<const ulonglong2*>(Bi + o));
-                f0 = dead ? 0ull : w.x - b.x;
-                f1 = dead ? 0ull : w.y - b.y;
-                if (!a.emit_f) *reinterpret_cast<ulonglong2*>(Fi + o) = make_ulonglong2(f0, f1);
-                b0 = b.x;
-                b1 = b.y;
+                off[it] = (size_t)row * a.K + ks;
+                w[it] = __ldcs(reinterpret_cast<const ulonglong2*>(wsrc));
+                b[it] = __ldcs(reinterpret_cast<const ulonglong2*>(Bi + off[it]));
             }
-            sB[r][kk] = b0;
-            sB[r][kk + 1] = b1;
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int r = it * 16 + (tid >> 4);
+            const u64 f0 = dead[it] ? 0ull : w[it].x - b[it].x;
+            const u64 f1 = dead[it] ? 0ull : w[it].y - b[it].y;
+            if (live[it] && !a.emit_f) *reinterpret_cast<ulonglong2*>(Fi + off[it]) = make_ulonglong2(f0, f1);
+            sB[r][kk] = b[it].x;
+            sB[r][kk + 1] = b[it].y;
             if (a.emit_f) {
                 sF[r][kk] = f0;
                 sF[r][kk + 1] = f1;
@@ -343,11 +352,15 @@ limb_prep_kernel(LimbPrepArgs a) {
             const int sb = k / a.bs;
             ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
         }
+        // every load of this thread's four rows first (up to twelve 16-byte requests in flight), then the sums
+        constexpr int ITERS = PREP_ROWS / 16;
+        ulonglong2 x[ITERS], y[ITERS], z[ITERS];
+        bool own_part[ITERS];                         // the party's A_i takes part at this position
 #pragma unroll
-        for (int it = 0; it < PREP_ROWS / 16; ++it) {
-            const int r = it * 16 + (tid >> 4);
-            int row = row0 + r;
-            u64 s0 = 0, s1 = 0, w0 = 0, w1 = 0;
+        for (int it = 0; it < ITERS; ++it) {
+            int row = row0 + it * 16 + (tid >> 4);
+            x[it] = y[it] = z[it] = make_ulonglong2(0ull, 0ull);
+            own_part[it] = false;
             if (row < rows && k < a.K) {
                 if (left) {
                     if (a.row_map) row = __ldg(a.row_map + row);
@@ -357,21 +370,24 @@ limb_prep_kernel(LimbPrepArgs a) {
                 }
                 const size_t o = (size_t)row * a.K + ks;
                 // the messages were written by the kernel before this one and are not read again on the path
-                const ulonglong2 x = __ldcs(reinterpret_cast<const ulonglong2*>(in0 + o));
-                const ulonglong2 y = __ldcs(reinterpret_cast<const ulonglong2*>(in1 + o));
-                s0 = x.x + y.x;                       // the exchange: both messages summed
-                s1 = x.y + y.y;
+                x[it] = __ldcs(reinterpret_cast<const ulonglong2*>(in0 + o));
+                y[it] = __ldcs(reinterpret_cast<const ulonglong2*>(in1 + o));
+                // where the per-token mask is zero the party's A_i is no part of the triple and counts as zero
                 if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + ks / a.bs] != 0)) {
-                    const ulonglong2 z = __ldcs(reinterpret_cast<const ulonglong2*>(own + o));
-                    w0 = z.x + (party ? s0 : 0ull);   // V_i = A_i + i*E
-                    w1 = z.y + (party ? s1 : 0ull);
+                    own_part[it] = true;
+                    z[it] = __ldcs(reinterpret_cast<const ulonglong2*>(own + o));
                 }
             }
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int r = it * 16 + (tid >> 4);
+            const u64 s0 = x[it].x + y[it].x, s1 = x[it].y + y[it].y;      // the exchange: both messages summed
             sS[r][kk] = s0;
             sS[r][kk + 1] = s1;
             if (left) {
-                sW[r][kk] = w0;
-                sW[r][kk + 1] = w1;
+                sW[r][kk] = own_part[it] ? z[it].x + (party ? s0 : 0ull) : 0ull;       // V_i = A_i + i*E
+                sW[r][kk + 1] = own_part[it] ? z[it].y + (party ? s1 : 0ull) : 0ull;
             }
         }
     }
