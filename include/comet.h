@@ -199,7 +199,13 @@ int comet_set_mask(comet_ctx* ctx, const uint8_t* block_mask, int location, int3
  * transpose), then after the exchange Z_i = C_i + E B_i + A_i F + i E F over the
  * active columns only, at scale 2f.  Needs X, W1 (and WG), A_UP, B_UP, C_UP.
  * Result in COMET_Z_UP; messages in COMET_E_UP / COMET_F_UP.  With n = 0 it does
- * nothing. */
+ * nothing.
+ * On the tensor-core path the call also starts on the down-projection with what
+ * is loaded already: with W2 and B_DN it opens that product's weight side
+ * (COMET_F_DN), and with C_DN as well it copies C'_i into COMET_Y, the value the
+ * down-projection's sums are added to.  So from this call on COMET_F_DN and
+ * COMET_Y no longer hold the previous step's values: read those back (or enqueue
+ * the comet_get) before the next comet_ffn_up. */
 int comet_ffn_up(comet_ctx* ctx, int32_t tokens);
 
 /* Protocols 2 and 3 in general: the sparsity distribution may differ from token to

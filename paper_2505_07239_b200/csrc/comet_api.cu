@@ -47,6 +47,8 @@ struct comet_ctx {
     bool side_pending;                // ev_join not yet waited for on the main stream
     bool dn_right_ready;              // F'_i and the right planes of the down-projection are current
     bool dn_right_few;                // ... and were laid out for the few-token kernel (128-row tiles)
+    bool dn_copy_ready;               // Y_i already holds C'_i (copied beside the up-projection)
+    int32_t dn_copy_tokens;           // ... for this many token rows
     bool f_as_planes[2];              // the messages F_i of the last up / down product exist as planes only
     uint8_t* d_mask;
     // a block mask given in host memory is counted on the host and copied from a pinned staging slot of the
@@ -661,10 +663,11 @@ static int set_shares(comet_ctx* c, int party, int tensor_id, const uint64_t* pt
     tensor_shape(c, tensor_id, rows, &er, &ec);
     if (rows != er || cols != ec) return COMET_ERR_SHAPE;
     if (rows * cols > c->cap_words[tensor_id]) return COMET_ERR_SHAPE;
-    if (tensor_id == COMET_W2 || tensor_id == COMET_B_DN) {
+    if (tensor_id == COMET_W2 || tensor_id == COMET_B_DN || tensor_id == COMET_C_DN) {
         const int rc = join_side(c);       // the side stream may still be reading the old contents
         if (rc != COMET_OK) return rc;
-        c->dn_right_ready = false;
+        if (tensor_id == COMET_C_DN) c->dn_copy_ready = false;
+        else c->dn_right_ready = false;
     }
     if (bind && rows * cols > 0) {
         c->buf[party][tensor_id] = const_cast<u64*>(reinterpret_cast<const u64*>(ptr));   // only ever read
@@ -699,27 +702,40 @@ int comet_set_mask(comet_ctx* c, const uint8_t* block_mask, int location, int32_
     c->dn_right_ready = false;
     const uint8_t* dmask = block_mask;         // a device mask is read in place
     int32_t host_count = -1;                   // number of active blocks when the host could count them itself
+    bool launched = false;
     if (location == COMET_HOST) {
-        // The count is public (Section 3.2) and the mask is in host memory: count here, hand the bytes to the copy
-        // engine from a pinned slot of our own (the caller's buffer is free again on return) and do not wait.
-        const int slot = c->stage_next;
-        c->stage_next = (slot + 1) % 4;
-        if (c->stage_used[slot]) COMET_CUDA(c, cudaEventSynchronize(c->stage_done[slot]));
-        uint8_t* stage = c->h_mask_stage + (size_t)slot * n_blocks;
-        std::memcpy(stage, block_mask, (size_t)n_blocks);
+        // The count is public (Section 3.2) and the mask is in host memory: count here and do not wait for the
+        // device.  A mask that fits into a kernel's parameter block travels with the launch; a larger one is handed
+        // to the copy engine from a pinned slot of our own (the caller's buffer is free again on return either way).
         host_count = 0;
-        for (int32_t b = 0; b < n_blocks; ++b) host_count += stage[b] != 0;
-        COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, stage, (size_t)n_blocks, cudaMemcpyHostToDevice, c->stream));
-        COMET_CUDA(c, cudaEventRecord(c->stage_done[slot], c->stream));
-        c->stage_used[slot] = true;
-        dmask = c->d_mask;
+        for (int32_t b = 0; b < n_blocks; ++b) host_count += block_mask[b] != 0;
+        if (n_blocks <= comet::MaskBytes::CAPACITY) {
+            comet::MaskBytes arg;
+            std::memcpy(arg.bytes, block_mask, (size_t)n_blocks);
+            PhaseTimer timer(c, COMET_PHASE_COMPACT, 1);
+            c->ticket += 1;
+            COMET_CUDA(c, launch_chained(comet::compact_mask_arg_kernel, dim3(1), dim3(1024), 0, c->stream, nullptr, arg,
+                                         (int)n_blocks, c->d_ids, c->d_count, (int32_t*)nullptr, c->ticket));
+            launched = true;
+        } else {
+            const int slot = c->stage_next;
+            c->stage_next = (slot + 1) % 4;
+            if (c->stage_used[slot]) COMET_CUDA(c, cudaEventSynchronize(c->stage_done[slot]));
+            uint8_t* stage = c->h_mask_stage + (size_t)slot * n_blocks;
+            std::memcpy(stage, block_mask, (size_t)n_blocks);
+            COMET_CUDA(c, cudaMemcpyAsync(c->d_mask, stage, (size_t)n_blocks, cudaMemcpyHostToDevice, c->stream));
+            COMET_CUDA(c, cudaEventRecord(c->stage_done[slot], c->stream));
+            c->stage_used[slot] = true;
+            dmask = c->d_mask;
+        }
     }
-    {
+    if (!launched) {
         PhaseTimer timer(c, COMET_PHASE_COMPACT, 1);
         // the kernel reports {count, error flag} straight into mapped host memory: no copy to enqueue
         c->ticket += 1;
-        comet::compact_mask_kernel<<<1, 1024, 0, c->stream>>>(dmask, n_blocks, c->d_ids, c->d_count, c->h_count_dev,
-                                                              c->ticket);
+        COMET_CUDA(c, launch_chained(comet::compact_mask_kernel, dim3(1), dim3(1024), 0, c->stream, nullptr, dmask,
+                                     (int)n_blocks, c->d_ids, c->d_count, host_count < 0 ? c->h_count_dev : (int32_t*)nullptr,
+                                     c->ticket));
     }
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
@@ -868,13 +884,18 @@ int comet_ffn_up(comet_ctx* c, int32_t tokens) {
         if (early) {
             COMET_CUDA(c, cudaEventRecord(c->ev_fork, c->stream));
             COMET_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+            // ... and if the triple's C' share is there too, Y_i <- C'_i, the value the down-projection's sums are
+            // added to, is copied in the same launch
+            const bool copy = c->loaded[0][COMET_C_DN] && c->loaded[1][COMET_C_DN];
             rc = limb_open(c, dn, false, true, c->side);
-            if (rc == COMET_OK) rc = limb_prep(c, dn, false, true, false, c->side);
+            if (rc == COMET_OK) rc = limb_prep(c, dn, false, true, copy, c->side);
             if (rc != COMET_OK) return rc;
             COMET_CUDA(c, cudaEventRecord(c->ev_join, c->side));
             c->side_pending = true;
             c->dn_right_ready = true;
             c->dn_right_few = limb_few(dn);
+            c->dn_copy_ready = copy;
+            c->dn_copy_tokens = tokens;
         }
         {
             PhaseTimer timer(c, COMET_PHASE_PREP, 1);
@@ -948,6 +969,7 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
         if (!limb_fits(c, dn)) return COMET_ERR_SHAPE;
         // opened early, during the up-projection, and in the plane layout this token count needs
         const bool have_right = c->dn_right_ready && c->dn_right_few == limb_few(dn);
+        const bool have_copy = c->dn_right_ready && c->dn_copy_ready && c->dn_copy_tokens == tokens;
         int rc = join_side(c);
         if (rc != COMET_OK) return rc;
         {
@@ -957,10 +979,11 @@ int comet_ffn_down(comet_ctx* c, int32_t tokens) {
         if (rc != COMET_OK) return rc;
         {
             PhaseTimer timer(c, COMET_PHASE_PREP, 1);
-            rc = limb_prep(c, dn, true, !have_right, true, c->stream);
+            rc = limb_prep(c, dn, true, !have_right, !have_copy, c->stream);
         }
         if (rc != COMET_OK) return rc;
         c->dn_right_ready = false;                     // a triple serves one product
+        c->dn_copy_ready = false;
         return limb_combine(c, dn);
     }
 

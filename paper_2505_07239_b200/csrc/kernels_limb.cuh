@@ -95,7 +95,7 @@ __device__ __forceinline__ void limb_emit_planes(const LimbTile& src, int r, int
 
 __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows, int row, int kblocks, int kb,
                                                    int* rin) {
-    const int tile = row / tile_rows;
+    const int tile = row >> (31 - __clz(tile_rows));          // tile_rows is 32, 64 or 128
     *rin = row - tile * tile_rows;
     return base + ((size_t)tile * kblocks + kb) * (size_t)(limb::PLANES * tile_rows * limb::KC);
 }
@@ -191,6 +191,40 @@ limb_open_kernel(LimbOpenArgs a) {
     const int row0 = (tile_id / a.kblocks) * PREP_ROWS;
     const u64* __restrict__ Bi = party ? a.B[1] : a.B[0];
     u64* __restrict__ Fi = party ? a.F[1] : a.F[0];
+    // What depends on the row alone (which row of which weight matrix is gathered, where the row lies in B_i / F_i,
+    // whether its block is in use) is worked out once per row, by one thread, and shared: the index arithmetic
+    // would otherwise be repeated by the sixteen threads of every row and make the kernel instruction-bound.
+    __shared__ const u64* s_wrow[PREP_ROWS];          // first word of the gathered row of W_i; null: no such row
+    __shared__ long long s_orow[PREP_ROWS];           // offset of the row in B_i and F_i
+    __shared__ unsigned char s_dead[PREP_ROWS];
+    if (tid < PREP_ROWS) {
+        int row = row0 + tid;
+        const u64* wp = nullptr;
+        long long o = 0;
+        bool dead = false;
+        if (row < a.rows) {
+            if (a.col_map) {
+                const int sb = row / a.bs;
+                row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
+            }
+            if (a.down) {
+                wp = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw;
+            } else {
+                const int grp = (row >= a.n) + (row >= 2 * a.n), j = row - grp * a.n;
+                const int blk = j / a.bs;
+                const int neuron = __ldg(a.ids + blk) * a.bs + (j - blk * a.bs);
+                dead = a.blk_label && a.blk_label[blk] < 0;
+                wp = (grp == 0 ? (party ? a.W0[1] : a.W0[0])
+                               : grp == 1 ? (party ? a.W1[1] : a.W1[0]) : (party ? a.W2g[1] : a.W2g[0])) +
+                     (size_t)neuron * a.ldw;
+            }
+            o = (long long)row * a.K;
+        }
+        s_wrow[tid] = wp;
+        s_orow[tid] = o;
+        s_dead[tid] = dead ? 1 : 0;
+    }
+    __syncthreads();
     {
         const int kk = (tid & 15) * 2;
         const int k = kb * KC + kk;
@@ -199,42 +233,31 @@ limb_open_kernel(LimbOpenArgs a) {
             const int sb = k / a.bs;
             ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
         }
-        // down: the strip of W that holds compact contraction indices ks, ks+1
-        const int kcol = a.down && k < a.K ? a.ids[ks / a.bs] * a.bs + (ks % a.bs) : 0;
+        // down: the strip of W that holds compact contraction indices ks, ks+1, and whether its block is in use
+        int kcol = k;
+        bool dead_k = false;
+        if (a.down && k < a.K) {
+            const int blk = ks / a.bs;
+            kcol = __ldg(a.ids + blk) * a.bs + (ks - blk * a.bs);
+            dead_k = a.blk_label && a.blk_label[blk] < 0;     // a block without a non-zero column of X
+        }
         // First every load of this thread's four rows is issued (eight 16-byte requests in flight per thread), then
-        // the words are used: the kernel is bound by memory latency otherwise.  Shares and triples are read once per
-        // product: streaming loads, so that the messages and planes written here are still in L2 when the next
-        // kernel reads them.
+        // the words are used.  Shares and triples are read once per product: streaming loads, so that the messages
+        // and planes written here are still in L2 when the next kernel reads them.
         constexpr int ITERS = PREP_ROWS / 16;
         ulonglong2 w[ITERS], b[ITERS];
         size_t off[ITERS];
         bool live[ITERS], dead[ITERS];
 #pragma unroll
         for (int it = 0; it < ITERS; ++it) {
-            int row = row0 + it * 16 + (tid >> 4);
-            live[it] = row < a.rows && k < a.K;
-            dead[it] = false;
+            const int r = it * 16 + (tid >> 4);
+            const u64* wp = s_wrow[r];
+            live[it] = wp != nullptr && k < a.K;
+            dead[it] = dead_k || s_dead[r] != 0;
             w[it] = b[it] = make_ulonglong2(0ull, 0ull);
-            off[it] = 0;
+            off[it] = (size_t)s_orow[r] + ks;
             if (live[it]) {
-                const u64* wsrc;
-                if (a.col_map) {
-                    const int sb = row / a.bs;
-                    row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
-                }
-                if (a.down) {
-                    dead[it] = a.blk_label && a.blk_label[ks / a.bs] < 0;     // a block without a non-zero column of X
-                    wsrc = (party ? a.W0[1] : a.W0[0]) + (size_t)row * a.ldw + kcol;
-                } else {
-                    const int grp = row / a.n, j = row - grp * a.n;
-                    const int neuron = a.ids[j / a.bs] * a.bs + (j % a.bs);
-                    dead[it] = a.blk_label && a.blk_label[j / a.bs] < 0;
-                    wsrc = (grp == 0 ? (party ? a.W0[1] : a.W0[0])
-                                     : grp == 1 ? (party ? a.W1[1] : a.W1[0]) : (party ? a.W2g[1] : a.W2g[0])) +
-                           (size_t)neuron * a.ldw + k;
-                }
-                off[it] = (size_t)row * a.K + ks;
-                w[it] = __ldcs(reinterpret_cast<const ulonglong2*>(wsrc));
+                w[it] = __ldcs(reinterpret_cast<const ulonglong2*>(wp + kcol));
                 b[it] = __ldcs(reinterpret_cast<const ulonglong2*>(Bi + off[it]));
             }
         }
@@ -1050,7 +1073,7 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                 zrow = (sg.party ? a.Z[1] : a.Z[0]) + (size_t)row * a.N + col0;
 #pragma unroll
             for (int h = 0; h < 32 / OUT_COLS; ++h) {          // this thread's 32 columns, OUT_COLS at a time
-                ptx::bulk_wait_group_read0();                  // the previous reduction has read this thread's staging row
+                u64 v[OUT_COLS];
 #pragma unroll
                 for (int c = 0; c < OUT_COLS / 8; ++c) {
                     uint32_t d[PLANES][8];
@@ -1058,19 +1081,19 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                     for (int s = 0; s < PLANES; ++s) ptx::tmem_ld8(lane_base + BN * s + h * OUT_COLS + c * 8, d[s]);
                     ptx::tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 8; j += 2) {
-                        const u64 v0 = limb_recombine(d[0][j], d[1][j], d[2][j], d[3][j], d[4][j], d[5][j], d[6][j],
+                    for (int j = 0; j < 8; ++j)
+                        v[c * 8 + j] = limb_recombine(d[0][j], d[1][j], d[2][j], d[3][j], d[4][j], d[5][j], d[6][j],
                                                       d[7][j]);
-                        const u64 v1 = limb_recombine(d[0][j + 1], d[1][j + 1], d[2][j + 1], d[3][j + 1], d[4][j + 1],
-                                                      d[5][j + 1], d[6][j + 1], d[7][j + 1]);
-                        *reinterpret_cast<ulonglong2*>(my_row + (c * 8 + j) * 8) = make_ulonglong2(v0, v1);
-                    }
                 }
                 if (h == 32 / OUT_COLS - 1) {
-                    // every accumulator has been read: hand TMEM back before the reduction traffic of this round
+                    // every accumulator has been read: hand TMEM back before anything that waits on the copy engine
                     ptx::fence_before_sync();
                     ptx::mbar_arrive(ptx::smem_u32(&accum_empty_bar));
                 }
+                ptx::bulk_wait_group_read0();                  // the previous reduction has read this thread's staging row
+#pragma unroll
+                for (int j = 0; j < OUT_COLS; j += 2)
+                    *reinterpret_cast<ulonglong2*>(my_row + j * 8) = make_ulonglong2(v[j], v[j + 1]);
                 int cols = a.N - col0 - h * OUT_COLS;
                 if (cols > OUT_COLS) cols = OUT_COLS;
                 if (row < a.M && cols > 0) {

@@ -25,13 +25,13 @@ struct PartyOut {
 // ranks each active block inside its warp, a shuffle scan over the 32 warp
 // totals gives each warp's base, and a running base carries across chunks.
 // `count` points at two words {count, error flag}; both are also written to
-// `host_report` (mapped host memory) so that the host needs no copy, followed
-// by `ticket` in host_report[2]: the host may watch that word instead of
-// waiting for the stream.
+// `host_report` (mapped host memory, or null when the host needs no report) so
+// that the host needs no copy, followed by `ticket` in host_report[2]: the host
+// may watch that word instead of waiting for the stream.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids, int32_t* __restrict__ count,
-                    int32_t* __restrict__ host_report, int32_t ticket) {
+__device__ __forceinline__ void compact_mask_body(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids,
+                                                  int32_t* __restrict__ count, int32_t* __restrict__ host_report,
+                                                  int32_t ticket) {
     __shared__ int warp_excl[32];
     __shared__ int chunk_total;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -61,6 +61,7 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
     }
     if (threadIdx.x == 0) {
         *count = running;
+        if (host_report == nullptr) return;    // the host counted the mask itself and does not wait for this report
         // {count, error flag raised by an earlier kernel's bounded wait} for the host, in mapped pinned memory
         host_report[0] = running;
         host_report[1] = count[1];
@@ -68,6 +69,29 @@ compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restric
         *reinterpret_cast<volatile int32_t*>(host_report + 2) = ticket;
         __threadfence_system();
     }
+}
+
+__global__ void __launch_bounds__(1024)
+compact_mask_kernel(const uint8_t* __restrict__ mask, int nb, int32_t* __restrict__ ids, int32_t* __restrict__ count,
+                    int32_t* __restrict__ host_report, int32_t ticket) {
+    pdl_wait();
+    pdl_launch_dependents();
+    compact_mask_body(mask, nb, ids, count, host_report, ticket);
+}
+
+// The same with the mask bytes passed in the kernel's parameter block: a mask the host holds (the public sparsity
+// distribution, one byte per block) needs no copy to the device at all while it fits there.
+struct MaskBytes {
+    static constexpr int CAPACITY = 3584;
+    uint8_t bytes[CAPACITY];
+};
+
+__global__ void __launch_bounds__(1024)
+compact_mask_arg_kernel(const __grid_constant__ MaskBytes mask, int nb, int32_t* __restrict__ ids,
+                        int32_t* __restrict__ count, int32_t* __restrict__ host_report, int32_t ticket) {
+    pdl_wait();
+    pdl_launch_dependents();
+    compact_mask_body(mask.bytes, nb, ids, count, host_report, ticket);
 }
 
 // ---------------------------------------------------------------------------
