@@ -266,7 +266,7 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     }
     a.emit_f = limb_few(pr) ? 1 : 0;       // few-token products read the messages as planes (no plane of their sum)
     a.left_pairs = left ? (long long)pr.M * pr.K / 2 : 0;
-    a.left_blocks = left ? ew_grid(c, a.left_pairs, 256) : 0;
+    a.left_blocks = left ? ew_grid(c, a.left_pairs, lb::OPEN_THREADS) : 0;
     a.ids = c->d_ids;
     a.n = c->n_active;
     a.bs = c->cfg.block;
@@ -282,12 +282,23 @@ int limb_open(comet_ctx* c, const Proj& pr, bool left, bool right, cudaStream_t 
     a.blk_label = c->tmask_set ? c->d_blk_label : nullptr;
     a.col_map = (!pr.down && c->grouped) ? c->d_col_map : nullptr;
     a.kmap = (pr.down && c->grouped) ? c->d_kmap : nullptr;
-    const int right_tiles = right ? kb * ceil_div(pr.N, lb::PREP_ROWS) : 0;
+    // right CTAs: 32 rows x kb_per_cta k-blocks each, over whole plane tiles (rows past the operand are zero planes);
+    // enough k-blocks per CTA for the copies of one to fly under the work on another, enough CTAs to fill the device
+    const int row_tiles = right ? ceil_div(pr.N, a.right_tile_rows) * (a.right_tile_rows / lb::OPEN_ROWS) : 0;
+    {
+        const long long fill = (long long)c->sm_count * 6;
+        long long per = fill > 0 ? 2ll * row_tiles * kb / fill : 1;
+        if (per < 1) per = 1;
+        if (per > lb::OPEN_MAX_KB_PER_CTA) per = lb::OPEN_MAX_KB_PER_CTA;
+        a.kb_per_cta = (int)per;
+        a.kchunks = ceil_div(kb, a.kb_per_cta);
+    }
+    const int right_tiles = row_tiles * a.kchunks;
     if (a.left_blocks + right_tiles == 0) return COMET_OK;
     if (right_tiles) c->f_as_planes[pr.down ? 1 : 0] = a.emit_f != 0;
-    const size_t smem = right_tiles ? (a.emit_f ? 2 : 1) * sizeof(comet::LimbTile) : 0;
-    COMET_CUDA(c, launch_chained(comet::limb_open_kernel, dim3(2 * (a.left_blocks + right_tiles)), dim3(256), smem,
-                                 stream, nullptr, a));
+    const size_t smem = right_tiles ? lb::OPEN_SMEM_BYTES : 0;
+    COMET_CUDA(c, launch_chained(comet::limb_open_kernel, dim3(2 * (a.left_blocks + right_tiles)),
+                                 dim3(lb::OPEN_THREADS), smem, stream, nullptr, a));
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;

@@ -38,6 +38,16 @@ constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <
 constexpr int EPI_WARPS = 8;                      // warp w drains TMEM lanes 32*(w%4).., columns 32*(w/4)..
 constexpr int THREADS = 32 * (EPI_WARPS + 2);     // warps 0-7 epilogue, warp 8 copy producer, warp 9 MMA issuer
 constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
+// The opening kernel streams tiles of 32 rows x one k-block of the weight share and of the triple share through a
+// two-stage ring in shared memory (asynchronous 16-byte copies, which hold no registers while in flight), several
+// consecutive k-blocks per CTA: the copies of the next k-block fly while the current one is turned into the message
+// and the planes.
+constexpr int OPEN_ROWS = 32, OPEN_THREADS = 128, OPEN_STAGES = 2;
+constexpr int OPEN_STRIDE = KC + 2;               // words per staged row: 272 bytes keep every row 16-byte aligned and
+                                                  // the 16-byte reads of eight consecutive rows on distinct banks
+constexpr int OPEN_TILE_BYTES = OPEN_ROWS * OPEN_STRIDE * 8;
+constexpr size_t OPEN_SMEM_BYTES = (size_t)OPEN_STAGES * 2 * OPEN_TILE_BYTES;      // a W and a B tile per stage: 34 KiB
+constexpr int OPEN_MAX_KB_PER_CTA = 8;
 constexpr int OUT_COLS = 16;                      // words per staged output row (a thread's 32 go in two rounds)
 constexpr int OUT_ROW_BYTES = OUT_COLS * 8 + 16;  // padded against bank conflicts
 constexpr size_t SMEM_BYTES = (size_t)STAGES * (A_BLOCK_BYTES + B_BLOCK_BYTES) + (size_t)EPI_WARPS * 32 * OUT_ROW_BYTES + 128;
@@ -93,6 +103,41 @@ __device__ __forceinline__ void limb_emit_planes(const LimbTile& src, int r, int
         *reinterpret_cast<uint4*>(blk + limb::block_offset(tile_rows, p, rin, half * 16)) = plane[p];
 }
 
+// The same for 16 consecutive words at `src` (16-byte aligned, shared memory).
+__device__ __forceinline__ void limb_emit_planes16(const u64* src, int half, uint8_t* blk, int tile_rows, int rin) {
+    unsigned lo[16], hi[16];
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(src + j);
+        lo[j] = (unsigned)v.x;
+        hi[j] = (unsigned)(v.x >> 32);
+        lo[j + 1] = (unsigned)v.y;
+        hi[j + 1] = (unsigned)(v.y >> 32);
+    }
+    uint4 plane[8];
+    limb_transpose4(lo[0], lo[1], lo[2], lo[3], plane[0].x, plane[1].x, plane[2].x, plane[3].x);
+    limb_transpose4(lo[4], lo[5], lo[6], lo[7], plane[0].y, plane[1].y, plane[2].y, plane[3].y);
+    limb_transpose4(lo[8], lo[9], lo[10], lo[11], plane[0].z, plane[1].z, plane[2].z, plane[3].z);
+    limb_transpose4(lo[12], lo[13], lo[14], lo[15], plane[0].w, plane[1].w, plane[2].w, plane[3].w);
+    limb_transpose4(hi[0], hi[1], hi[2], hi[3], plane[4].x, plane[5].x, plane[6].x, plane[7].x);
+    limb_transpose4(hi[4], hi[5], hi[6], hi[7], plane[4].y, plane[5].y, plane[6].y, plane[7].y);
+    limb_transpose4(hi[8], hi[9], hi[10], hi[11], plane[4].z, plane[5].z, plane[6].z, plane[7].z);
+    limb_transpose4(hi[12], hi[13], hi[14], hi[15], plane[4].w, plane[5].w, plane[6].w, plane[7].w);
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
+        *reinterpret_cast<uint4*>(blk + limb::block_offset(tile_rows, p, rin, half * 16)) = plane[p];
+}
+
+// 16-byte asynchronous copy global -> shared that bypasses L1; with `bytes` = 0 nothing is read and the 16 bytes
+// are filled with zeros.  (The form that also carries an L2 cache-policy operand raised an illegal-instruction
+// error on this part when combined with the byte count, so no eviction hint is given here.)
+__device__ __forceinline__ void limb_copy16_async(uint32_t dst_smem, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void limb_copy_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void limb_copy_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
 __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows, int row, int kblocks, int kb,
                                                    int* rin) {
     const int tile = row >> (31 - __clz(tile_rows));          // tile_rows is 32, 64 or 128
@@ -107,9 +152,11 @@ __device__ __forceinline__ uint8_t* limb_block_ptr(uint8_t* base, int tile_rows,
 //                 own B_i (it is in registers anyway, so it is not read a second time later).
 // gather: up   (down = 0): row c of the right operand is row neuron(c) of W (whole rows of `ldw` words);
 //         down (down = 1): contraction index c is column neuron(c) of W (strips of `bs` words in every row).
-// grid = 2 * (left_blocks + kblocks * ceil(rows / 64)), 256 threads, the party being the lowest bit of the block
-// index (both parties' messages are then written in the same order, which the next kernel reads backwards);
-// dynamic shared memory: one LimbTile when there are right tiles, two with emit_f.
+// grid = 2 * (left_blocks + row_tiles * kchunks), 128 threads, the party being the lowest bit of the block index
+// (both parties' messages are then written in the same order, which the next kernel reads backwards).  A right CTA
+// owns 32 rows and kb_per_cta consecutive k-blocks: while it turns one k-block into the message and the planes, the
+// loads of the next one are in flight (the kernel is bound by memory latency, not by bandwidth, when a CTA loads,
+// waits and works in turn).  Dynamic shared memory: OPEN_SMEM_BYTES when there are right tiles.
 // ---------------------------------------------------------------------------
 struct LimbOpenArgs {
     const u64* X[2];
@@ -128,6 +175,7 @@ struct LimbOpenArgs {
     int rows, K;             // logical size of the right operand [rows, K]
     int ldw;                 // words per row of W
     int kblocks, down;
+    int kb_per_cta, kchunks; // k-blocks per right CTA and CTAs per row tile: kchunks = ceil(kblocks / kb_per_cta)
     int right_tile_rows;     // rows per plane tile of the right operand: 64, or 128 for the few-token kernel
     // Protocol 3 with per-column row sets: per-token mask over the active blocks, [rows of X, tmask_ld] bytes, or
     // null.  Where it is zero the entry of X is no non-zero: it is not opened and E_i is zero there.
@@ -153,7 +201,7 @@ struct LimbOpenArgs {
     int emit_f;
 };
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(limb::OPEN_THREADS)
 limb_open_kernel(LimbOpenArgs a) {
     using namespace limb;
     pdl_wait();
@@ -165,8 +213,8 @@ limb_open_kernel(LimbOpenArgs a) {
         const ulonglong2* __restrict__ x = reinterpret_cast<const ulonglong2*>(party ? a.X[1] : a.X[0]);
         const ulonglong2* __restrict__ m = reinterpret_cast<const ulonglong2*>(party ? a.A[1] : a.A[0]);
         ulonglong2* __restrict__ e = reinterpret_cast<ulonglong2*>(party ? a.E[1] : a.E[0]);
-        const long long stride = (long long)a.left_blocks * 256;
-        for (long long t = (long long)bid * 256 + tid; t < a.left_pairs; t += stride) {
+        const long long stride = (long long)a.left_blocks * OPEN_THREADS;
+        for (long long t = (long long)bid * OPEN_THREADS + tid; t < a.left_pairs; t += stride) {
             if (a.tmask) {
                 const unsigned word = (unsigned)(2 * t), row = word / (unsigned)a.K, col = word - row * (unsigned)a.K;
                 if (a.tmask[(size_t)row * a.tmask_ld + col / (unsigned)a.bs] == 0) {
@@ -183,21 +231,20 @@ limb_open_kernel(LimbOpenArgs a) {
         }
         return;
     }
-    extern __shared__ __align__(16) uint8_t open_smem[];
-    LimbTile& sB = *reinterpret_cast<LimbTile*>(open_smem);
-    LimbTile& sF = *reinterpret_cast<LimbTile*>(open_smem + sizeof(LimbTile));      // only with emit_f
+    extern __shared__ __align__(16) uint8_t open_smem[];      // [stage][W tile | B tile], rows of OPEN_STRIDE words
     const int tile_id = bid - a.left_blocks;
-    const int kb = tile_id % a.kblocks;
-    const int row0 = (tile_id / a.kblocks) * PREP_ROWS;
+    const int chunk = tile_id % a.kchunks;
+    const int row0 = (tile_id / a.kchunks) * OPEN_ROWS;
+    const int kb0 = chunk * a.kb_per_cta;
+    const int kb1 = min(kb0 + a.kb_per_cta, a.kblocks);
     const u64* __restrict__ Bi = party ? a.B[1] : a.B[0];
     u64* __restrict__ Fi = party ? a.F[1] : a.F[0];
     // What depends on the row alone (which row of which weight matrix is gathered, where the row lies in B_i / F_i,
-    // whether its block is in use) is worked out once per row, by one thread, and shared: the index arithmetic
-    // would otherwise be repeated by the sixteen threads of every row and make the kernel instruction-bound.
-    __shared__ const u64* s_wrow[PREP_ROWS];          // first word of the gathered row of W_i; null: no such row
-    __shared__ long long s_orow[PREP_ROWS];           // offset of the row in B_i and F_i
-    __shared__ unsigned char s_dead[PREP_ROWS];
-    if (tid < PREP_ROWS) {
+    // whether its block is in use) is worked out once per row and shared.
+    __shared__ const u64* s_wrow[OPEN_ROWS];          // first word of the gathered row of W_i; null: no such row
+    __shared__ long long s_orow[OPEN_ROWS];           // offset of the row in B_i and F_i
+    __shared__ unsigned char s_dead[OPEN_ROWS];
+    if (tid < OPEN_ROWS) {
         int row = row0 + tid;
         const u64* wp = nullptr;
         long long o = 0;
@@ -225,64 +272,87 @@ limb_open_kernel(LimbOpenArgs a) {
         s_dead[tid] = dead ? 1 : 0;
     }
     __syncthreads();
-    {
-        const int kk = (tid & 15) * 2;
-        const int k = kb * KC + kk;
-        int ks = k;                                   // compact contraction index of plane position k
+
+    // This thread's part of every tile: the 16-byte column c16 (contraction indices 2 c16, 2 c16 + 1 of the k-block)
+    // of the rows rbase, rbase + 8, rbase + 16, rbase + 24.
+    const int c16 = tid & 15, rbase = tid >> 4;
+
+    // contraction index of this thread's column in k-block kb: plane position k, compact index ks, column kcol of the
+    // gathered row of W_i, and whether the block it belongs to is in use (down only)
+    auto column = [&](int kb, int& k, int& ks, int& kcol, bool& dead_k) {
+        k = kb * KC + 2 * c16;
+        ks = k;
         if (a.kmap && k < a.K) {
             const int sb = k / a.bs;
             ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
         }
-        // down: the strip of W that holds compact contraction indices ks, ks+1, and whether its block is in use
-        int kcol = k;
-        bool dead_k = false;
+        kcol = k;
+        dead_k = false;
         if (a.down && k < a.K) {
             const int blk = ks / a.bs;
             kcol = __ldg(a.ids + blk) * a.bs + (ks - blk * a.bs);
             dead_k = a.blk_label && a.blk_label[blk] < 0;     // a block without a non-zero column of X
         }
-        // First every load of this thread's four rows is issued (eight 16-byte requests in flight per thread), then
-        // the words are used.  Shares and triples are read once per product: streaming loads, so that the messages
-        // and planes written here are still in L2 when the next kernel reads them.
-        constexpr int ITERS = PREP_ROWS / 16;
-        ulonglong2 w[ITERS], b[ITERS];
-        size_t off[ITERS];
-        bool live[ITERS], dead[ITERS];
+    };
+    // asynchronous 16-byte copies of this thread's part of k-block kb into a stage; what lies outside the operand
+    // is filled with zeros
+    const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(open_smem);
+    auto issue = [&](int kb, int stage) {
+        int k, ks, kcol;
+        bool dead_k;
+        column(kb, k, ks, kcol, dead_k);
+        const uint32_t w_tile = smem0 + (uint32_t)stage * 2u * OPEN_TILE_BYTES, b_tile = w_tile + OPEN_TILE_BYTES;
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            const int r = it * 16 + (tid >> 4);
+        for (int i = 0; i < OPEN_ROWS / 8; ++i) {
+            const int r = rbase + 8 * i;
             const u64* wp = s_wrow[r];
-            live[it] = wp != nullptr && k < a.K;
-            dead[it] = dead_k || s_dead[r] != 0;
-            w[it] = b[it] = make_ulonglong2(0ull, 0ull);
-            off[it] = (size_t)s_orow[r] + ks;
-            if (live[it]) {
-                w[it] = __ldcs(reinterpret_cast<const ulonglong2*>(wp + kcol));
-                b[it] = __ldcs(reinterpret_cast<const ulonglong2*>(Bi + off[it]));
-            }
+            const bool live = wp != nullptr && k < a.K;
+            const uint32_t at = (uint32_t)(r * OPEN_STRIDE * 8 + c16 * 16);
+            limb_copy16_async(w_tile + at, live ? (const void*)(wp + kcol) : (const void*)Bi, live ? 16u : 0u);
+            limb_copy16_async(b_tile + at, live ? (const void*)(Bi + s_orow[r] + ks) : (const void*)Bi, live ? 16u : 0u);
         }
+        limb_copy_commit();
+    };
+
+    issue(kb0, 0);
+    for (int kb = kb0; kb < kb1; ++kb) {
+        const int stage = (kb - kb0) & 1;
+        if (kb + 1 < kb1) {
+            issue(kb + 1, stage ^ 1);        // that stage was released by the barrier that ended the last round
+            limb_copy_wait<1>();
+        } else {
+            limb_copy_wait<0>();
+        }
+        __syncthreads();                     // every thread's copies of this stage have landed
+        u64* w_tile = reinterpret_cast<u64*>(open_smem + (size_t)stage * 2 * OPEN_TILE_BYTES);
+        u64* b_tile = w_tile + OPEN_ROWS * OPEN_STRIDE;
+        int k, ks, kcol;
+        bool dead_k;
+        column(kb, k, ks, kcol, dead_k);
+        // the message F_i = gather(W_i) - B_i: written as words, or left in place of the W tile for the planes
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            const int r = it * 16 + (tid >> 4);
-            const u64 f0 = dead[it] ? 0ull : w[it].x - b[it].x;
-            const u64 f1 = dead[it] ? 0ull : w[it].y - b[it].y;
-            if (live[it] && !a.emit_f) *reinterpret_cast<ulonglong2*>(Fi + off[it]) = make_ulonglong2(f0, f1);
-            sB[r][kk] = b[it].x;
-            sB[r][kk + 1] = b[it].y;
-            if (a.emit_f) {
-                sF[r][kk] = f0;
-                sF[r][kk + 1] = f1;
-            }
+        for (int i = 0; i < OPEN_ROWS / 8; ++i) {
+            const int r = rbase + 8 * i;
+            const bool live = s_wrow[r] != nullptr && k < a.K;
+            const bool dead = dead_k || s_dead[r] != 0;
+            ulonglong2* wv = reinterpret_cast<ulonglong2*>(w_tile + r * OPEN_STRIDE + 2 * c16);
+            const ulonglong2 w = *wv;
+            const ulonglong2 b = *reinterpret_cast<const ulonglong2*>(b_tile + r * OPEN_STRIDE + 2 * c16);
+            const ulonglong2 f = dead ? make_ulonglong2(0ull, 0ull) : make_ulonglong2(w.x - b.x, w.y - b.y);
+            if (a.emit_f) *wv = f;
+            else if (live) *reinterpret_cast<ulonglong2*>(Fi + s_orow[r] + ks) = f;
         }
+        if (a.emit_f) __syncthreads();       // the planes of F_i are built from words other threads wrote
+        // planes of B_i (threads 0-63) and, with emit_f, of F_i (threads 64-127): 16 words of one row each
+        const int which = tid >> 6, half = (tid >> 5) & 1, r = tid & 31;
+        if (which == 0 || a.emit_f) {
+            int rin;
+            uint8_t* blk = limb_block_ptr(which ? (party ? a.Fpl[1] : a.Fpl[0]) : (party ? a.Bpl[1] : a.Bpl[0]),
+                                          a.right_tile_rows, row0 + r, a.kblocks, kb, &rin);
+            limb_emit_planes16((which ? w_tile : b_tile) + r * OPEN_STRIDE + half * 16, half, blk, a.right_tile_rows, rin);
+        }
+        __syncthreads();                     // the stage may be overwritten by the copies issued next round
     }
-    __syncthreads();
-    const int which = tid >> 7;                       // 0: planes of B_i, 1: planes of F_i
-    if (which == 1 && !a.emit_f) return;
-    const int half = (tid >> 6) & 1, r = tid & 63;
-    int rin;
-    uint8_t* blk = limb_block_ptr(which ? (party ? a.Fpl[1] : a.Fpl[0]) : (party ? a.Bpl[1] : a.Bpl[0]),
-                                  a.right_tile_rows, row0 + r, a.kblocks, kb, &rin);
-    limb_emit_planes(which ? sF : sB, r, half, blk, a.right_tile_rows, rin);
 }
 
 // Blocked limb planes back to words: out[row, k] for a [rows, K] operand whose plane tiles have `tile_rows` rows.
