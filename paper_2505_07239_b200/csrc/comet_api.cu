@@ -337,15 +337,28 @@ int limb_prep(comet_ctx* c, const Proj& pr, bool left, bool right, bool copy, cu
     a.tmask = (pr.down && c->tmask_set) ? c->d_tmask : nullptr;
     a.tmask_ld = c->n_active_blocks;
     a.bs = c->cfg.block;
-    a.left_tiles = left ? kb * ceil_div(a.M, lb::PREP_ROWS) : 0;
+    // tile CTAs: 32 rows x kb_per_cta k-blocks each, over whole plane tiles (rows past the operand are zero planes)
+    const int left_rows32 = left ? ceil_div(a.M, a.left_tile_rows) * (a.left_tile_rows / lb::OPEN_ROWS) : 0;
     // few-token products take the planes of the two messages as limb_open_kernel wrote them
-    a.right_tiles = (right && !limb_few(pr)) ? kb * ceil_div(a.N, lb::PREP_ROWS) : 0;
+    const int right_rows32 = (right && !limb_few(pr))
+                                 ? ceil_div(a.N, a.right_tile_rows) * (a.right_tile_rows / lb::OPEN_ROWS) : 0;
+    {
+        const long long fill = (long long)c->sm_count * 4;
+        long long per = fill > 0 ? 2ll * (left_rows32 + right_rows32) * kb / fill : 1;
+        if (per < 1) per = 1;
+        if (per > lb::OPEN_MAX_KB_PER_CTA) per = lb::OPEN_MAX_KB_PER_CTA;
+        a.kb_per_cta = (int)per;
+        a.kchunks = ceil_div(kb, a.kb_per_cta);
+    }
+    a.left_tiles = left_rows32 * a.kchunks;
+    a.right_tiles = right_rows32 * a.kchunks;
     a.copy_pairs = copy ? (long long)pr.M * pr.N / 2 : 0;
-    a.copy_blocks = copy ? ew_grid(c, a.copy_pairs, 256) : 0;
+    a.copy_blocks = copy ? ew_grid(c, a.copy_pairs, lb::OPEN_THREADS) : 0;
     const int blocks = a.left_tiles + a.right_tiles + a.copy_blocks;
     if (blocks == 0) return COMET_OK;
-    const size_t smem = (left ? 2 : 1) * sizeof(comet::LimbTile);
-    COMET_CUDA(c, launch_chained(comet::limb_prep_kernel, dim3(2 * blocks), dim3(256), smem, stream, nullptr, a));
+    const size_t smem = (size_t)lb::OPEN_STAGES * (left ? 3 : 2) * lb::OPEN_TILE_BYTES;
+    COMET_CUDA(c, launch_chained(comet::limb_prep_kernel, dim3(2 * blocks), dim3(lb::OPEN_THREADS), smem, stream,
+                                 nullptr, a));
     c->stats.kernel_launches += 1;
     COMET_CUDA(c, cudaGetLastError());
     return COMET_OK;
@@ -570,6 +583,8 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
         ok = ok && cudaFuncSetAttribute(comet::limb_prep_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                         (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(comet::limb_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(lb::OPEN_STAGES * 3 * lb::OPEN_TILE_BYTES)) == cudaSuccess;
         ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;

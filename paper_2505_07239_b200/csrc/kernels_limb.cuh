@@ -37,7 +37,6 @@ constexpr int STAGES = 3;
 constexpr int MAX_SEGMENT_UNITS = 16384 / KC;     // keeps the limb sums for s <= 3 below 2^32
 constexpr int EPI_WARPS = 8;                      // warp w drains TMEM lanes 32*(w%4).., columns 32*(w/4)..
 constexpr int THREADS = 32 * (EPI_WARPS + 2);     // warps 0-7 epilogue, warp 8 copy producer, warp 9 MMA issuer
-constexpr int PREP_ROWS = 64;                     // rows per CTA of the plane-building kernel
 // The opening kernel streams tiles of 32 rows x one k-block of the weight share and of the triple share through a
 // two-stage ring in shared memory (asynchronous 16-byte copies, which hold no registers while in flight), several
 // consecutive k-blocks per CTA: the copies of the next k-block fly while the current one is turned into the message
@@ -62,9 +61,9 @@ __host__ __device__ __forceinline__ int block_offset(int rows, int p, int r, int
 
 // ---------------------------------------------------------------------------
 // Blocked limb planes: helpers shared by the two memory-side kernels below.
-// A CTA tile is 64 rows x 32 contraction elements; words are staged in shared memory as [row][33] so that
-// the coalesced 16-byte global loads (16 threads per row) and the per-row 16-word reads of the byte
-// transposition are both conflict free.
+// A CTA tile is 32 rows x 32 contraction elements; words are staged in shared memory as [row][34], which keeps
+// every row 16-byte aligned for the asynchronous copies (16 threads per row) and puts the 16-byte reads of eight
+// consecutive rows, as the byte transposition issues them, on distinct banks.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void limb_transpose4(unsigned x0, unsigned x1, unsigned x2, unsigned x3,
                                                 unsigned& p0, unsigned& p1, unsigned& p2, unsigned& p3) {
@@ -76,34 +75,8 @@ __device__ __forceinline__ void limb_transpose4(unsigned x0, unsigned x1, unsign
     p3 = __byte_perm(t2, t3, 0x7632);
 }
 
-typedef u64 LimbTile[limb::PREP_ROWS][limb::KC + 1];
-
-// Split the 16 words src[r][16*half .. 16*half+15] into 8 limb planes of 16 bytes and store them at
+// Split the 16 words at `src` (16-byte aligned, shared memory) into 8 limb planes of 16 bytes and store them at
 // (plane, row `rin`, k = 16*half) of the block `blk`, whose tiles have `tile_rows` rows.
-__device__ __forceinline__ void limb_emit_planes(const LimbTile& src, int r, int half, uint8_t* blk, int tile_rows,
-                                                 int rin) {
-    unsigned lo[16], hi[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        const u64 v = src[r][half * 16 + j];
-        lo[j] = (unsigned)v;
-        hi[j] = (unsigned)(v >> 32);
-    }
-    uint4 plane[8];
-    limb_transpose4(lo[0], lo[1], lo[2], lo[3], plane[0].x, plane[1].x, plane[2].x, plane[3].x);
-    limb_transpose4(lo[4], lo[5], lo[6], lo[7], plane[0].y, plane[1].y, plane[2].y, plane[3].y);
-    limb_transpose4(lo[8], lo[9], lo[10], lo[11], plane[0].z, plane[1].z, plane[2].z, plane[3].z);
-    limb_transpose4(lo[12], lo[13], lo[14], lo[15], plane[0].w, plane[1].w, plane[2].w, plane[3].w);
-    limb_transpose4(hi[0], hi[1], hi[2], hi[3], plane[4].x, plane[5].x, plane[6].x, plane[7].x);
-    limb_transpose4(hi[4], hi[5], hi[6], hi[7], plane[4].y, plane[5].y, plane[6].y, plane[7].y);
-    limb_transpose4(hi[8], hi[9], hi[10], hi[11], plane[4].z, plane[5].z, plane[6].z, plane[7].z);
-    limb_transpose4(hi[12], hi[13], hi[14], hi[15], plane[4].w, plane[5].w, plane[6].w, plane[7].w);
-#pragma unroll
-    for (int p = 0; p < 8; ++p)
-        *reinterpret_cast<uint4*>(blk + limb::block_offset(tile_rows, p, rin, half * 16)) = plane[p];
-}
-
-// The same for 16 consecutive words at `src` (16-byte aligned, shared memory).
 __device__ __forceinline__ void limb_emit_planes16(const u64* src, int half, uint8_t* blk, int tile_rows, int rin) {
     unsigned lo[16], hi[16];
 #pragma unroll
@@ -377,7 +350,8 @@ limb_planes_to_words_kernel(const uint8_t* __restrict__ planes, u64* __restrict_
 //   left tiles : E = E_0 + E_1 -> planes(E);  V_i = A_i + i*E -> planes(V_i)      [M, K], 128-row blocks
 //   right tiles: F = F_0 + F_1 -> planes(F)                                      [N, K],  64-row blocks
 //   copy blocks: Z_i <- C_i (the accumulation target starts from the triple's C share)
-// grid = 2 * (kblocks * (ceil(M/64) + ceil(N/64)) + copy_blocks), 256 threads.  Any part may be empty.
+// grid = 2 * (left_tiles + right_tiles + copy_blocks), 128 threads; a tile CTA owns 32 rows x kb_per_cta k-blocks.
+// Any part may be empty.  Dynamic shared memory: 2 stages x (3 tiles with a left part, else 2) x OPEN_TILE_BYTES.
 // The party is the lowest bit of the block index: the two parties' CTAs of one tile read the same two messages and
 // run side by side, so the second read comes from L2.  Tiles are taken from the last to the first: the kernel before
 // this one wrote the messages in ascending order, and its last tiles are the ones most likely still in L2.
@@ -387,10 +361,11 @@ struct LimbPrepArgs {
     const u64* A[2];
     uint8_t* Epl[2];
     uint8_t* Vpl[2];
-    int M, left_tiles;       // left_tiles = kblocks * ceil(M / 64), or 0
+    int M, left_tiles;       // left_tiles = (32-row tiles of whole plane tiles) * kchunks, or 0
+    int kb_per_cta, kchunks; // k-blocks per tile CTA and CTAs per row tile: kchunks = ceil(kblocks / kb_per_cta)
     const u64* F0; const u64* F1;
     uint8_t* Fpl[2];
-    int N, right_tiles;      // right_tiles = kblocks * ceil(N / 64), or 0
+    int N, right_tiles;      // likewise for the right operand
     int K, kblocks;
     int left_tile_rows, right_tile_rows;   // rows per plane tile: 128 / 64, or 32 / 128 for the few-token kernel
     const uint8_t* tmask;    // per-token mask over the active blocks (see LimbOpenArgs), or null: where it is zero
@@ -408,7 +383,7 @@ struct LimbPrepArgs {
     const int32_t* kmap;
 };
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(limb::OPEN_THREADS)
 limb_prep_kernel(LimbPrepArgs a) {
     using namespace limb;
     pdl_wait();
@@ -422,78 +397,116 @@ limb_prep_kernel(LimbPrepArgs a) {
         id -= a.left_tiles + a.right_tiles;
         const ulonglong2* __restrict__ s = reinterpret_cast<const ulonglong2*>(party ? a.C[1] : a.C[0]);
         ulonglong2* __restrict__ d = reinterpret_cast<ulonglong2*>(party ? a.Z[1] : a.Z[0]);
-        const long long stride = (long long)a.copy_blocks * 256;
-        for (long long t = (long long)id * 256 + tid; t < a.copy_pairs; t += stride) d[t] = __ldcs(s + t);
+        const long long stride = (long long)a.copy_blocks * OPEN_THREADS;
+        for (long long t = (long long)id * OPEN_THREADS + tid; t < a.copy_pairs; t += stride) d[t] = __ldcs(s + t);
         return;
     }
-    extern __shared__ __align__(16) uint8_t prep_smem[];     // one tile (right/copy only) or two (left present)
-    LimbTile& sS = *reinterpret_cast<LimbTile*>(prep_smem);
-    LimbTile& sW = *reinterpret_cast<LimbTile*>(prep_smem + sizeof(LimbTile));
+    // A tile CTA owns 32 rows and kb_per_cta consecutive k-blocks and streams them through a two-stage ring of
+    // asynchronous copies, as the opening kernel does: per stage the two messages and, on the left, the party's A_i.
+    extern __shared__ __align__(16) uint8_t prep_smem[];     // [stage][message 0 | message 1 | (left) A_i]
     const bool left = id < a.left_tiles;
     if (!left) id -= a.left_tiles;
-    const int kb = id % a.kblocks;
-    const int row0 = (id / a.kblocks) * PREP_ROWS;
+    const int chunk = id % a.kchunks;
+    const int row0 = (id / a.kchunks) * OPEN_ROWS;
+    const int kb0 = chunk * a.kb_per_cta;
+    const int kb1 = min(kb0 + a.kb_per_cta, a.kblocks);
     const int rows = left ? a.M : a.N;
+    const int tiles_per_stage = left ? 3 : 2;
     const u64* __restrict__ in0 = left ? a.E0 : a.F0;
     const u64* __restrict__ in1 = left ? a.E1 : a.F1;
     const u64* __restrict__ own = party ? a.A[1] : a.A[0];
-    {
-        const int kk = (tid & 15) * 2;
-        const int k = kb * KC + kk;
-        int ks = k;                                   // compact contraction index of plane position k
+    __shared__ int s_row[OPEN_ROWS];                  // the row of the operands a tile row stands for; -1: none
+    if (tid < OPEN_ROWS) {
+        int row = row0 + tid;
+        if (row >= rows) {
+            row = -1;
+        } else if (left) {
+            if (a.row_map) row = __ldg(a.row_map + row);
+        } else if (a.col_map) {
+            const int sb = row / a.bs;
+            row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
+        }
+        s_row[tid] = row;
+    }
+    __syncthreads();
+
+    const int c16 = tid & 15, rbase = tid >> 4;
+    const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(prep_smem);
+    const uint32_t stage_bytes = (uint32_t)tiles_per_stage * OPEN_TILE_BYTES;
+    // plane position k of this thread's column in k-block kb and its compact contraction index ks
+    auto column = [&](int kb, int& k, int& ks) {
+        k = kb * KC + 2 * c16;
+        ks = k;
         if (a.kmap && k < a.K) {
             const int sb = k / a.bs;
             ks = __ldg(a.kmap + sb) * a.bs + (k - sb * a.bs);
         }
-        // every load of this thread's four rows first (up to twelve 16-byte requests in flight), then the sums
-        constexpr int ITERS = PREP_ROWS / 16;
-        ulonglong2 x[ITERS], y[ITERS], z[ITERS];
-        bool own_part[ITERS];                         // the party's A_i takes part at this position
+    };
+    auto issue = [&](int kb, int stage) {
+        int k, ks;
+        column(kb, k, ks);
+        const uint32_t t0 = smem0 + (uint32_t)stage * stage_bytes;
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            int row = row0 + it * 16 + (tid >> 4);
-            x[it] = y[it] = z[it] = make_ulonglong2(0ull, 0ull);
-            own_part[it] = false;
-            if (row < rows && k < a.K) {
-                if (left) {
-                    if (a.row_map) row = __ldg(a.row_map + row);
-                } else if (a.col_map) {
-                    const int sb = row / a.bs;
-                    row = __ldg(a.col_map + sb) * a.bs + (row - sb * a.bs);
-                }
-                const size_t o = (size_t)row * a.K + ks;
-                // the messages were written by the kernel before this one and are not read again on the path
-                x[it] = __ldcs(reinterpret_cast<const ulonglong2*>(in0 + o));
-                y[it] = __ldcs(reinterpret_cast<const ulonglong2*>(in1 + o));
-                // where the per-token mask is zero the party's A_i is no part of the triple and counts as zero
-                if (left && (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + ks / a.bs] != 0)) {
-                    own_part[it] = true;
-                    z[it] = __ldcs(reinterpret_cast<const ulonglong2*>(own + o));
-                }
-            }
+        for (int i = 0; i < OPEN_ROWS / 8; ++i) {
+            const int r = rbase + 8 * i;
+            const int row = s_row[r];
+            const bool live = row >= 0 && k < a.K;
+            const size_t o = live ? (size_t)row * a.K + ks : 0;
+            const uint32_t at = (uint32_t)(r * OPEN_STRIDE * 8 + c16 * 16);
+            limb_copy16_async(t0 + at, in0 + o, live ? 16u : 0u);
+            limb_copy16_async(t0 + OPEN_TILE_BYTES + at, in1 + o, live ? 16u : 0u);
+            if (left) limb_copy16_async(t0 + 2 * OPEN_TILE_BYTES + at, own + o, live ? 16u : 0u);
         }
+        limb_copy_commit();
+    };
+
+    issue(kb0, 0);
+    for (int kb = kb0; kb < kb1; ++kb) {
+        const int stage = (kb - kb0) & 1;
+        if (kb + 1 < kb1) {
+            issue(kb + 1, stage ^ 1);        // that stage was released by the barrier that ended the last round
+            limb_copy_wait<1>();
+        } else {
+            limb_copy_wait<0>();
+        }
+        __syncthreads();                     // every thread's copies of this stage have landed
+        u64* t_sum = reinterpret_cast<u64*>(prep_smem + (size_t)stage * stage_bytes);      // message 0, then the sum
+        u64* t_in1 = t_sum + OPEN_ROWS * OPEN_STRIDE;
+        u64* t_own = t_in1 + OPEN_ROWS * OPEN_STRIDE;                                       // A_i, then V_i (left)
+        int k, ks;
+        column(kb, k, ks);
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            const int r = it * 16 + (tid >> 4);
-            const u64 s0 = x[it].x + y[it].x, s1 = x[it].y + y[it].y;      // the exchange: both messages summed
-            sS[r][kk] = s0;
-            sS[r][kk + 1] = s1;
+        for (int i = 0; i < OPEN_ROWS / 8; ++i) {
+            const int r = rbase + 8 * i;
+            const int at = r * OPEN_STRIDE + 2 * c16;
+            ulonglong2* sv = reinterpret_cast<ulonglong2*>(t_sum + at);
+            const ulonglong2 x = *sv, y = *reinterpret_cast<const ulonglong2*>(t_in1 + at);
+            const ulonglong2 sum = make_ulonglong2(x.x + y.x, x.y + y.y);       // the exchange: both messages summed
+            *sv = sum;
             if (left) {
-                sW[r][kk] = own_part[it] ? z[it].x + (party ? s0 : 0ull) : 0ull;       // V_i = A_i + i*E
-                sW[r][kk + 1] = own_part[it] ? z[it].y + (party ? s1 : 0ull) : 0ull;
+                // where the per-token mask is zero the party's A_i is no part of the triple and counts as zero
+                const int row = s_row[r];
+                const bool own_part = row >= 0 && k < a.K &&
+                                      (!a.tmask || a.tmask[(size_t)row * a.tmask_ld + ks / a.bs] != 0);
+                ulonglong2* ov = reinterpret_cast<ulonglong2*>(t_own + at);
+                const ulonglong2 z = *ov;
+                *ov = own_part ? make_ulonglong2(z.x + (party ? sum.x : 0ull), z.y + (party ? sum.y : 0ull))   // V_i = A_i + i*E
+                               : make_ulonglong2(0ull, 0ull);
             }
         }
+        __syncthreads();                     // the planes are built from words other threads wrote
+        // threads 0-63: planes of the summed message; threads 64-127 (left only): planes of V_i; 16 words of a row each
+        const int which = tid >> 6, half = (tid >> 5) & 1, r = tid & 31;
+        if (which == 0 || left) {
+            const int tile_rows = left ? a.left_tile_rows : a.right_tile_rows;
+            uint8_t* base = left ? (which ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]))
+                                 : (party ? a.Fpl[1] : a.Fpl[0]);
+            int rin;
+            uint8_t* blk = limb_block_ptr(base, tile_rows, row0 + r, a.kblocks, kb, &rin);
+            limb_emit_planes16((which ? t_own : t_sum) + r * OPEN_STRIDE + half * 16, half, blk, tile_rows, rin);
+        }
+        __syncthreads();                     // the stage may be overwritten by the copies issued next round
     }
-    __syncthreads();
-    const int which = tid >> 7;                       // 0: the summed message, 1: the party's own operand
-    if (which == 1 && !left) return;
-    const int half = (tid >> 6) & 1, r = tid & 63;
-    const int tile_rows = left ? a.left_tile_rows : a.right_tile_rows;
-    uint8_t* base = left ? (which ? (party ? a.Vpl[1] : a.Vpl[0]) : (party ? a.Epl[1] : a.Epl[0]))
-                         : (party ? a.Fpl[1] : a.Fpl[0]);
-    int rin;
-    uint8_t* blk = limb_block_ptr(base, tile_rows, row0 + r, a.kblocks, kb, &rin);
-    limb_emit_planes(which ? sW : sS, r, half, blk, tile_rows, rin);
 }
 
 // ---------------------------------------------------------------------------
