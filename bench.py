@@ -39,8 +39,8 @@ L2_FLUSH_BYTES = 512 << 20
 # kernels_limb.cuh.
 COMBINE_LIMB_TRAFFIC = {
     "workload": ("opt1.3b", 0.9),
-    "kernel_sha256": "2b11a0e9ac0c4abc86695f6910f87b457e3c798c2c32f2706a7a40a5865b64d4",
-    "bytes_per_launch": 122312192,
+    "kernel_sha256": "0f2e1699f0109bf7b914f0fe698b6c08b30d5eb70620faf5cffb1cb7cfccd669",
+    "bytes_per_launch": 132884480,
 }
 
 
