@@ -1107,7 +1107,10 @@ __device__ __forceinline__ void combine_limb_body(const LimbArgs a) {
                     // instruction of N = 64*(8-p), cut at 256.  When a plane issues two instructions the second
                     // takes the left operand from the collector instead of shared memory.
 #pragma unroll
-                    for (int p = 0; p < PLANES; ++p) {
+                    for (int i = 0; i < PLANES; ++i) {
+                        // wide and narrow instructions alternate (plane 0, which overwrites every accumulator when a
+                        // segment starts, stays first)
+                        const int p = (i & 1) ? PLANES - 1 - (i >> 1) : (i >> 1);
                         const uint32_t ap = a_lo + ((p * BM * KC) >> 4);
                         const int n_total = BN * (PLANES - p);
                         const uint32_t acc_p = p == 0 ? acc : 1u;
