@@ -614,7 +614,7 @@ int comet_init(const comet_config* cfg, void* cuda_stream, comet_ctx** out) {
     ok = ok && cudaMemset(c->d_count, 0, 2 * sizeof(int32_t)) == cudaSuccess;
     if (ok) c->d_error = c->d_count + 1;
     ok = ok && cudaHostAlloc((void**)&c->h_count, 4 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
-    if (ok) c->h_count[2] = c->h_count[3] = 0;
+    if (ok) c->h_count[0] = c->h_count[1] = c->h_count[2] = c->h_count[3] = 0;     // pinned memory is not zeroed
     ok = ok && cudaHostGetDevicePointer((void**)&c->h_count_dev, c->h_count, 0) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
