@@ -60,6 +60,20 @@ def test_ragged_token_counts(hz, path, tokens):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("tokens", [5, 40, 140])
+def test_contraction_depths_that_end_inside_a_k_block(hz, path, tokens):
+    """d_model = 48 and n = 48 (three 16-neuron blocks): both projections contract over one and a half 32-deep
+    blocks, and 48 weight rows end inside a 64-row plane tile; with 5, 40 and 140 token rows the few-token kernel,
+    one ragged row tile and two row tiles are covered."""
+    cfg = wl.FFNConfig("ragged-k", tokens, 48, 160, 16, 14, False, 0.3, "uniform", "normal", "normal0.02")
+    m = np.zeros(cfg.n_blocks, np.uint8)
+    m[[1, 4, 9]] = 1
+    r = _ok(hz.run_and_compare_full(cfg, seed=41 + tokens, mask=m, matmul_path=path), path)
+    assert r["n_active"] == 48 and r["up_reconstructs"]
+    assert r["float64_max_abs_err"] < 2.0 ** -10
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_gated_small(hz, path):
     cfg = wl.FFNConfig("gated-small", 40, 128, 512, 64, 16, True, 0.25, "uniform", "normal", "normal0.02")
     r = _ok(hz.run_and_compare_full(cfg, seed=5, matmul_path=path), path)
